@@ -1,0 +1,234 @@
+"""Unit-scaled ops and the FFN block, forward and backward (test infrastructure, fp64).
+
+Each function is the paper's definition of the op evaluated in float64 on
+operands that have already been rounded to their storage format:
+
+  * scaled ops f* = alpha f, f*_grad_i = beta_i f_grad_i   (section "Scaled ops");
+  * matmul*, matmul*_grad_1, matmul*_grad_2                 (section "Example");
+  * gelu(x) = x Phi(x) with its scale factors               ("Table of unit scaling factors");
+  * fixed(tau) residual sqrt(1-tau) x + sqrt(tau) f(x) and the rewrite that
+    moves the backward factor to the branch entry           (section "Weighted addition");
+  * FP8 only on matmul inputs, E4 for activations / weights and E5 for
+    gradients, outputs in higher precision                  (sections "Mixed precision",
+    "Trade-offs of low-precision training").
+
+Scale factors arrive as the float32 constants the device library receives and
+are promoted to float64 before use.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+from scipy import special
+
+from . import formats as F
+from . import scales as S
+
+
+def _f32(c) -> float:
+    """The float32-rounded value of a scalar, as a Python float (double)."""
+    return float(np.float32(c))
+
+
+# --------------------------------------------------------------------------- linear
+
+def linear_fwd(X, W, alpha):
+    """matmul*(X, W) = alpha * X W;  X [b x m], W [m x n] -> [b x n]."""
+    return _f32(alpha) * (np.asarray(X, np.float64) @ np.asarray(W, np.float64))
+
+
+def linear_bwd_x(G, W, beta_x):
+    """matmul*_grad(X, W, G)_1 = beta_1 * G W^T;  G [b x n], W [m x n] -> [b x m]."""
+    return _f32(beta_x) * (np.asarray(G, np.float64) @ np.asarray(W, np.float64).T)
+
+
+def linear_bwd_w(X, G, beta_w):
+    """matmul*_grad(X, W, G)_2 = beta_2 * X^T G;  X [b x m], G [b x n] -> [m x n]."""
+    return _f32(beta_w) * (np.asarray(X, np.float64).T @ np.asarray(G, np.float64))
+
+
+# --------------------------------------------------------------------------- gelu
+
+def _Phi(z):
+    return 0.5 * special.erfc(-z / math.sqrt(2.0))      # = (1 + erf(z / sqrt 2)) / 2, accurate in the lower tail
+
+
+def _phi(z):
+    return np.exp(-0.5 * z * z) / math.sqrt(2.0 * math.pi)
+
+
+def gelu_fwd(H, s_in, alpha_g):
+    """A = alpha_g * gelu(s_in * H), gelu(x) = x Phi(x)."""
+    z = _f32(s_in) * np.asarray(H, np.float64)
+    return _f32(alpha_g) * z * _Phi(z)
+
+
+def gelu_bwd(H, dA, s_in, beta_g):
+    """dH = beta_g * s_in * gelu'(s_in * H) * dA, gelu'(x) = Phi(x) + x phi(x)."""
+    z = _f32(s_in) * np.asarray(H, np.float64)
+    return _f32(beta_g) * _f32(s_in) * (_Phi(z) + z * _phi(z)) * np.asarray(dA, np.float64)
+
+
+# --------------------------------------------------------------------------- residual
+
+def weighted_add(a, b, coef_a, coef_b):
+    """coef_a * a + coef_b * b with float32-rounded coefficients."""
+    return _f32(coef_a) * np.asarray(a, np.float64) + _f32(coef_b) * np.asarray(b, np.float64)
+
+
+def residual_add(skip, branch, tau):
+    """fixed(tau): sqrt(1 - tau) * skip + sqrt(tau) * branch.
+
+    The same expression serves the backward pass: the branch output receives the
+    incoming gradient unscaled, and the factor sqrt(tau) is applied where the
+    branch's input gradient rejoins the skip gradient.
+    """
+    ca, cb = S.residual_coefficients(tau)
+    return weighted_add(skip, branch, ca, cb)
+
+
+# --------------------------------------------------------------------------- storage rounding
+
+def store(v, dtype: str):
+    """Round float64 values to a storage format; returns (values float64, codes or None)."""
+    if dtype == "f64":          # no rounding: used by exact-arithmetic checks
+        return np.asarray(v, np.float64), None
+    if dtype == "f32":
+        with np.errstate(over="ignore"):
+            return np.asarray(v, np.float64).astype(np.float32).astype(np.float64), None
+    fmt = F.FORMATS[dtype]
+    q = F.quantise(v, fmt)
+    return q, F.encode(q, fmt)
+
+
+# --------------------------------------------------------------------------- fused epilogue
+
+@dataclass
+class Epilogue:
+    """What a linear call may fuse after the scaled accumulator.
+
+    act: "none" | "gelu" | "gelu_grad".  For "gelu" the pre-activation is stored
+    in `aux_dtype` (the copy the backward pass reads); for "gelu_grad" `aux`
+    holds that stored pre-activation.  skip: optional tensor combined as
+    skip_coef * skip + out_coef * value.
+    """
+
+    act: str = "none"
+    act_in_scale: float = 1.0
+    act_out_scale: float = 1.0
+    aux: np.ndarray | None = None
+    aux_dtype: str = "bf16"
+    skip: np.ndarray | None = None
+    skip_coef: float = 0.0
+    out_coef: float = 1.0
+
+
+def apply_epilogue(val, ep: Epilogue | None, out_dtype: str):
+    """Chain scaled accumulator -> activation -> residual -> one rounding to out_dtype.
+
+    Returns (out values, out codes or None, stored pre-activation values or None).
+    """
+    aux_saved = None
+    if ep is not None:
+        if ep.act == "gelu":
+            aux_saved, _ = store(val, ep.aux_dtype)
+            val = gelu_fwd(val, ep.act_in_scale, ep.act_out_scale)
+        elif ep.act == "gelu_grad":
+            val = gelu_bwd(ep.aux, val, ep.act_in_scale, ep.act_out_scale)
+        elif ep.act != "none":
+            raise ValueError(ep.act)
+        if ep.skip is not None:
+            val = weighted_add(ep.skip, val, ep.skip_coef, ep.out_coef)
+    out, codes = store(val, out_dtype)
+    return out, codes, aux_saved
+
+
+# --------------------------------------------------------------------------- FFN block
+
+@dataclass
+class FFNScales:
+    alpha1: float
+    alpha2: float
+    beta_x1: float
+    beta_x2: float
+    beta_w: float
+    alpha_g: float
+    beta_g: float
+    s_in: float = 1.0
+    tau: float = 0.5
+
+    @staticmethod
+    def unconstrained(T: int, d: int, f: int, tau: float = 0.5) -> "FFNScales":
+        a1, bx1, bw = S.linear_scales(T, d, f)
+        a2, bx2, _ = S.linear_scales(T, f, d)
+        ag, bg = S.gelu_scales()
+        return FFNScales(a1, a2, bx1, bx2, bw, ag, bg, 1.0, tau)
+
+    @staticmethod
+    def constrained(T: int, d: int, f: int, tau: float = 0.5) -> "FFNScales":
+        """alpha = beta_X for both matmuls and for gelu (the residual makes X a non-cut edge)."""
+        a1, bx1, bw = S.linear_scales(T, d, f, constrained=True)
+        a2, bx2, _ = S.linear_scales(T, f, d, constrained=True)
+        ag, bg = S.gelu_scales(constrained=True)
+        return FFNScales(a1, a2, bx1, bx2, bw, ag, bg, 1.0, tau)
+
+
+@dataclass
+class FFNResult:
+    Xq: np.ndarray = None
+    W1q: np.ndarray = None
+    W2q: np.ndarray = None
+    Gq: np.ndarray = None
+    H: np.ndarray = None        # stored pre-activation (values)
+    Aq: np.ndarray = None       # q_E4(alpha_g gelu(H)) values
+    Aq_codes: np.ndarray = None
+    R: np.ndarray = None        # block output
+    dHq: np.ndarray = None
+    dHq_codes: np.ndarray = None
+    dW2: np.ndarray = None
+    dW1: np.ndarray = None
+    dX: np.ndarray = None
+
+
+def ffn_block(X, W1, W2, G, sc: FFNScales, *, operand: str = "fp8",
+              h_dtype: str = "bf16", io_dtype: str = "bf16") -> FFNResult:
+    """Unit-scaled Transformer FFN with a fixed(tau) residual, forward and backward.
+
+    Forward:  H = alpha1 q(X) q(W1);  A = alpha_g gelu(s_in H);  Y = alpha2 q(A) q(W2);
+              R = sqrt(1-tau) X + sqrt(tau) Y.
+    Backward, G = dL/dR:  the branch output gradient is G itself;
+              dA = beta_x2 q(G) q(W2)^T;  dH = beta_g s_in gelu'(s_in H) dA;
+              dW2 = beta_w q(A)^T q(G);   dXb = beta_x1 q(dH) q(W1)^T;
+              dW1 = beta_w q(X)^T q(dH);  dX = sqrt(1-tau) G + sqrt(tau) dXb.
+    q is E4 for activations / weights and E5 for gradients when operand == "fp8";
+    for "bf16" / "fp16" every matmul input is rounded to that format instead, and
+    for "f64" nothing is rounded (pair it with h_dtype = io_dtype = "f64").
+    """
+    act_fmt = "e4m3" if operand == "fp8" else operand
+    grad_fmt = "e5m2" if operand == "fp8" else operand
+    r = FFNResult()
+    r.Xq, _ = store(np.asarray(X), act_fmt)
+    r.W1q, _ = store(np.asarray(W1), act_fmt)
+    r.W2q, _ = store(np.asarray(W2), act_fmt)
+    r.Gq, _ = store(np.asarray(G), grad_fmt)
+    c_skip, c_branch = S.residual_coefficients(sc.tau)
+
+    ep1 = Epilogue(act="gelu", act_in_scale=sc.s_in, act_out_scale=sc.alpha_g, aux_dtype=h_dtype)
+    r.Aq, r.Aq_codes, r.H = apply_epilogue(linear_fwd(r.Xq, r.W1q, sc.alpha1), ep1, act_fmt)
+    ep2 = Epilogue(skip=np.asarray(X, np.float64), skip_coef=c_skip, out_coef=c_branch)
+    r.R, _, _ = apply_epilogue(linear_fwd(r.Aq, r.W2q, sc.alpha2), ep2, io_dtype)
+
+    ep3 = Epilogue(act="gelu_grad", act_in_scale=sc.s_in, act_out_scale=sc.beta_g, aux=r.H)
+    r.dHq, r.dHq_codes, _ = apply_epilogue(linear_bwd_x(r.Gq, r.W2q, sc.beta_x2), ep3, grad_fmt)
+    r.dW2, _, _ = apply_epilogue(linear_bwd_w(r.Aq, r.Gq, sc.beta_w), None, "f32")
+    ep5 = Epilogue(skip=np.asarray(G, np.float64), skip_coef=c_skip, out_coef=c_branch)
+    r.dX, _, _ = apply_epilogue(linear_bwd_x(r.dHq, r.W1q, sc.beta_x1), ep5, io_dtype)
+    r.dW1, _, _ = apply_epilogue(linear_bwd_w(r.Xq, r.dHq, sc.beta_w), None, "f32")
+    return r
+
+
+def ffn_flops(T: int, d: int, f: int) -> float:
+    """Matmul FLOPs of one FFN block, forward + backward: two linear layers x 6 b m n."""
+    return 2 * 6.0 * T * d * f

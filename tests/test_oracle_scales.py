@@ -1,0 +1,85 @@
+"""Pins for the oracle's scale factors: the paper's table, closed forms, Monte Carlo."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import scales as S
+from tests.golden.load import load
+
+GOLD = load("paper_constants.txt")
+
+
+def test_matmul_factors_closed_form():
+    a, bx, bw = S.linear_scales(8192, 1024, 4096)
+    assert a == 2.0 ** -5 and bx == 2.0 ** -6 and math.isclose(bw, 1 / math.sqrt(8192), rel_tol=1e-15)
+    a, bx, bw = S.linear_scales(256, 128, 512, constrained=True)
+    assert math.isclose(a, (128 * 512) ** -0.25, rel_tol=1e-14) and a == bx and bw == 1 / 16
+
+
+def test_geometric_mean():
+    assert math.isclose(S.geometric_mean([2.0, 8.0]), 4.0, rel_tol=1e-15)
+    assert math.isclose(S.geometric_mean([1.0, 10.0, 100.0]), 10.0, rel_tol=1e-14)
+
+
+def test_integrator_on_relu_closed_form():
+    """The table gives relu analytically: alpha = sqrt(2 / (1 - 1/pi)), beta = sqrt(2)."""
+    a, b = S.relu_scales()
+    assert math.isclose(a, math.sqrt(2 / (1 - 1 / math.pi)), rel_tol=1e-10)
+    assert math.isclose(b, math.sqrt(2), rel_tol=1e-10)
+
+
+@pytest.mark.parametrize("name,fn,digits", [
+    ("gelu", S.gelu_scales, 3), ("tanh", S.tanh_scales, 3),
+])
+def test_printed_activation_constants(name, fn, digits):
+    a, b = fn()
+    assert round(a, digits) == GOLD[f"{name}_alpha"]
+    assert round(b, digits) == GOLD[f"{name}_beta"]
+
+
+def test_printed_sigmoid_constants_to_three_significant_digits():
+    # the table prints 4.802 / 4.722; quadrature gives 4.8013 / 4.7226, so only the
+    # first three significant digits of alpha are reproducible
+    a, b = S.sigmoid_scales()
+    assert abs(a - GOLD["sigmoid_alpha"]) < 1.5e-3 and round(b, 2) == round(GOLD["sigmoid_beta"], 2)
+
+
+def test_gelu_scales_by_monte_carlo():
+    z = np.random.default_rng(0).standard_normal(4_000_000)
+    a, b = S.gelu_scales()
+    assert abs(np.std(a * S.gelu(z)) - 1) < 5e-3
+    g = np.random.default_rng(1).standard_normal(z.size)
+    assert abs(np.std(b * S.gelu_grad(z) * g) - 1) < 5e-3
+
+
+def test_gelu_special_values_and_derivative():
+    assert S.gelu(np.float64(0.0)) == 0.0 and S.gelu_grad(np.float64(0.0)) == 0.5
+    assert math.isclose(S.gelu(np.float64(10.0)), 10.0, rel_tol=1e-15)
+    assert abs(S.gelu(np.float64(-10.0))) < 1e-20
+    x = np.linspace(-5, 5, 201)
+    h = 1e-5
+    fd = (S.gelu(x + h) - S.gelu(x - h)) / (2 * h)
+    assert np.max(np.abs(fd - S.gelu_grad(x))) < 1e-9
+    # independent closed form: Phi via erfc
+    assert np.allclose(S.gelu(x), 0.5 * x * np.array([math.erfc(-t / math.sqrt(2)) for t in x]), rtol=0, atol=1e-15)
+
+
+def test_constrained_gelu_is_geometric_mean():
+    a, b = S.gelu_scales()
+    c, c2 = S.gelu_scales(constrained=True)
+    assert c == c2 and math.isclose(c, math.sqrt(a * b), rel_tol=1e-14)
+
+
+def test_residual_coefficients_preserve_unit_variance():
+    for tau in (0.1, 0.5, 0.9):
+        ca, cb = S.residual_coefficients(tau)
+        assert math.isclose(ca * ca + cb * cb, 1.0, rel_tol=1e-15)
+    assert S.residual_coefficients(0.5) == (math.sqrt(0.5), math.sqrt(0.5))
+
+
+def test_flop_overhead_figures():
+    # (1/6)(1/b + 1/m + 1/n) <= 1 / (2 min(b, m, n)); BERT-large: 4 / (2 * 1024) ~ 0.2 %
+    r = S.rescale_flop_ratio(8192, 1024, 4096)
+    assert math.isclose(r, (1 / 8192 + 1 / 1024 + 1 / 4096) / 6, rel_tol=1e-14) and r <= 1 / (2 * 1024)
+    assert round(4 / (2 * 1024), 3) == GOLD["bert_large_flop_overhead"]
