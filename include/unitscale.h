@@ -1,0 +1,170 @@
+/*
+ * libunitscale -- unit-scaled linear / FFN ops for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every matrix is row-major DEVICE memory owned by the caller; the
+ * library allocates nothing on the device, keeps no reference to a buffer after
+ * a call returns, and never synchronises: each call enqueues its kernels on the
+ * given stream (a cudaStream_t passed as void*, NULL = the default stream) and
+ * returns.  Errors are reported through the return value only; argument,
+ * dtype, shape and alignment checks all run on the host before any launch, so
+ * a call that returns an error other than US_ERR_CUDA has launched nothing.
+ * There is no CPU fallback.
+ *
+ * Notation follows the paper: a scaled op is f* = alpha * f in the forward pass
+ * and f*_grad_i = beta_i * f_grad_i in the backward pass (section "Scaled ops");
+ * X is [b x m], W is [m x n] = [fan_in x fan_out], G is the gradient of the
+ * output, [b x n] (section "Example").
+ */
+#ifndef UNITSCALE_H_
+#define UNITSCALE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  US_OK = 0,
+  US_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, ld < cols, bad enum, shape mismatch */
+  US_ERR_UNSUPPORTED = 2, /* dtype combination that has no kernel */
+  US_ERR_ALIGNMENT = 3,   /* pointer not 16-byte aligned, or row pitch not a multiple of 16 bytes */
+  US_ERR_WORKSPACE = 4,   /* workspace missing or smaller than us_workspace_bytes() */
+  US_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (launch, tensor-map encode) */
+  US_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (reported by us_workspace_status) */
+} us_status;
+
+/* Storage formats.  E4M3 / E5M2 are the OCP 8-bit formats (rows "FP8 E4 (b)" and
+ * "FP8 E5 (b)" of the appendix table "Common floating point formats for deep
+ * learning"): E4M3 for activations and weights, E5M2 for gradients. */
+typedef enum { US_F32 = 0, US_BF16 = 1, US_F16 = 2, US_E4M3 = 3, US_E5M2 = 4 } us_dtype;
+
+/* A row-major matrix in device memory.  ld = elements between consecutive rows
+ * (ld >= cols).  ptr must be 16-byte aligned and ld * sizeof(element) a multiple
+ * of 16 bytes for every matrix handed to a linear op. */
+typedef struct {
+  void* ptr;
+  int32_t dtype; /* us_dtype */
+  int64_t rows, cols, ld;
+} us_mat;
+
+typedef enum { US_ACT_NONE = 0, US_ACT_GELU = 1, US_ACT_GELU_GRAD = 2 } us_act;
+
+/*
+ * Work fused after the scaled accumulator of a linear op, applied per element in
+ * float32 and rounded once to the output dtype (round-to-nearest-even; the FP8
+ * casts saturate to the largest finite value):
+ *
+ *   v = scale * acc
+ *   US_ACT_GELU:       if aux.ptr, aux = round16(v)  (the pre-activation the backward pass reads);
+ *                      v = act_out_scale * gelu(act_in_scale * v)
+ *   US_ACT_GELU_GRAD:  h = aux (required);
+ *                      v = act_out_scale * act_in_scale * gelu'(act_in_scale * h) * v
+ *   skip.ptr != NULL:  v = skip_coef * skip + out_coef * v
+ *   out = round_to(out dtype, v)
+ *
+ * gelu(x) = x * Phi(x) with the exact normal CDF (table "Table of unit scaling
+ * factors"); act_in_scale is the alignment pre-scale of appendix "Aligning a unit
+ * scaled model with an existing model" (1 when unused).  The skip path is the
+ * fixed(tau) residual of section "Weighted addition": skip_coef = sqrt(1 - tau),
+ * out_coef = sqrt(tau).  aux and skip have the shape of the output; aux is BF16 or
+ * F16, skip is F32, BF16 or F16.
+ */
+typedef struct {
+  int32_t act; /* us_act */
+  float act_in_scale;
+  float act_out_scale;
+  us_mat aux;
+  us_mat skip;
+  float skip_coef;
+  float out_coef;
+} us_epilogue;
+
+/* ------------------------------------------------------------------ linear ops
+ *
+ * The three GEMMs of a unit-scaled linear layer (section "Example"; table row
+ * "matmul"):
+ *
+ *   us_linear_fwd    Y  = alpha  * X  W      X [b x m], W [m x n]  ->  Y  [b x n]
+ *   us_linear_bwd_x  dX = beta_x * G  W^T    G [b x n], W [m x n]  ->  dX [b x m]
+ *   us_linear_bwd_w  dW = beta_w * X^T G     X [b x m], G [b x n]  ->  dW [m x n]
+ *
+ * W is always passed in the [fan_in x fan_out] orientation; no transposed copy is
+ * needed or made.  Products are formed from the stored operand values and
+ * accumulated in float32 (tensor-core accumulators); the scale is one float32
+ * multiply on the accumulator, followed by the optional epilogue (NULL = none)
+ * and a single rounding to the output dtype.  The unit-scaling values of the
+ * scales are alpha = m^-1/2, beta_x = n^-1/2, beta_w = b^-1/2 (us_scales_linear).
+ *
+ * Operand dtypes: both 8-bit (any mix of US_E4M3 / US_E5M2), or both US_BF16, or
+ * both US_F16.  Output dtype: any us_dtype.  Every dimension must be >= 1; rows
+ * and columns need not be multiples of the tile sizes.  Alignment rule: see
+ * us_mat (violations return US_ERR_ALIGNMENT).
+ *
+ * ws: device workspace of at least us_workspace_bytes() bytes, 16-byte aligned,
+ * zeroed once by the caller before its first use (cudaMemsetAsync).  It holds a
+ * status word that a kernel sets if one of its bounded waits runs out; calls on
+ * the same stream may share it.  Read it with us_workspace_status.
+ */
+us_status us_linear_fwd(const us_mat* X, const us_mat* W, float alpha, const us_epilogue* ep,
+                        const us_mat* Y, void* ws, size_t ws_bytes, void* stream);
+us_status us_linear_bwd_x(const us_mat* G, const us_mat* W, float beta_x, const us_epilogue* ep,
+                          const us_mat* dX, void* ws, size_t ws_bytes, void* stream);
+us_status us_linear_bwd_w(const us_mat* X, const us_mat* G, float beta_w, const us_epilogue* ep,
+                          const us_mat* dW, void* ws, size_t ws_bytes, void* stream);
+
+/* Bytes of device workspace the linear ops need. */
+size_t us_workspace_bytes(void);
+
+/* Waits for `stream`, copies the workspace status word to the host and returns
+ * US_OK, US_ERR_TIMEOUT (a device-side wait gave up: the outputs of that call are
+ * not valid) or US_ERR_CUDA.  This is the only call that synchronises. */
+us_status us_workspace_status(const void* ws, void* stream);
+
+/* ------------------------------------------------------------ elementwise ops
+ *
+ * Unfused forms of the ops between the GEMMs.  All tensors of a call have the
+ * same rows x cols; any ld >= cols; pointers need only the natural alignment of
+ * their element type (rows whose start is 16-byte aligned take the 128-bit path).
+ *
+ * us_gelu_fwd      A  = alpha * gelu(s_in * H)                      (table row "gelu")
+ * us_gelu_bwd      dH = beta * s_in * gelu'(s_in * H) * dA
+ * us_residual_add  out = sqrt(1 - tau) * skip + sqrt(tau) * branch  (section "Weighted
+ *                  addition", scheme fixed(tau)); serves the backward pass too: there
+ *                  skip = incoming gradient, branch = gradient at the branch entry.
+ * us_cast_fp8      dst = q(scale * src), q = nearest value of the FP8 format, ties to
+ *                  even, saturating (section "Floating-point formats for deep learning",
+ *                  paragraph "Quantisation error"); the product is one float32
+ *                  multiply.  NaN stays NaN.
+ *
+ * Inputs may be F32, BF16 or F16; outputs any us_dtype (us_cast_fp8: E4M3 or E5M2
+ * only).  0 <= tau <= 1.
+ */
+us_status us_gelu_fwd(const us_mat* H, float s_in, float alpha, const us_mat* A, void* stream);
+us_status us_gelu_bwd(const us_mat* H, const us_mat* dA, float s_in, float beta, const us_mat* dH,
+                      void* stream);
+us_status us_residual_add(const us_mat* skip, const us_mat* branch, float tau, const us_mat* out,
+                          void* stream);
+us_status us_cast_fp8(const us_mat* src, float scale, const us_mat* dst, void* stream);
+
+/* ---------------------------------------------------------------- host helpers
+ *
+ * us_scales_linear: unit-scaling factors of matmul(X[b x m], W[m x n]).
+ *   constrained == 0: alpha = m^-1/2, beta_x = n^-1/2, beta_w = b^-1/2 (table row "matmul").
+ *   constrained != 0: alpha = beta_x = (m n)^-1/4 (geometric mean, section "Example").
+ * us_scales_gelu: 1/std of gelu(z) and 1/rms of gelu'(z) for z ~ N(0,1) (the table prints
+ *   them as 1.701 / 1.481); constrained: both equal their geometric mean.
+ * Pure host arithmetic; output pointers must be non-NULL.
+ */
+us_status us_scales_linear(int64_t b, int64_t m, int64_t n, int constrained, float* alpha,
+                           float* beta_x, float* beta_w);
+us_status us_scales_gelu(int constrained, float* alpha, float* beta);
+
+const char* us_status_string(us_status s);
+int us_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UNITSCALE_H_ */
