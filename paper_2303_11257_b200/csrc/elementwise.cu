@@ -1,0 +1,146 @@
+// Unfused elementwise ops of libunitscale: FP8 cast, scaled GELU forward/backward,
+// tau-weighted residual add.  All are HBM-bandwidth bound: each thread moves 16
+// elements per iteration with 128-bit loads and stores; the grid is a multiple of
+// the SM count and strides over the tensor.
+#include "common.cuh"
+#include "host.h"
+
+namespace us {
+
+constexpr int kVec = 16;       // elements per thread per iteration
+constexpr int kThreads = 256;
+
+struct EwTensor {
+  void* ptr;
+  int dt;
+  int64_t ld;
+};
+
+struct EwArgs {
+  EwTensor in0, in1, out;
+  int64_t rows, cols;
+  int64_t chunks_per_row;  // ceil(cols / kVec)
+  int vec_ok;              // every row start of every tensor is 16-byte aligned
+  float c0, c1, c2;        // op constants
+};
+
+enum EwOp { kCast = 0, kGeluFwd = 1, kGeluBwd = 2, kResidual = 3 };
+
+template <int OP>
+__device__ __forceinline__ float ew_apply(float a, float b, const EwArgs& p) {
+  if (OP == kCast) return p.c0 * a;                                   // scale * x, then the store rounds
+  if (OP == kGeluFwd) return gelu_scaled(a, p.c0, p.c1);              // c0 = s_in, c1 = alpha
+  if (OP == kGeluBwd) return gelu_grad_scaled(a, b, p.c0, p.c1);      // a = H, b = dA, c1 = beta
+  return fmaf(p.c0, a, p.c1 * b);                                     // c0 = sqrt(1-tau), c1 = sqrt(tau)
+}
+
+template <int OP>
+__global__ void __launch_bounds__(kThreads) ew_kernel(const EwArgs p) {
+  constexpr bool kTwoInputs = (OP == kGeluBwd || OP == kResidual);
+  const int64_t total = p.rows * p.chunks_per_row;
+  for (int64_t c = blockIdx.x * (int64_t)kThreads + threadIdx.x; c < total;
+       c += (int64_t)gridDim.x * kThreads) {
+    const int64_t row = c / p.chunks_per_row;
+    const int64_t col = (c - row * p.chunks_per_row) * kVec;
+    const int64_t i0 = row * p.in0.ld + col, i1 = row * p.in1.ld + col, io = row * p.out.ld + col;
+    if (p.vec_ok && col + kVec <= p.cols) {
+      float a[kVec], b[kVec], o[kVec];
+      load_vec<kVec>(static_cast<const char*>(p.in0.ptr) + i0 * dtype_size(p.in0.dt), p.in0.dt, a);
+      if (kTwoInputs) load_vec<kVec>(static_cast<const char*>(p.in1.ptr) + i1 * dtype_size(p.in1.dt), p.in1.dt, b);
+#pragma unroll
+      for (int i = 0; i < kVec; ++i) o[i] = ew_apply<OP>(a[i], kTwoInputs ? b[i] : 0.f, p);
+      store_vec<kVec>(static_cast<char*>(p.out.ptr) + io * dtype_size(p.out.dt), p.out.dt, o);
+    } else {
+      const int n = (int)min((int64_t)kVec, p.cols - col);
+      for (int i = 0; i < n; ++i) {
+        const float a = load_one(p.in0.ptr, p.in0.dt, i0 + i);
+        const float b = kTwoInputs ? load_one(p.in1.ptr, p.in1.dt, i1 + i) : 0.f;
+        store_one(p.out.ptr, p.out.dt, io + i, ew_apply<OP>(a, b, p));
+      }
+    }
+  }
+}
+
+static bool row_starts_aligned(const us_mat* m, bool contiguous) {
+  const int es = dtype_size(m->dtype);
+  if (reinterpret_cast<uintptr_t>(m->ptr) % 16) return false;
+  return contiguous || (m->ld * es) % 16 == 0;
+}
+
+template <int OP>
+static us_status ew_launch(const us_mat* in0, const us_mat* in1, const us_mat* out, float c0, float c1,
+                           void* stream) {
+  EwArgs p{};
+  // A tensor set without row padding is one long row: chunking then never straddles a row end.
+  const bool contiguous = in0->ld == in0->cols && (!in1 || in1->ld == in1->cols) && out->ld == out->cols;
+  p.rows = contiguous ? 1 : in0->rows;
+  p.cols = contiguous ? in0->rows * in0->cols : in0->cols;
+  p.in0 = {in0->ptr, in0->dtype, in0->ld};
+  p.in1 = in1 ? EwTensor{in1->ptr, in1->dtype, in1->ld} : p.in0;
+  p.out = {out->ptr, out->dtype, out->ld};
+  p.chunks_per_row = (p.cols + kVec - 1) / kVec;
+  p.vec_ok = row_starts_aligned(in0, contiguous) && (!in1 || row_starts_aligned(in1, contiguous)) &&
+             row_starts_aligned(out, contiguous);
+  p.c0 = c0; p.c1 = c1;
+  const int64_t total = p.rows * p.chunks_per_row;
+  if (total == 0) return US_OK;
+  const int sms = host::sm_count();
+  if (sms <= 0) return US_ERR_CUDA;
+  const int64_t want = (total + kThreads - 1) / kThreads;
+  const int64_t cap = (int64_t)sms * 8;                 // 8 resident CTAs of 256 threads per SM
+  const int grid = (int)(want < cap ? want : cap);
+  ew_kernel<OP><<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
+}
+
+}  // namespace us
+
+using namespace us;
+
+static bool is_float_in(int dt) { return dt == US_F32 || dt == US_BF16 || dt == US_F16; }
+static bool is_dtype(int dt) { return dt >= US_F32 && dt <= US_E5M2; }
+
+static us_status check_ew(const us_mat* a, const us_mat* b, const us_mat* out) {
+  const us_mat* ms[3] = {a, b, out};
+  for (int i = 0; i < 3; ++i) {
+    const us_mat* m = ms[i];
+    if (i == 1 && !m) continue;
+    if (!m || m->rows < 0 || m->cols < 0 || m->ld < m->cols) return US_ERR_INVALID_ARG;
+    if (m->rows != a->rows || m->cols != a->cols) return US_ERR_INVALID_ARG;
+    if (m->rows * m->cols > 0 && !m->ptr) return US_ERR_INVALID_ARG;
+    if (i < 2 ? !is_float_in(m->dtype) : !is_dtype(m->dtype)) return US_ERR_UNSUPPORTED;
+    if (m->ptr && reinterpret_cast<uintptr_t>(m->ptr) % dtype_size(m->dtype)) return US_ERR_ALIGNMENT;
+  }
+  return US_OK;
+}
+
+extern "C" us_status us_cast_fp8(const us_mat* src, float scale, const us_mat* dst, void* stream) {
+  us_status s = check_ew(src, nullptr, dst);
+  if (s != US_OK) return s;
+  if (dst->dtype != US_E4M3 && dst->dtype != US_E5M2) return US_ERR_UNSUPPORTED;
+  return ew_launch<kCast>(src, nullptr, dst, scale, 0.f, stream);
+}
+
+extern "C" us_status us_gelu_fwd(const us_mat* H, float s_in, float alpha, const us_mat* A, void* stream) {
+  us_status s = check_ew(H, nullptr, A);
+  if (s != US_OK) return s;
+  return ew_launch<kGeluFwd>(H, nullptr, A, s_in, alpha, stream);
+}
+
+extern "C" us_status us_gelu_bwd(const us_mat* H, const us_mat* dA, float s_in, float beta, const us_mat* dH,
+                                 void* stream) {
+  if (!dA) return US_ERR_INVALID_ARG;
+  us_status s = check_ew(H, dA, dH);
+  if (s != US_OK) return s;
+  return ew_launch<kGeluBwd>(H, dA, dH, s_in, beta, stream);
+}
+
+extern "C" us_status us_residual_add(const us_mat* skip, const us_mat* branch, float tau, const us_mat* out,
+                                     void* stream) {
+  if (!branch) return US_ERR_INVALID_ARG;
+  us_status s = check_ew(skip, branch, out);
+  if (s != US_OK) return s;
+  if (!(tau >= 0.f && tau <= 1.f)) return US_ERR_INVALID_ARG;
+  const float c_skip = (float)sqrt(1.0 - (double)tau), c_branch = (float)sqrt((double)tau);
+  return ew_launch<kResidual>(skip, branch, out, c_skip, c_branch, stream);
+}

@@ -1,0 +1,60 @@
+// Host-only entry points of libunitscale: scale-factor helpers, status strings, device queries.
+#include <math.h>
+
+#include "host.h"
+
+namespace us {
+namespace host {
+int sm_count() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return -1;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+}  // namespace host
+}  // namespace us
+
+// 1 / std(gelu(z)) and 1 / rms(gelu'(z)) for z ~ N(0,1), gelu(x) = x Phi(x): the values the
+// table of unit scaling factors prints as 1.701 and 1.481, here to double precision.
+static const double kGeluAlpha = 1.7009262433633;
+static const double kGeluBeta = 1.4811144127083;
+
+extern "C" us_status us_scales_linear(int64_t b, int64_t m, int64_t n, int constrained, float* alpha,
+                                      float* beta_x, float* beta_w) {
+  if (b < 1 || m < 1 || n < 1 || !alpha || !beta_x || !beta_w) return US_ERR_INVALID_ARG;
+  double a = 1.0 / sqrt((double)m), bx = 1.0 / sqrt((double)n), bw = 1.0 / sqrt((double)b);
+  if (constrained) a = bx = sqrt(a * bx);  // geometric mean of the constrained pair
+  *alpha = (float)a;
+  *beta_x = (float)bx;
+  *beta_w = (float)bw;
+  return US_OK;
+}
+
+extern "C" us_status us_scales_gelu(int constrained, float* alpha, float* beta) {
+  if (!alpha || !beta) return US_ERR_INVALID_ARG;
+  double a = kGeluAlpha, b = kGeluBeta;
+  if (constrained) a = b = sqrt(a * b);
+  *alpha = (float)a;
+  *beta = (float)b;
+  return US_OK;
+}
+
+extern "C" const char* us_status_string(us_status s) {
+  switch (s) {
+    case US_OK: return "ok";
+    case US_ERR_INVALID_ARG: return "invalid argument";
+    case US_ERR_UNSUPPORTED: return "unsupported dtype combination";
+    case US_ERR_ALIGNMENT: return "pointer or row pitch not 16-byte aligned";
+    case US_ERR_WORKSPACE: return "workspace missing or too small";
+    case US_ERR_CUDA: return "CUDA call failed";
+    case US_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+extern "C" int us_version(void) { return 100; }
