@@ -1,0 +1,193 @@
+"""ctypes binding of libunitscale: same names as the C ABI, argument marshalling only.
+
+Tensors are torch CUDA tensors (device memory and streams come from torch); every
+computation happens inside the library's kernels.  Importing this module needs the
+compiled library: there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+US_OK = 0
+STATUS_NAMES = {
+    0: "US_OK", 1: "US_ERR_INVALID_ARG", 2: "US_ERR_UNSUPPORTED", 3: "US_ERR_ALIGNMENT",
+    4: "US_ERR_WORKSPACE", 5: "US_ERR_CUDA", 6: "US_ERR_TIMEOUT",
+}
+US_F32, US_BF16, US_F16, US_E4M3, US_E5M2 = range(5)
+US_ACT_NONE, US_ACT_GELU, US_ACT_GELU_GRAD = range(3)
+
+_TORCH_DTYPES = {
+    torch.float32: US_F32, torch.bfloat16: US_BF16, torch.float16: US_F16,
+    torch.float8_e4m3fn: US_E4M3, torch.float8_e5m2: US_E5M2,
+}
+
+
+class us_mat(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("dtype", C.c_int32), ("rows", C.c_int64), ("cols", C.c_int64), ("ld", C.c_int64)]
+
+
+class us_epilogue(C.Structure):
+    _fields_ = [
+        ("act", C.c_int32), ("act_in_scale", C.c_float), ("act_out_scale", C.c_float),
+        ("aux", us_mat), ("skip", us_mat), ("skip_coef", C.c_float), ("out_coef", C.c_float),
+    ]
+
+
+class UnitScaleError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn}: {STATUS_NAMES.get(status, status)}")
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libunitscale.so")
+
+
+def _load() -> C.CDLL:
+    path = library_path()
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2303_11257_b200.build` "
+            "(there is no fallback implementation)")
+    lib = C.CDLL(path)
+    P, MP, EP, F, V, SZ = C.c_void_p, C.POINTER(us_mat), C.POINTER(us_epilogue), C.c_float, C.c_void_p, C.c_size_t
+    for name in ("us_linear_fwd", "us_linear_bwd_x", "us_linear_bwd_w"):
+        fn = getattr(lib, name)
+        fn.argtypes = [MP, MP, F, EP, MP, V, SZ, V]
+        fn.restype = C.c_int
+    lib.us_workspace_bytes.argtypes = []
+    lib.us_workspace_bytes.restype = SZ
+    lib.us_workspace_status.argtypes = [V, V]
+    lib.us_workspace_status.restype = C.c_int
+    lib.us_gelu_fwd.argtypes = [MP, F, F, MP, V]
+    lib.us_gelu_bwd.argtypes = [MP, MP, F, F, MP, V]
+    lib.us_residual_add.argtypes = [MP, MP, F, MP, V]
+    lib.us_cast_fp8.argtypes = [MP, F, MP, V]
+    for name in ("us_gelu_fwd", "us_gelu_bwd", "us_residual_add", "us_cast_fp8"):
+        getattr(lib, name).restype = C.c_int
+    FP = C.POINTER(C.c_float)
+    lib.us_scales_linear.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_int, FP, FP, FP]
+    lib.us_scales_linear.restype = C.c_int
+    lib.us_scales_gelu.argtypes = [C.c_int, FP, FP]
+    lib.us_scales_gelu.restype = C.c_int
+    lib.us_status_string.argtypes = [C.c_int]
+    lib.us_status_string.restype = C.c_char_p
+    lib.us_version.argtypes = []
+    lib.us_version.restype = C.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def raw() -> C.CDLL:
+    """The loaded CDLL, for callers that want to build us_mat structures themselves."""
+    return _lib
+
+
+def mat(t: torch.Tensor) -> us_mat:
+    """Describe a 2-D row-major torch tensor (last stride 1) without copying it."""
+    if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError("expected a 2-D tensor with unit column stride")
+    ld = t.stride(0) if t.shape[0] > 1 else max(t.shape[1], t.stride(0))
+    return us_mat(t.data_ptr(), _TORCH_DTYPES[t.dtype], t.shape[0], t.shape[1], ld)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(fn: str, status: int) -> None:
+    if status != US_OK:
+        raise UnitScaleError(fn, status)
+
+
+def epilogue(act: int = US_ACT_NONE, act_in_scale: float = 1.0, act_out_scale: float = 1.0,
+             aux: torch.Tensor | None = None, skip: torch.Tensor | None = None,
+             skip_coef: float = 0.0, out_coef: float = 1.0) -> us_epilogue:
+    ep = us_epilogue()
+    ep.act, ep.act_in_scale, ep.act_out_scale = act, act_in_scale, act_out_scale
+    if aux is not None:
+        ep.aux = mat(aux)
+    if skip is not None:
+        ep.skip = mat(skip)
+    ep.skip_coef, ep.out_coef = skip_coef, out_coef
+    return ep
+
+
+def us_workspace_bytes() -> int:
+    return int(_lib.us_workspace_bytes())
+
+
+def new_workspace(device="cuda") -> torch.Tensor:
+    """A zeroed workspace of the size the linear ops ask for."""
+    return torch.zeros(us_workspace_bytes(), dtype=torch.uint8, device=device)
+
+
+def us_workspace_status(ws: torch.Tensor, stream=None) -> int:
+    return int(_lib.us_workspace_status(ws.data_ptr(), _stream(stream)))
+
+
+def _linear(name, a, b, scale, ep, out, ws, stream):
+    fn = getattr(_lib, name)
+    epp = C.byref(ep) if ep is not None else None
+    _check(name, fn(C.byref(mat(a)), C.byref(mat(b)), scale, epp, C.byref(mat(out)),
+                    ws.data_ptr(), ws.numel() * ws.element_size(), _stream(stream)))
+    return out
+
+
+def us_linear_fwd(X, W, alpha, Y, ws, ep=None, stream=None):
+    return _linear("us_linear_fwd", X, W, alpha, ep, Y, ws, stream)
+
+
+def us_linear_bwd_x(G, W, beta_x, dX, ws, ep=None, stream=None):
+    return _linear("us_linear_bwd_x", G, W, beta_x, ep, dX, ws, stream)
+
+
+def us_linear_bwd_w(X, G, beta_w, dW, ws, ep=None, stream=None):
+    return _linear("us_linear_bwd_w", X, G, beta_w, ep, dW, ws, stream)
+
+
+def us_gelu_fwd(H, s_in, alpha, A, stream=None):
+    _check("us_gelu_fwd", _lib.us_gelu_fwd(C.byref(mat(H)), s_in, alpha, C.byref(mat(A)), _stream(stream)))
+    return A
+
+
+def us_gelu_bwd(H, dA, s_in, beta, dH, stream=None):
+    _check("us_gelu_bwd", _lib.us_gelu_bwd(C.byref(mat(H)), C.byref(mat(dA)), s_in, beta, C.byref(mat(dH)), _stream(stream)))
+    return dH
+
+
+def us_residual_add(skip, branch, tau, out, stream=None):
+    _check("us_residual_add", _lib.us_residual_add(C.byref(mat(skip)), C.byref(mat(branch)), tau, C.byref(mat(out)), _stream(stream)))
+    return out
+
+
+def us_cast_fp8(src, scale, dst, stream=None):
+    _check("us_cast_fp8", _lib.us_cast_fp8(C.byref(mat(src)), scale, C.byref(mat(dst)), _stream(stream)))
+    return dst
+
+
+def us_scales_linear(b: int, m: int, n: int, constrained: bool = False):
+    a, bx, bw = C.c_float(), C.c_float(), C.c_float()
+    _check("us_scales_linear", _lib.us_scales_linear(b, m, n, int(constrained), C.byref(a), C.byref(bx), C.byref(bw)))
+    return a.value, bx.value, bw.value
+
+
+def us_scales_gelu(constrained: bool = False):
+    a, b = C.c_float(), C.c_float()
+    _check("us_scales_gelu", _lib.us_scales_gelu(int(constrained), C.byref(a), C.byref(b)))
+    return a.value, b.value
+
+
+def us_status_string(status: int) -> str:
+    return _lib.us_status_string(status).decode()
+
+
+def us_version() -> int:
+    return int(_lib.us_version())
