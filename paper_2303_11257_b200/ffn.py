@@ -1,0 +1,124 @@
+"""Unit-scaled Transformer FFN block (forward + backward) as a sequence of libunitscale calls.
+
+A driver only: it owns the device buffers and issues the C-ABI calls in order; every step
+of the computation happens in the library's kernels.
+
+Forward (Figure "PyTorch examples", scaled FFN; section "Weighted addition"):
+    Xq = q(X); W1q = q(W1); W2q = q(W2)                                   us_cast_fp8
+    H  = alpha1 Xq W1q ; A = q(alpha_g gelu(s_in H)), H kept in 16 bit    us_linear_fwd + GELU epilogue
+    R  = sqrt(1-tau) X + sqrt(tau) alpha2 A W2q                           us_linear_fwd + residual epilogue
+Backward, G = dL/dR (the branch output receives G unscaled):
+    Gq  = q(G)                                                            us_cast_fp8
+    dH  = q(beta_g s_in gelu'(s_in H) * beta_x2 Gq W2q^T)                 us_linear_bwd_x + GELU-grad epilogue
+    dW2 = beta_w A^T Gq                                                   us_linear_bwd_w
+    dX  = sqrt(1-tau) G + sqrt(tau) beta_x1 dH W1q^T                      us_linear_bwd_x + residual epilogue
+    dW1 = beta_w Xq^T dH                                                  us_linear_bwd_w
+q is E4M3 for activations / weights and E5M2 for gradients in "fp8" mode; in "bf16" / "fp16"
+mode the matmul inputs are rounded to that format instead (no loss scale, same fixed scales).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+
+import torch
+
+from . import lib as L
+
+
+@dataclass
+class FFNScales:
+    alpha1: float
+    alpha2: float
+    beta_x1: float
+    beta_x2: float
+    beta_w: float
+    alpha_g: float
+    beta_g: float
+    s_in: float = 1.0
+    tau: float = 0.5
+
+    @staticmethod
+    def unit(T: int, d: int, f: int, tau: float = 0.5, constrained: bool = False) -> "FFNScales":
+        a1, bx1, bw = L.us_scales_linear(T, d, f, constrained)
+        a2, bx2, _ = L.us_scales_linear(T, f, d, constrained)
+        ag, bg = L.us_scales_gelu(constrained)
+        return FFNScales(a1, a2, bx1, bx2, bw, ag, bg, 1.0, tau)
+
+
+_OPERAND = {
+    "fp8": (torch.float8_e4m3fn, torch.float8_e5m2),
+    "bf16": (torch.bfloat16, torch.bfloat16),
+    "fp16": (torch.float16, torch.float16),
+}
+
+
+class UnitScaledFFN:
+    """Buffers + call sequence for one FFN block of T tokens, width d, hidden width f."""
+
+    def __init__(self, T: int, d: int, f: int, scales: FFNScales | None = None, operand: str = "fp8",
+                 h_dtype=torch.bfloat16, io_dtype=torch.bfloat16, device="cuda"):
+        self.T, self.d, self.f = T, d, f
+        self.sc = scales or FFNScales.unit(T, d, f)
+        self.operand = operand
+        act_dt, grad_dt = _OPERAND[operand]
+        e = lambda r, c, dt: torch.empty((r, c), dtype=dt, device=device)
+        self.Xq, self.W1q, self.W2q, self.Gq = e(T, d, act_dt), e(d, f, act_dt), e(f, d, act_dt), e(T, d, grad_dt)
+        self.H = e(T, f, h_dtype)
+        self.Aq = e(T, f, act_dt)
+        self.dHq = e(T, f, grad_dt)
+        self.R, self.dX = e(T, d, io_dtype), e(T, d, io_dtype)
+        self.dW1 = e(d, f, torch.float32)
+        self.dW2 = e(f, d, torch.float32)
+        self.ws = L.new_workspace(device)
+        c_skip, c_branch = math.sqrt(1.0 - self.sc.tau), math.sqrt(self.sc.tau)
+        self._c = (c_skip, c_branch)
+        self.launches_per_step = 10
+
+    def _cast(self, src, dst, stream):
+        if dst.dtype in (torch.float8_e4m3fn, torch.float8_e5m2):
+            L.us_cast_fp8(src, 1.0, dst, stream)
+        else:
+            # 16-bit operand mode: rounding fp32 -> bf16/fp16 is the residual kernel with tau = 0
+            L.us_residual_add(src, src, 0.0, dst, stream)
+
+    def cast_weights(self, W1, W2, stream=None):
+        self._cast(W1, self.W1q, stream)
+        self._cast(W2, self.W2q, stream)
+
+    def forward(self, X, stream=None):
+        sc, (c_skip, c_branch) = self.sc, self._c
+        self._cast(X, self.Xq, stream)
+        ep1 = L.epilogue(act=L.US_ACT_GELU, act_in_scale=sc.s_in, act_out_scale=sc.alpha_g, aux=self.H)
+        L.us_linear_fwd(self.Xq, self.W1q, sc.alpha1, self.Aq, self.ws, ep1, stream)
+        ep2 = L.epilogue(skip=X, skip_coef=c_skip, out_coef=c_branch)
+        L.us_linear_fwd(self.Aq, self.W2q, sc.alpha2, self.R, self.ws, ep2, stream)
+        return self.R
+
+    def backward(self, G, stream=None):
+        sc, (c_skip, c_branch) = self.sc, self._c
+        self._cast(G, self.Gq, stream)
+        ep3 = L.epilogue(act=L.US_ACT_GELU_GRAD, act_in_scale=sc.s_in, act_out_scale=sc.beta_g, aux=self.H)
+        L.us_linear_bwd_x(self.Gq, self.W2q, sc.beta_x2, self.dHq, self.ws, ep3, stream)
+        L.us_linear_bwd_w(self.Aq, self.Gq, sc.beta_w, self.dW2, self.ws, None, stream)
+        ep5 = L.epilogue(skip=G, skip_coef=c_skip, out_coef=c_branch)
+        L.us_linear_bwd_x(self.dHq, self.W1q, sc.beta_x1, self.dX, self.ws, ep5, stream)
+        L.us_linear_bwd_w(self.Xq, self.dHq, sc.beta_w, self.dW1, self.ws, None, stream)
+        return self.dX, self.dW1, self.dW2
+
+    def step(self, X, W1, W2, G, stream=None):
+        """One pass of the whole path: weight casts, forward, backward (10 kernel launches)."""
+        self.cast_weights(W1, W2, stream)
+        self.forward(X, stream)
+        return self.backward(G, stream)
+
+    def check(self) -> None:
+        """Synchronise and raise if any kernel reported a timed-out wait."""
+        st = L.us_workspace_status(self.ws)
+        if st != L.US_OK:
+            raise L.UnitScaleError("UnitScaledFFN", st)
+
+    @staticmethod
+    def flops(T: int, d: int, f: int) -> float:
+        """Matmul FLOPs, forward + backward: 2 linear layers x 3 GEMMs x 2 T d f."""
+        return 12.0 * T * d * f

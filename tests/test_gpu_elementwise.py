@@ -1,0 +1,84 @@
+"""Unfused scaled GELU forward/backward and the tau-weighted residual add against the oracle.
+
+Tolerance: the kernels evaluate Phi with the Abramowitz-Stegun 7.1.26 rational form in float32
+(|erf error| <= 1.5e-7), so gelu / gelu' values carry an absolute error below 1e-6 at unit scale;
+the checks allow 2e-6 absolute plus the rounding of the output format (1 ulp for 16-bit, one code
+step for FP8)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ops as O
+from oracle import scales as S
+from tests import util as U
+
+pytestmark = pytest.mark.gpu
+ABS = 2e-6
+
+
+def _lib():
+    from paper_2303_11257_b200 import lib, synth
+    return lib, synth
+
+
+@pytest.mark.parametrize("in_fmt", ["f32", "bf16", "fp16"])
+@pytest.mark.parametrize("out_fmt", ["f32", "bf16", "fp16", "e4m3", "e5m2"])
+@pytest.mark.parametrize("shape,ld", [((257, 1000), None), ((33, 48), 64)])
+def test_gelu_fwd_bwd(in_fmt, out_fmt, shape, ld):
+    L, synth = _lib()
+    ag, bg = S.gelu_scales()
+    s_in = 0.875
+    h = synth.normal(3, 0, shape, 1.5)
+    h[0, :8] = [0.0, -0.0, 6.0, -6.0, 10.0, -10.0, 1e-8, -37.0]
+    g = synth.normal(3, 1, shape)
+    Ht, Gt = U.to_device(h, in_fmt, ld), U.to_device(g, in_fmt, ld)
+    hv, gv = U.values_of(h, in_fmt), U.values_of(g, in_fmt)
+    out = U.empty(shape[0], shape[1], out_fmt, ld)
+    L.us_gelu_fwd(Ht, s_in, ag, out)
+    U.assert_close_stored(out, O.gelu_fwd(hv, s_in, ag), out_fmt, ABS * ag, "gelu_fwd")
+    L.us_gelu_bwd(Ht, Gt, s_in, bg, out)
+    ref = O.gelu_bwd(hv, gv, s_in, bg)
+    U.assert_close_stored(out, ref, out_fmt, ABS * bg * np.abs(gv).max(), "gelu_bwd")
+
+
+@pytest.mark.parametrize("in_fmt", ["f32", "bf16", "fp16"])
+@pytest.mark.parametrize("out_fmt", ["f32", "bf16", "fp16", "e4m3"])
+@pytest.mark.parametrize("tau", [0.0, 0.25, 0.5, 1.0])
+def test_residual_add(in_fmt, out_fmt, tau):
+    L, synth = _lib()
+    shape = (129, 515)
+    a, b = synth.normal(4, 0, shape), synth.normal(4, 1, shape)
+    out = U.empty(shape[0], shape[1], out_fmt)
+    L.us_residual_add(U.to_device(a, in_fmt), U.to_device(b, in_fmt), tau, out)
+    ref = O.residual_add(U.values_of(a, in_fmt), U.values_of(b, in_fmt), tau)
+    U.assert_close_stored(out, ref, out_fmt, 1e-6, "residual")
+
+
+def test_unit_variance_on_device():
+    """alpha_g gelu(z) has unit std and beta_g gelu'(z) g unit std for unit-normal inputs."""
+    L, synth = _lib()
+    ag, bg = L.us_scales_gelu()
+    assert abs(ag - S.gelu_scales()[0]) < 1e-6 and abs(bg - S.gelu_scales()[1]) < 1e-6
+    z = torch.from_numpy(synth.normal(5, 0, (2048, 2048))).cuda()
+    g = torch.from_numpy(synth.normal(5, 1, (2048, 2048))).cuda()
+    out = torch.empty_like(z)
+    L.us_gelu_fwd(z, 1.0, ag, out)
+    assert abs(out.std().item() - 1) < 5e-3
+    L.us_gelu_bwd(z, g, 1.0, bg, out)
+    assert abs(out.std().item() - 1) < 5e-3
+
+
+def test_elementwise_argument_errors():
+    L, _ = _lib()
+    a = torch.zeros((4, 8), device="cuda")
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_residual_add(a, a, 1.5, a)
+    assert e.value.status == 1
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_gelu_fwd(U.empty(4, 8, "e4m3"), 1.0, 1.0, a)
+    assert e.value.status == 2
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_gelu_bwd(a, torch.zeros((4, 7), device="cuda"), 1.0, 1.0, a)
+    assert e.value.status == 1
