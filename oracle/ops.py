@@ -185,6 +185,7 @@ class FFNResult:
     Aq: np.ndarray = None       # q_E4(alpha_g gelu(H)) values
     Aq_codes: np.ndarray = None
     R: np.ndarray = None        # block output
+    dA: np.ndarray = None       # beta_x2 q(G) q(W2)^T before the gelu-gradient factor (not stored on device)
     dHq: np.ndarray = None
     dHq_codes: np.ndarray = None
     dW2: np.ndarray = None
@@ -221,7 +222,8 @@ def ffn_block(X, W1, W2, G, sc: FFNScales, *, operand: str = "fp8",
     r.R, _, _ = apply_epilogue(linear_fwd(r.Aq, r.W2q, sc.alpha2), ep2, io_dtype)
 
     ep3 = Epilogue(act="gelu_grad", act_in_scale=sc.s_in, act_out_scale=sc.beta_g, aux=r.H)
-    r.dHq, r.dHq_codes, _ = apply_epilogue(linear_bwd_x(r.Gq, r.W2q, sc.beta_x2), ep3, grad_fmt)
+    r.dA = linear_bwd_x(r.Gq, r.W2q, sc.beta_x2)
+    r.dHq, r.dHq_codes, _ = apply_epilogue(r.dA, ep3, grad_fmt)
     r.dW2, _, _ = apply_epilogue(linear_bwd_w(r.Aq, r.Gq, sc.beta_w), None, "f32")
     ep5 = Epilogue(skip=np.asarray(G, np.float64), skip_coef=c_skip, out_coef=c_branch)
     r.dX, _, _ = apply_epilogue(linear_bwd_x(r.dHq, r.W1q, sc.beta_x1), ep5, io_dtype)

@@ -117,6 +117,7 @@ def epilogue(act: int = US_ACT_NONE, act_in_scale: float = 1.0, act_out_scale: f
     if skip is not None:
         ep.skip = mat(skip)
     ep.skip_coef, ep.out_coef = skip_coef, out_coef
+    ep._keep_alive = (aux, skip)      # the struct holds raw pointers only
     return ep
 
 

@@ -120,7 +120,8 @@ def test_gelu_grad_and_residual_epilogues(shape):
         skip = synth.normal(4, 8, (b, m))
         out = U.empty(b, m, out_fmt)
         cs, cb = S.residual_coefficients(0.3)
-        ep = L.epilogue(skip=U.to_device(skip, skip_fmt), skip_coef=float(cs), out_coef=float(cb))
+        skip_t = U.to_device(skip, skip_fmt)
+        ep = L.epilogue(skip=skip_t, skip_coef=float(cs), out_coef=float(cb))
         L.us_linear_bwd_x(U.to_device(G, "e5m2"), U.to_device(W, "e4m3"), float(bx), out, ws, ep)
         ref = O.weighted_add(U.values_of(skip, skip_fmt), val, cs, cb)
         U.assert_close_stored(out, ref, out_fmt, TOL, "residual epilogue")

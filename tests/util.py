@@ -81,7 +81,32 @@ def ulp_of(ref: np.ndarray, fmt: str) -> np.ndarray:
     return np.ldexp(1.0, e - f.M)
 
 
-def assert_close_stored(got: torch.Tensor, ref: np.ndarray, fmt: str, abs_tol: float, what: str = ""):
+def code_deltas(got: torch.Tensor, want_codes: np.ndarray, fmt: str, extra=0.0, max_flip_fraction: float = 2e-3):
+    """FP8 output check.  Every stored code must be within one step of the oracle's code, or -- where
+    `extra` (an element-wise value-space allowance derived from a legitimate upstream rounding flip)
+    is non-zero -- within one format spacing plus that allowance in value.  Differences must be rare.
+    Returns (device value - oracle value) per element (zero except at those places)."""
+    f = F.FORMATS[fmt]
+    gc = codes_of(got)
+    d = code_distance(gc, want_codes, fmt)
+    delta = F.decode(gc, f) - F.decode(want_codes, f)
+    ref = F.decode(want_codes, f)
+    ok = (d <= 1) | (np.abs(delta) <= ulp_of(ref, fmt) + extra)
+    assert ok.all(), f"FP8 output off by more than one step at {(~ok).sum()} places, worst code distance {d[~ok].max()}"
+    assert (d > 0).mean() <= max_flip_fraction, f"flip fraction {(d > 0).mean():.2e}"
+    return delta
+
+
+def propagated(a: np.ndarray, b: np.ndarray, sparse_side: str) -> np.ndarray:
+    """|a| @ |b|, where the operand named by sparse_side ("a" or "b") is a sparse matrix of rare
+    upstream rounding flips: an element-wise bound on how far they can move a downstream matmul."""
+    from scipy import sparse
+    if sparse_side == "a":
+        return np.asarray(sparse.csr_matrix(np.abs(a)) @ np.abs(b))
+    return np.asarray((sparse.csr_matrix(np.abs(b).T) @ np.abs(a).T).T)
+
+
+def assert_close_stored(got: torch.Tensor, ref: np.ndarray, fmt: str, abs_tol, what: str = ""):
     """Output-vs-oracle check for one stored tensor.
 
     f32: |d| <= abs_tol.  16-bit: |d| <= abs_tol + 1 ulp of the format at the reference.
