@@ -82,35 +82,56 @@ class UnitScaledFFN:
             # 16-bit operand mode: rounding fp32 -> bf16/fp16 is the residual kernel with tau = 0
             L.us_residual_add(src, src, 0.0, dst, stream)
 
+    def stages(self, X, W1, W2, G):
+        """The ten launches of one pass, in order, as (name, kind, callable(stream)) triples.
+
+        kind is "cast" or "gemm"; forward(), backward() and step() run exactly these."""
+        sc, (c_skip, c_branch) = self.sc, self._c
+        ep1 = L.epilogue(act=L.US_ACT_GELU, act_in_scale=sc.s_in, act_out_scale=sc.alpha_g, aux=self.H)
+        ep2 = L.epilogue(skip=X, skip_coef=c_skip, out_coef=c_branch)
+        ep3 = L.epilogue(act=L.US_ACT_GELU_GRAD, act_in_scale=sc.s_in, act_out_scale=sc.beta_g, aux=self.H)
+        ep5 = L.epilogue(skip=G, skip_coef=c_skip, out_coef=c_branch)
+        ws = self.ws
+        return [
+            ("cast_W1", "cast", lambda st=None: self._cast(W1, self.W1q, st)),
+            ("cast_W2", "cast", lambda st=None: self._cast(W2, self.W2q, st)),
+            ("cast_X", "cast", lambda st=None: self._cast(X, self.Xq, st)),
+            ("fwd1_gelu", "gemm", lambda st=None: L.us_linear_fwd(self.Xq, self.W1q, sc.alpha1, self.Aq, ws, ep1, st)),
+            ("fwd2_residual", "gemm", lambda st=None: L.us_linear_fwd(self.Aq, self.W2q, sc.alpha2, self.R, ws, ep2, st)),
+            ("cast_G", "cast", lambda st=None: self._cast(G, self.Gq, st)),
+            ("bwd_x2_gelu_grad", "gemm", lambda st=None: L.us_linear_bwd_x(self.Gq, self.W2q, sc.beta_x2, self.dHq, ws, ep3, st)),
+            ("bwd_w2", "gemm", lambda st=None: L.us_linear_bwd_w(self.Aq, self.Gq, sc.beta_w, self.dW2, ws, None, st)),
+            ("bwd_x1_residual", "gemm", lambda st=None: L.us_linear_bwd_x(self.dHq, self.W1q, sc.beta_x1, self.dX, ws, ep5, st)),
+            ("bwd_w1", "gemm", lambda st=None: L.us_linear_bwd_w(self.Xq, self.dHq, sc.beta_w, self.dW1, ws, None, st)),
+        ]
+
     def cast_weights(self, W1, W2, stream=None):
         self._cast(W1, self.W1q, stream)
         self._cast(W2, self.W2q, stream)
 
     def forward(self, X, stream=None):
-        sc, (c_skip, c_branch) = self.sc, self._c
-        self._cast(X, self.Xq, stream)
-        ep1 = L.epilogue(act=L.US_ACT_GELU, act_in_scale=sc.s_in, act_out_scale=sc.alpha_g, aux=self.H)
-        L.us_linear_fwd(self.Xq, self.W1q, sc.alpha1, self.Aq, self.ws, ep1, stream)
-        ep2 = L.epilogue(skip=X, skip_coef=c_skip, out_coef=c_branch)
-        L.us_linear_fwd(self.Aq, self.W2q, sc.alpha2, self.R, self.ws, ep2, stream)
+        for name, _, fn in self.stages(X, None, None, None)[2:5]:
+            fn(stream)
         return self.R
 
     def backward(self, G, stream=None):
-        sc, (c_skip, c_branch) = self.sc, self._c
-        self._cast(G, self.Gq, stream)
-        ep3 = L.epilogue(act=L.US_ACT_GELU_GRAD, act_in_scale=sc.s_in, act_out_scale=sc.beta_g, aux=self.H)
-        L.us_linear_bwd_x(self.Gq, self.W2q, sc.beta_x2, self.dHq, self.ws, ep3, stream)
-        L.us_linear_bwd_w(self.Aq, self.Gq, sc.beta_w, self.dW2, self.ws, None, stream)
-        ep5 = L.epilogue(skip=G, skip_coef=c_skip, out_coef=c_branch)
-        L.us_linear_bwd_x(self.dHq, self.W1q, sc.beta_x1, self.dX, self.ws, ep5, stream)
-        L.us_linear_bwd_w(self.Xq, self.dHq, sc.beta_w, self.dW1, self.ws, None, stream)
+        for name, _, fn in self.stages(None, None, None, G)[5:]:
+            fn(stream)
         return self.dX, self.dW1, self.dW2
 
     def step(self, X, W1, W2, G, stream=None):
         """One pass of the whole path: weight casts, forward, backward (10 kernel launches)."""
-        self.cast_weights(W1, W2, stream)
-        self.forward(X, stream)
-        return self.backward(G, stream)
+        for name, _, fn in self.stages(X, W1, W2, G):
+            fn(stream)
+        return self.dX, self.dW1, self.dW2
+
+    def capture(self, X, W1, W2, G):
+        """Records step() into a CUDA graph (run step() eagerly at least once before).  The graph
+        reads X, W1, W2, G from the tensors given here; refill those in place between replays."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.step(X, W1, W2, G)
+        return g
 
     def check(self) -> None:
         """Synchronise and raise if any kernel reported a timed-out wait."""
