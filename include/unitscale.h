@@ -122,6 +122,32 @@ size_t us_workspace_bytes(void);
  * not valid) or US_ERR_CUDA.  This is the only call that synchronises. */
 us_status us_workspace_status(const void* ws, void* stream);
 
+/*
+ * us_linear_fwd_static_ws: us_linear_fwd for callers that cannot supply a workspace.
+ * (The paper has no counterpart; this is a property of the library, not of the method.)
+ *
+ * Same computation, arguments and errors as us_linear_fwd, except that the scratch the kernel
+ * needs comes from a fixed 1024-byte array built into the library instead of from the caller.
+ * It is meant for code that has no way to allocate device memory: a plug-in that receives only
+ * its input and output buffers from the runtime hosting it, a serving loop that bans allocation
+ * once it is running because cudaMalloc stalls the device, a process whose framework has
+ * claimed all device memory for its own pool.  The call allocates and frees nothing, directly
+ * or through a library; each GPU that loads the library holds the 1024 bytes until exit.
+ *
+ *  - The first call on a device looks up the array's device address (a one-time set-up with
+ *    that device current).  Make that first call before starting any stream capture.
+ *  - All calls share the one array and it keeps the previous call's contents, so every call
+ *    first clears the status word on `stream`.  Two calls that overlap on the GPU (different
+ *    streams) race on that word: keep calls to this entry point on one stream, or order them.
+ *  - If the kernel's scratch requirement ever exceeds the built-in 1024 bytes the call returns
+ *    US_ERR_WORKSPACE and launches nothing; the requirement does not depend on the matrix sizes.
+ *  - ws_out (may be NULL) receives the device address of the built-in scratch; pass it to
+ *    us_workspace_status to learn whether this call's kernel timed out, before the next call
+ *    clears the word.
+ */
+us_status us_linear_fwd_static_ws(const us_mat* X, const us_mat* W, float alpha, const us_epilogue* ep,
+                                  const us_mat* Y, void** ws_out, void* stream);
+
 /* ------------------------------------------------------------ elementwise ops
  *
  * Unfused forms of the ops between the GEMMs.  All tensors of a call have the

@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libunitscale.so")
-SOURCES = ["host.cu", "elementwise.cu", "gemm.cu"]
+SOURCES = ["host.cu", "elementwise.cu", "gemm.cu", "static_ws.cu"]
 HEADERS = ["common.cuh", "sm100.cuh", "gemm_kernel.cuh", "host.h", os.path.join("..", "..", "include", "unitscale.h")]
 
 

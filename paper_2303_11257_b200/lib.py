@@ -58,6 +58,8 @@ def _load() -> C.CDLL:
         fn = getattr(lib, name)
         fn.argtypes = [MP, MP, F, EP, MP, V, SZ, V]
         fn.restype = C.c_int
+    lib.us_linear_fwd_static_ws.argtypes = [MP, MP, F, EP, MP, C.POINTER(C.c_void_p), V]
+    lib.us_linear_fwd_static_ws.restype = C.c_int
     lib.us_workspace_bytes.argtypes = []
     lib.us_workspace_bytes.restype = SZ
     lib.us_workspace_status.argtypes = [V, V]
@@ -152,6 +154,23 @@ def us_linear_bwd_x(G, W, beta_x, dX, ws, ep=None, stream=None):
 
 def us_linear_bwd_w(X, G, beta_w, dW, ws, ep=None, stream=None):
     return _linear("us_linear_bwd_w", X, G, beta_w, ep, dW, ws, stream)
+
+
+def us_linear_fwd_static_ws(X, W, alpha, Y, ep=None, stream=None) -> int:
+    """us_linear_fwd without a caller workspace: the library's built-in scratch array is used and
+    nothing is allocated.  For callers that cannot allocate device memory (see the header).
+    Returns the device address of the built-in scratch, which us_workspace_status_ptr accepts."""
+    ws = C.c_void_p()
+    epp = C.byref(ep) if ep is not None else None
+    _check("us_linear_fwd_static_ws",
+           _lib.us_linear_fwd_static_ws(C.byref(mat(X)), C.byref(mat(W)), alpha, epp, C.byref(mat(Y)),
+                                        C.byref(ws), _stream(stream)))
+    return ws.value
+
+
+def us_workspace_status_ptr(ws_ptr: int, stream=None) -> int:
+    """us_workspace_status for a raw device address."""
+    return int(_lib.us_workspace_status(ws_ptr, _stream(stream)))
 
 
 def us_gelu_fwd(H, s_in, alpha, A, stream=None):
