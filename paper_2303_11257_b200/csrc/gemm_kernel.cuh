@@ -2,14 +2,17 @@
 //
 //   out[M x N] = epilogue( scale * sum_k A(m, k) B(n, k) )
 //
-// One persistent CTA per SM walks over 128 x BN output tiles.  Warp roles:
+// One persistent CTA per SM.  A CTA walks over 128 x BN output tiles on its own, or a cluster of
+// two CTAs (cta_group::2) walks over 256 x BN tiles: each CTA then loads only its half of the B
+// tile, which cuts the operand bytes per tensor-core cycle by a third.  Warp roles:
 //   warp 0   TMA producer: fills a ring of shared-memory stages (one 128-byte-swizzled
 //            A tile + B tile per stage, 128 bytes of K each) with cp.async.bulk.tensor;
 //   warp 1   MMA issuer: one thread issues tcgen05.mma (4 per stage) into one of two
 //            float32 accumulators in tensor memory, commits stage release and
 //            accumulator-ready barriers; the warp owns the TMEM allocation;
-//   warps 2-5 epilogue: tcgen05.ld their 32-lane quarter of the finished accumulator,
-//            apply scale / GELU / GELU-gradient / residual, round once, store.
+//   warps 2-9 epilogue: tcgen05.ld 32-column slices of their 32-lane quarter of the finished
+//            accumulator (two warps per quarter), apply scale / GELU / GELU-gradient /
+//            residual, round once, store.
 // While the epilogue drains accumulator i, the MMA warp already fills accumulator i^1.
 //
 // Either operand may be stored K-major (row = M or N index, K contiguous) or MN-major
@@ -36,23 +39,29 @@ struct GemmParams {
   void* aux; int aux_dt; int64_t aux_ld;
   const void* skip; int skip_dt; int64_t skip_ld; float skip_coef, out_coef;
   unsigned int* status;
+  int staged;                               // 1: epilogue goes through shared memory and TMA (see epilogue_staged)
 };
 
 constexpr int kBM = 128;                 // tile rows = TMEM lanes
 constexpr int kStageKBytes = 128;        // bytes of K per stage = one swizzle atom
 constexpr int kKSteps = 4;               // MMAs per stage (32 bytes of K each)
-constexpr int kGemmThreads = 192;
+constexpr int kEpilogueWarps = 8;           // two per TMEM lane quarter, each takes every other 32-column slice
+constexpr int kGemmThreads = 64 + 32 * kEpilogueWarps;
+constexpr int kEpiWarpBytes = 8192;
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr unsigned int kStatusTimeout = 1;
 
-template <int BN>
+// Shared-memory plan of one CTA.  CG = CTAs cooperating on a tile (1, or 2 = cta_group::2 pair):
+// a pair computes 256 x BN, each CTA holding its 128 rows of A and its BN/2 rows of B.
+template <int BN, int CG>
 struct GemmSmem {
   static constexpr int kABytes = kBM * kStageKBytes;
-  static constexpr int kBBytes = BN * kStageKBytes;
+  static constexpr int kBBytes = (BN / CG) * kStageKBytes;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = (BN == 256) ? 4 : 6;
-  static constexpr int kBarrierBytes = 256;
-  static constexpr int kTotal = kStages * kStageBytes + kBarrierBytes + 1024;  // + alignment slack
+  static constexpr int kEpiBytes = kEpilogueWarps * kEpiWarpBytes;   // two 4 KB staging boxes per epilogue warp
+  static constexpr int kStages = (229376 - kEpiBytes) / kStageBytes; // 5 x 32 KB or 3 x 48 KB next to the 64 KB above
+  static constexpr int kBarrierBytes = 512;
+  static constexpr int kTotal = kStages * kStageBytes + kEpiBytes + kBarrierBytes + 1024;  // + alignment slack
 };
 
 // Bounded mbarrier wait.  Returns false if the CTA is aborting (this wait or another one timed out).
@@ -67,137 +76,410 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
   return false;
 }
 
-// One 32-column slice of one output row: v holds scale * acc on entry.
-template <bool kFull>
-__device__ __forceinline__ void epilogue_chunk(const GemmParams& p, float (&v)[32], int64_t row, int col, int ncols) {
-  // kFull: all 32 columns are inside the matrix and every access is a 16-byte vector.
-  if (p.act == US_ACT_GELU) {
-    if (p.aux) {
-      if (kFull) {
-        store_vec<32>(static_cast<char*>(p.aux) + (row * p.aux_ld + col) * 2, p.aux_dt, v);
-      } else {
+// Operands of the fused epilogue for one 32-column slice of one row, fetched as raw 16-byte
+// vectors before the accumulator is read so that their latency overlaps the TMEM load.
+struct EpiloguePrefetch {
+  uint4 aux[4];    // 32 x 16-bit stored pre-activation (GELU-gradient only)
+  uint4 skip[8];   // 32 x float32, or 32 x 16-bit in the first four
+};
+
+__device__ __forceinline__ void prefetch_full(const GemmParams& p, int64_t row, int col, EpiloguePrefetch& f) {
+  if (p.act == US_ACT_GELU_GRAD) {
+    const uint4* q = reinterpret_cast<const uint4*>(static_cast<const char*>(p.aux) + (row * p.aux_ld + col) * 2);
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (i < ncols) store_one(p.aux, p.aux_dt, row * p.aux_ld + col + i, v[i]);
-      }
+    for (int i = 0; i < 4; ++i) f.aux[i] = __ldg(q + i);
+  }
+  if (p.skip) {
+    const int es = dtype_size(p.skip_dt);
+    const uint4* q = reinterpret_cast<const uint4*>(static_cast<const char*>(p.skip) + (row * p.skip_ld + col) * es);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) f.skip[i] = __ldg(q + i);
+    if (es == 4) {
+#pragma unroll
+      for (int i = 4; i < 8; ++i) f.skip[i] = __ldg(q + i);
     }
+  }
+}
+
+template <int N>
+__device__ __forceinline__ void unpack16(const uint4* raw, int dt, float (&v)[N]) {
+#pragma unroll
+  for (int i = 0; i < N / 8; ++i) {
+    const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 t = (dt == US_BF16) ? unpack_bf16x2(w[j]) : unpack_f16x2(w[j]);
+      v[8 * i + 2 * j] = t.x; v[8 * i + 2 * j + 1] = t.y;
+    }
+  }
+}
+
+// Full 32-column slice of one output row, every access a 16-byte vector; v = scale * acc on entry.
+__device__ __forceinline__ void epilogue_chunk_full(const GemmParams& p, float (&v)[32], const EpiloguePrefetch& f,
+                                                    int64_t row, int col) {
+  if (p.act == US_ACT_GELU) {
+    if (p.aux) store_vec<32>(static_cast<char*>(p.aux) + (row * p.aux_ld + col) * 2, p.aux_dt, v);
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = gelu_scaled(v[i], p.act_in, p.act_out);
   } else if (p.act == US_ACT_GELU_GRAD) {
     float h[32];
-    if (kFull) {
-      load_vec<32>(static_cast<const char*>(p.aux) + (row * p.aux_ld + col) * 2, p.aux_dt, h);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i) h[i] = (i < ncols) ? load_one(p.aux, p.aux_dt, row * p.aux_ld + col + i) : 0.f;
-    }
+    unpack16<32>(f.aux, p.aux_dt, h);
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = gelu_grad_scaled(h[i], v[i], p.act_in, p.act_out);
   }
   if (p.skip) {
-    float s[32];
-    if (kFull) {
-      load_vec<32>(static_cast<const char*>(p.skip) + (row * p.skip_ld + col) * dtype_size(p.skip_dt), p.skip_dt, s);
-    } else {
+    float sk[32];
+    if (p.skip_dt == US_F32) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) s[i] = (i < ncols) ? load_one(p.skip, p.skip_dt, row * p.skip_ld + col + i) : 0.f;
+      for (int i = 0; i < 8; ++i) {
+        sk[4 * i] = __uint_as_float(f.skip[i].x); sk[4 * i + 1] = __uint_as_float(f.skip[i].y);
+        sk[4 * i + 2] = __uint_as_float(f.skip[i].z); sk[4 * i + 3] = __uint_as_float(f.skip[i].w);
+      }
+    } else {
+      unpack16<32>(f.skip, p.skip_dt, sk);
     }
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = fmaf(p.skip_coef, s[i], p.out_coef * v[i]);
+    for (int i = 0; i < 32; ++i) v[i] = fmaf(p.skip_coef, sk[i], p.out_coef * v[i]);
   }
-  if (kFull) {
-    store_vec<32>(static_cast<char*>(p.out) + (row * p.out_ld + col) * dtype_size(p.out_dt), p.out_dt, v);
-  } else {
+  store_vec<32>(static_cast<char*>(p.out) + (row * p.out_ld + col) * dtype_size(p.out_dt), p.out_dt, v);
+}
+
+// Ragged 32-column slice (fewer than 32 columns inside the matrix): element-wise accesses.
+__device__ __forceinline__ void epilogue_chunk_ragged(const GemmParams& p, float (&v)[32], int64_t row, int col, int ncols) {
+  if (p.act == US_ACT_GELU) {
+    if (p.aux) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i)
-      if (i < ncols) store_one(p.out, p.out_dt, row * p.out_ld + col + i, v[i]);
+      for (int i = 0; i < 32; ++i)
+        if (i < ncols) store_one(p.aux, p.aux_dt, row * p.aux_ld + col + i, v[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = gelu_scaled(v[i], p.act_in, p.act_out);
+  } else if (p.act == US_ACT_GELU_GRAD) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const float h = (i < ncols) ? load_one(p.aux, p.aux_dt, row * p.aux_ld + col + i) : 0.f;
+      v[i] = gelu_grad_scaled(h, v[i], p.act_in, p.act_out);
+    }
   }
+  if (p.skip) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const float sk = (i < ncols) ? load_one(p.skip, p.skip_dt, row * p.skip_ld + col + i) : 0.f;
+      v[i] = fmaf(p.skip_coef, sk, p.out_coef * v[i]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 32; ++i)
+    if (i < ncols) store_one(p.out, p.out_dt, row * p.out_ld + col + i, v[i]);
+}
+
+// Barrier addresses and identity the staged epilogue needs from the kernel.
+struct EpiCtx {
+  uint32_t tmem_base, acc_full0, acc_empty0, in_bar, buf0;   // buf0: this warp's two 4 KB boxes
+  volatile int* abort_flag;
+  int warp, lane, rank, group, num_groups, num_tiles;
+};
+
+// Epilogue through shared memory.  Each participating warp owns 32 rows x 128 columns of the
+// tile and two private 32-row x 128-byte boxes (128-byte-swizzled, like the TMA maps).  A row of a
+// box is written / read by the lane that owns that row, 16-byte chunk c at chunk (c ^ (row & 7)),
+// which is conflict free; global memory is touched by TMA only: box loads for the stored
+// pre-activation (GELU gradient) or the skip tensor, box stores for the output and for the
+// pre-activation the GELU epilogue keeps.  TMA clips stores and zero-fills loads at the matrix
+// edges, so ragged shapes need no special path.  No cross-warp synchronisation is involved.
+template <int BN, int CG>
+__device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUtensorMap* tm_out, const CUtensorMap* tm_aux,
+                                                const CUtensorMap* tm_skip, const EpiCtx& c) {
+  constexpr int kWarpCols = 128;
+  const int q = c.warp & 3, half = (c.warp - 2) >> 2;
+  if (half >= BN / kWarpCols) return;                       // BN = 128: one warp per lane quarter
+  const int lane = c.lane;
+  const int in_kind = p.act == US_ACT_GELU_GRAD ? 1 : (p.skip ? 2 : 0);
+  const int in_dt = in_kind == 1 ? p.aux_dt : p.skip_dt;
+  const int in_es = in_kind ? dtype_size(in_dt) : 4;
+  const CUtensorMap* tm_in = in_kind == 1 ? tm_aux : tm_skip;
+  const bool aux_out = p.act == US_ACT_GELU && p.aux != nullptr;
+  const int out_es = dtype_size(p.out_dt);
+  const int in_box_cols = 128 / in_es, out_box_cols = 128 / out_es;
+  const uint32_t buf_in = c.buf0, buf_aux = c.buf0;          // first box: input, or the kept pre-activation
+  const uint32_t row_off = (uint32_t)lane * 128u;
+  const uint32_t sw = (uint32_t)(lane & 7);
+  uint32_t in_phase = 0;
+  int plain_toggle = 0;
+  uint32_t buf_out = c.buf0 + 4096u;
+
+  auto tile_rows = [&](int tile) { return (tile % p.tiles_m) * (kBM * CG) + c.rank * kBM + q * 32; };
+  auto tile_cols = [&](int tile) { return (tile / p.tiles_m) * BN + half * kWarpCols; };
+  auto next_active_tile = [&](int tile) {
+    while (tile < c.num_tiles && tile_cols(tile) >= p.N) tile += c.num_groups;
+    return tile;
+  };
+  auto issue_in = [&](int col, int row0) {
+    if (lane == 0) {
+      ptx::mbar_expect_tx(c.in_bar, 4096);
+      ptx::tma_load_2d(buf_in, tm_in, c.in_bar, col, row0);
+    }
+  };
+  if (in_kind) {
+    const int t0 = next_active_tile(c.group);
+    if (t0 < c.num_tiles) issue_in(tile_cols(t0), tile_rows(t0));
+  }
+
+  uint32_t local = 0;
+  bool ok = true;
+  for (int tile = c.group; ok && tile < c.num_tiles; tile += c.num_groups, ++local) {
+    const uint32_t acc = local & 1u, acc_phase = (local >> 1) & 1u;
+    const int row0 = tile_rows(tile), n_w = tile_cols(tile);
+    ok = wait_bounded(c.acc_full0 + 8u * acc, acc_phase, c.abort_flag, p.status);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) break;
+    ptx::tc_fence_after_sync();
+    const uint32_t t_row = c.tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + half * kWarpCols;
+    if (n_w < p.N) {
+#pragma unroll 1
+      for (int sl = 0; sl < kWarpCols / 32; ++sl) {
+        const int col = n_w + 32 * sl;
+        if (col >= p.N) break;                               // warp-uniform
+        const bool last_slice = (sl == kWarpCols / 32 - 1) || (col + 32 >= p.N);
+        // ---- fused-epilogue operand for this slice, from the input box
+        uint4 raw[8];
+        if (in_kind) {
+          const int off = (32 * sl) % in_box_cols;
+          if (off == 0) {
+            ok = wait_bounded(c.in_bar, in_phase, c.abort_flag, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            in_phase ^= 1u;
+          }
+          const uint32_t cb = (uint32_t)(off * in_es) >> 4;
+          const int nchunk = 2 * in_es;                      // 32 values
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (j < nchunk) raw[j] = ptx::lds128(buf_in + row_off + (((cb + j) ^ sw) << 4));
+          if (off + 32 == in_box_cols || last_slice) {       // box consumed: fetch the next one into it
+            __syncwarp();
+            if (!last_slice) {
+              issue_in(col + 32, row0);
+            } else {
+              const int tn = next_active_tile(tile + c.num_groups);
+              if (tn < c.num_tiles) issue_in(tile_cols(tn), tile_rows(tn));
+            }
+          }
+        }
+        float v[32];
+        ptx::tmem_ld_32x32(t_row + 32 * sl, v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] *= p.scale;
+        // ---- pre-activation kept for the backward pass (16-bit, two slices per box)
+        if (aux_out) {
+          const int off = (32 * sl) % 64;
+          if (off == 0) {
+            if (lane == 0) ptx::bulk_wait_group_read<0>();
+            __syncwarp();
+          }
+          const uint32_t cb = (uint32_t)(off * 2) >> 4;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t w[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              w[k] = p.aux_dt == US_BF16 ? pack_bf16x2(v[8 * j + 2 * k], v[8 * j + 2 * k + 1])
+                                         : pack_f16x2(v[8 * j + 2 * k], v[8 * j + 2 * k + 1]);
+            ptx::sts128(buf_aux + row_off + (((cb + j) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+          }
+          if (off == 32 || last_slice) {
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) { ptx::tma_store_2d(tm_aux, buf_aux, col - off, row0); ptx::bulk_commit_group(); }
+          }
+        }
+        // ---- activation and residual
+        if (p.act == US_ACT_GELU) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = gelu_scaled(v[i], p.act_in, p.act_out);
+        } else if (p.act == US_ACT_GELU_GRAD) {
+          float h[32];
+          unpack16<32>(raw, in_dt, h);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = gelu_grad_scaled(h[i], v[i], p.act_in, p.act_out);
+        }
+        if (in_kind == 2) {
+          float sk[32];
+          if (in_dt == US_F32) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              sk[4 * i] = __uint_as_float(raw[i].x); sk[4 * i + 1] = __uint_as_float(raw[i].y);
+              sk[4 * i + 2] = __uint_as_float(raw[i].z); sk[4 * i + 3] = __uint_as_float(raw[i].w);
+            }
+          } else {
+            unpack16<32>(raw, in_dt, sk);
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = fmaf(p.skip_coef, sk[i], p.out_coef * v[i]);
+        }
+        // ---- output box
+        {
+          const int off = (32 * sl) % out_box_cols;
+          if (off == 0) {
+            if (!in_kind && !aux_out) {                      // both boxes hold outputs, used alternately
+              buf_out = c.buf0 + (plain_toggle ? 4096u : 0u);
+              plain_toggle ^= 1;
+              if (lane == 0) ptx::bulk_wait_group_read<1>();
+            } else {
+              if (lane == 0) ptx::bulk_wait_group_read<0>();
+            }
+            __syncwarp();
+          }
+          const uint32_t cb = (uint32_t)(off * out_es) >> 4;
+          const uint32_t dst = buf_out + row_off;
+          if (p.out_dt == US_F32) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              ptx::sts128(dst + (((cb + j) ^ sw) << 4),
+                          make_uint4(__float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]),
+                                     __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3])));
+          } else if (p.out_dt == US_BF16 || p.out_dt == US_F16) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t w[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                w[k] = p.out_dt == US_BF16 ? pack_bf16x2(v[8 * j + 2 * k], v[8 * j + 2 * k + 1])
+                                           : pack_f16x2(v[8 * j + 2 * k], v[8 * j + 2 * k + 1]);
+              ptx::sts128(dst + (((cb + j) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              uint32_t w[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float* e = &v[16 * j + 4 * k];
+                w[k] = p.out_dt == US_E5M2 ? cvt_fp8x4<true>(e[0], e[1], e[2], e[3]) : cvt_fp8x4<false>(e[0], e[1], e[2], e[3]);
+              }
+              ptx::sts128(dst + (((cb + j) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+            }
+          }
+          if (off + 32 == out_box_cols || last_slice) {
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) { ptx::tma_store_2d(tm_out, buf_out, col - off, row0); ptx::bulk_commit_group(); }
+          }
+        }
+      }
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) break;
+    ptx::tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) {
+      if (CG == 2) ptx::mbar_arrive_cluster(ptx::in_even_cta(c.acc_empty0 + 8u * acc));
+      else ptx::mbar_arrive(c.acc_empty0 + 8u * acc);
+    }
+  }
+  if (lane == 0) ptx::bulk_wait_group_read<0>();             // stores have left shared memory before the CTA may exit
+  __syncwarp();
 }
 
 // ES: operand element size in bytes (1 = FP8, 2 = BF16 / F16).
 // A_MN / B_MN: operand stored MN-major ([K x M] resp. [K x N] row-major) instead of K-major.
-template <int ES, bool A_MN, bool B_MN, int BN>
+// CG: 1 = every CTA computes its own 128 x BN tiles; 2 = clusters of two CTAs compute 256 x BN
+//     tiles with tcgen05.mma.cta_group::2 (the even CTA issues, both load and both run an epilogue).
+template <int ES, bool A_MN, bool B_MN, int BN, int CG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-            const GemmParams p) {
-  using S = GemmSmem<BN>;
+            const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_aux,
+            const __grid_constant__ CUtensorMap tmap_skip, const GemmParams p) {
+  using S = GemmSmem<BN, CG>;
   constexpr int kBK = kStageKBytes / ES;            // K elements per stage
   constexpr int kChunkElems = 128 / ES;             // MN elements per 128-byte row of an MN-major tile
   constexpr uint32_t kChunkBytes = kBK * 128;       // one MN-major chunk: kBK rows of 128 bytes
   constexpr uint32_t kTmemCols = 2 * BN;            // two accumulators
+  constexpr int kBRows = BN / CG;                   // B rows (N indices) this CTA loads
+  static_assert(CG == 1 || (kBRows % kChunkElems) == 0, "pair tiles need whole 128-byte chunks of N per CTA");
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
-  const uint32_t bars = smem_base + S::kStages * S::kStageBytes;
-  // barrier layout (8 bytes each): full[kStages], empty[kStages], acc_full[2], acc_empty[2], drained
+  const uint32_t epi_base = smem_base + S::kStages * S::kStageBytes;      // 1024-byte aligned staging boxes
+  const uint32_t bars = epi_base + S::kEpiBytes;
+  // barrier layout (8 bytes each): full[kStages], empty[kStages], acc_full[2], acc_empty[2], drained, epi_in[8]
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (S::kStages + s); };
   auto acc_full_bar = [&](int a) { return bars + 8u * (2 * S::kStages + a); };
   auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * S::kStages + 2 + a); };
   const uint32_t drained_bar = bars + 8u * (2 * S::kStages + 4);
-  uint8_t* tail = smem_gen + S::kStages * S::kStageBytes + 8 * (2 * S::kStages + 5);
+  auto epi_in_bar = [&](int w) { return bars + 8u * (2 * S::kStages + 5 + w); };
+  uint8_t* tail = smem_gen + S::kStages * S::kStageBytes + S::kEpiBytes + 8 * (2 * S::kStages + 5 + kEpilogueWarps);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int rank = (CG == 2) ? (int)ptx::cluster_ctarank() : 0;     // position in the pair
+  const int group = blockIdx.x / CG, num_groups = gridDim.x / CG;   // tile-walking unit: CTA or pair
+  const int num_tiles = p.tiles_m * p.tiles_n;                      // tiles of (128 * CG) x BN
   const int num_kb = (p.K + kBK - 1) / kBK;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::kStages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full_bar(a), 1); ptx::mbar_init(acc_empty_bar(a), 4); }
+    const int epi_arrivals = p.staged ? CG * 4 * (BN / 128) : CG * kEpilogueWarps;
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full_bar(a), 1); ptx::mbar_init(acc_empty_bar(a), epi_arrivals); }
     ptx::mbar_init(drained_bar, 1);
+    for (int w = 0; w < kEpilogueWarps; ++w) ptx::mbar_init(epi_in_bar(w), 1);
     *abort_flag = 0;
     ptx::mbar_init_fence();
     ptx::prefetch_tensormap(&tmap_a);
     ptx::prefetch_tensormap(&tmap_b);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
-    ptx::tmem_relinquish();
+    if (CG == 2) { ptx::tmem_alloc_pair(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), kTmemCols); ptx::tmem_relinquish_pair(); }
+    else { ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), kTmemCols); ptx::tmem_relinquish(); }
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
+  if (CG == 2) ptx::cluster_sync();                  // the partner's barriers and TMEM are ready too
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ TMA producer (every CTA)
     if (lane == 0) {
       uint32_t issued = 0;
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-        const int m0 = (tile % p.tiles_m) * kBM;
-        const int n0 = (tile / p.tiles_m) * BN;
+      for (int tile = group; ok && tile < num_tiles; tile += num_groups) {
+        const int m0 = (tile % p.tiles_m) * (kBM * CG) + rank * kBM;
+        const int n0 = (tile / p.tiles_m) * BN + rank * kBRows;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
           if (!ok) break;
           const uint32_t a_dst = smem_base + stage * S::kStageBytes;
           const uint32_t b_dst = a_dst + S::kABytes;
           const int k0 = kb * kBK;
-          ptx::mbar_expect_tx(full_bar(stage), S::kStageBytes);
+          // bytes of the whole tile stage are counted on the (even CTA's) full barrier
+          const uint32_t fb = (CG == 2) ? ptx::in_even_cta(full_bar(stage)) : full_bar(stage);
+          if (rank == 0) ptx::mbar_expect_tx(full_bar(stage), CG * S::kStageBytes);
+          auto load = [&](uint32_t dst, const void* tm, int x, int y) {
+            if (CG == 2) ptx::tma_load_2d_pair(dst, tm, fb, x, y); else ptx::tma_load_2d(dst, tm, fb, x, y);
+          };
           if (A_MN) {
 #pragma unroll
-            for (int c = 0; c < kBM / kChunkElems; ++c)
-              ptx::tma_load_2d(a_dst + c * kChunkBytes, &tmap_a, full_bar(stage), m0 + c * kChunkElems, k0);
+            for (int c = 0; c < kBM / kChunkElems; ++c) load(a_dst + c * kChunkBytes, &tmap_a, m0 + c * kChunkElems, k0);
           } else {
-            ptx::tma_load_2d(a_dst, &tmap_a, full_bar(stage), k0, m0);
+            load(a_dst, &tmap_a, k0, m0);
           }
           if (B_MN) {
 #pragma unroll
-            for (int c = 0; c < BN / kChunkElems; ++c)
-              ptx::tma_load_2d(b_dst + c * kChunkBytes, &tmap_b, full_bar(stage), n0 + c * kChunkElems, k0);
+            for (int c = 0; c < kBRows / kChunkElems; ++c) load(b_dst + c * kChunkBytes, &tmap_b, n0 + c * kChunkElems, k0);
           } else {
-            ptx::tma_load_2d(b_dst, &tmap_b, full_bar(stage), k0, n0);
+            load(b_dst, &tmap_b, k0, n0);
           }
           ++issued;
           if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (*abort_flag) {
+      if (*abort_flag && rank == 0) {
         // Let copies that are still in flight land before the CTA gives up its shared memory.
         const uint32_t n = issued < (uint32_t)S::kStages ? issued : (uint32_t)S::kStages;
         for (uint32_t i = 0; i < n; ++i) {
@@ -208,12 +490,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------ MMA issuer (even CTA of a pair only)
+    if (lane == 0 && rank == 0) {
       int stage = 0; uint32_t phase = 0;
       uint32_t local = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+      for (int tile = group; ok && tile < num_tiles; tile += num_groups, ++local) {
         const uint32_t acc = local & 1u, acc_phase = (local >> 1) & 1u;
         ok = wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status);
         if (!ok) break;
@@ -232,58 +514,80 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
                                         : ptx::smem_desc_sw128(a_src + k * 32, 16, 1024);
             const uint64_t bdesc = B_MN ? ptx::smem_desc_sw128(b_src + k * (kChunkBytes / kKSteps), kChunkBytes, 1024)
                                         : ptx::smem_desc_sw128(b_src + k * 32, 16, 1024);
-            ptx::mma_ss<ES == 1>(d_tmem, adesc, bdesc, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            if (CG == 2) ptx::mma_ss_pair<ES == 1>(d_tmem, adesc, bdesc, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            else ptx::mma_ss<ES == 1>(d_tmem, adesc, bdesc, p.idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          ptx::mma_commit(empty_bar(stage));        // stage reusable once these MMAs have read it
+          // stage reusable (in both CTAs of a pair) once these MMAs have read it
+          if (CG == 2) ptx::mma_commit_pair(empty_bar(stage), 3); else ptx::mma_commit(empty_bar(stage));
           if (++stage == S::kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) ptx::mma_commit(acc_full_bar(acc));  // accumulator complete
+        if (ok) {                                     // accumulator complete
+          if (CG == 2) ptx::mma_commit_pair(acc_full_bar(acc), 3); else ptx::mma_commit(acc_full_bar(acc));
+        }
       }
       if (*abort_flag) {
-        ptx::mma_commit(drained_bar);
+        if (CG == 2) ptx::mma_commit_pair(drained_bar, 1); else ptx::mma_commit(drained_bar);
         for (uint32_t it = 0; it < kWaitLimit && !ptx::mbar_try_wait(drained_bar, 0); ++it) {}
       }
     }
+  } else if (p.staged) {
+    // ------------------------------------------------------------ epilogue warps, through shared memory + TMA
+    EpiCtx c;
+    c.tmem_base = tmem_base; c.acc_full0 = acc_full_bar(0); c.acc_empty0 = acc_empty_bar(0);
+    c.in_bar = epi_in_bar(warp - 2); c.buf0 = epi_base + (warp - 2) * kEpiWarpBytes;
+    c.abort_flag = abort_flag; c.warp = warp; c.lane = lane; c.rank = rank;
+    c.group = group; c.num_groups = num_groups; c.num_tiles = num_tiles;
+    epilogue_staged<BN, CG>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
   } else {
-    // ------------------------------------------------------------ epilogue warps
+    // ------------------------------------------------------------ epilogue warps, direct global accesses
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;                // which of the two interleaved sets of 32-column slices
     uint32_t local = 0;
     bool ok = true;
-    const bool vec_ok = true;                        // host guarantees 16-byte aligned rows
-    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+    for (int tile = group; ok && tile < num_tiles; tile += num_groups, ++local) {
       const uint32_t acc = local & 1u, acc_phase = (local >> 1) & 1u;
-      const int m0 = (tile % p.tiles_m) * kBM;
+      const int m0 = (tile % p.tiles_m) * (kBM * CG) + rank * kBM;
       const int n0 = (tile / p.tiles_m) * BN;
+      const int64_t row = m0 + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      EpiloguePrefetch pf;
+      const int c_first = 32 * half;
+      if (row_ok && n0 + c_first + 32 <= p.N) prefetch_full(p, row, n0 + c_first, pf);
       ok = wait_bounded(acc_full_bar(acc), acc_phase, abort_flag, p.status);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       ptx::tc_fence_after_sync();
-      const int64_t row = m0 + q * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN;
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = c_first; c < BN; c += 64) {
         if (n0 + c >= p.N) break;                    // warp-uniform
         float v[32];
         ptx::tmem_ld_32x32(t_row + c, v);
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] *= p.scale;
-        if (row < p.M) {
-          const int ncols = min(32, p.N - (n0 + c));
-          if (vec_ok && ncols == 32) epilogue_chunk<true>(p, v, row, n0 + c, 32);
-          else epilogue_chunk<false>(p, v, row, n0 + c, ncols);
+        const int ncols = min(32, p.N - (n0 + c));
+        if (row_ok) {
+          if (ncols == 32) epilogue_chunk_full(p, v, pf, row, n0 + c);
+          else epilogue_chunk_ragged(p, v, row, n0 + c, ncols);
         }
+        // operands of this warp's next slice, in flight while the next TMEM load is issued
+        if (row_ok && c + 64 < BN && n0 + c + 64 + 32 <= p.N) prefetch_full(p, row, n0 + c + 64, pf);
       }
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(acc_empty_bar(acc));
+      if (lane == 0) {                               // the issuing (even) CTA owns the accumulator-free barrier
+        if (CG == 2) ptx::mbar_arrive_cluster(ptx::in_even_cta(acc_empty_bar(acc)));
+        else ptx::mbar_arrive(acc_empty_bar(acc));
+      }
     }
   }
 
   ptx::tc_fence_before_sync();
   __syncthreads();
+  if (CG == 2) ptx::cluster_sync();                  // no CTA leaves while its partner may still signal it
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    if (CG == 2) ptx::tmem_dealloc_pair(tmem_base, kTmemCols); else ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
