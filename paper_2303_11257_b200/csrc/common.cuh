@@ -127,47 +127,41 @@ __device__ __forceinline__ void store_one(void* base, int dt, int64_t idx, float
 }
 
 // ---------------------------------------------------------------- scaled GELU
-// Normal CDF pieces from the rational approximation 7.1.26 of Abramowitz & Stegun
-// (|error in erf| <= 1.5e-7): with x = |z| / sqrt 2 and t = 1 / (1 + p x),
-//   erfc(x) ~ (a1 t + a2 t^2 + a3 t^3 + a4 t^4 + a5 t^5) exp(-x^2).
-// Returns q = Phi(-|z|) and e = exp(-z^2 / 2); Phi(z) = z >= 0 ? 1 - q : q.
-__device__ __forceinline__ float rcp_approx(float x) {
-  float r;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-  return r;
-}
+// Lower normal tail q(a) = Phi(-a), a = |z|, as 2^R(a) with R a degree-6 polynomial fitted to
+// log2 Phi(-a) on [0, 7.5] (fit_normal_tail.py regenerates the coefficients): one ex2 and six FMAs,
+// |q error| <= 2.7e-7, |a q error| <= 1.5e-7 in float32.  Beyond 7.5 the tail is below 4e-14 and a
+// is clamped.  Phi(z) = z >= 0 ? 1 - q : q, and gelu(z) = z Phi(z) = max(z, 0) - |z| q(|z|).
 __device__ __forceinline__ float ex2_approx(float x) {
   float r;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
   return r;
 }
-__device__ __forceinline__ void normal_tail(float z, float& q, float& e) {
-  const float az = fabsf(z);
-  const float t = rcp_approx(fmaf(0.3275911f * 0.70710678118654752f, az, 1.0f));
-  e = ex2_approx((-0.72134752044448170f * z) * z);  // exp(-z^2/2) = 2^(-z^2 log2(e) / 2)
-  float p = 0.5f * 1.061405429f;
-  p = fmaf(p, t, 0.5f * -1.453152027f);
-  p = fmaf(p, t, 0.5f * 1.421413741f);
-  p = fmaf(p, t, 0.5f * -0.284496736f);
-  p = fmaf(p, t, 0.5f * 0.254829592f);
-  q = p * t * e;
+__device__ __forceinline__ float normal_tail(float z) {
+  const float a = fminf(fabsf(z), 7.5f);
+  float r = 2.772329208e-05f;
+  r = fmaf(r, a, -7.209949545e-04f);
+  r = fmaf(r, a, 7.917892188e-03f);
+  r = fmaf(r, a, -5.315330625e-02f);
+  r = fmaf(r, a, -4.589684010e-01f);
+  r = fmaf(r, a, -1.151137114e+00f);
+  r = fmaf(r, a, -9.999993443e-01f);
+  return ex2_approx(r);
 }
 
 // out_scale * gelu(in_scale * h), gelu(x) = x Phi(x)
 __device__ __forceinline__ float gelu_scaled(float h, float in_scale, float out_scale) {
   const float z = in_scale * h;
-  float q, e;
-  normal_tail(z, q, e);
-  const float Phi = z >= 0.f ? 1.0f - q : q;
-  return (out_scale * z) * Phi;
+  const float q = normal_tail(z);
+  const float oz = out_scale * z;
+  return fmaf(-fabsf(oz), q, fmaxf(oz, 0.f));
 }
 
 // out_scale * in_scale * gelu'(in_scale * h) * g, gelu'(x) = Phi(x) + x phi(x)
 __device__ __forceinline__ float gelu_grad_scaled(float h, float g, float in_scale, float out_scale) {
   const float z = in_scale * h;
-  float q, e;
-  normal_tail(z, q, e);
+  const float q = normal_tail(z);
   const float Phi = z >= 0.f ? 1.0f - q : q;
+  const float e = ex2_approx((-0.72134752044448170f * z) * z);   // exp(-z^2 / 2) = 2^(-z^2 log2(e) / 2)
   const float d = fmaf(z * 0.39894228040143268f, e, Phi);
   return (out_scale * in_scale) * d * g;
 }

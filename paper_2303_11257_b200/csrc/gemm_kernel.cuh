@@ -495,27 +495,40 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int stage = 0; uint32_t phase = 0;
       uint32_t local = 0;
       bool ok = true;
+      // The issuing thread is a single instruction stream that has to start four MMAs every ~500
+      // cycles, so the loop body is kept minimal: descriptors differ from stage to stage and from
+      // k-step to k-step only in their 14-bit start-address field, i.e. by adding a constant to the
+      // low word (no carry: shared memory addresses / 16 stay below 2^14).
+      const uint64_t a_desc0 = A_MN ? ptx::smem_desc_sw128(smem_base, kChunkBytes, 1024) : ptx::smem_desc_sw128(smem_base, 16, 1024);
+      const uint64_t b_desc0 = B_MN ? ptx::smem_desc_sw128(smem_base + S::kABytes, kChunkBytes, 1024)
+                                    : ptx::smem_desc_sw128(smem_base + S::kABytes, 16, 1024);
+      const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), b_hi = (uint32_t)(b_desc0 >> 32);
+      const uint32_t a_lo0 = (uint32_t)a_desc0, b_lo0 = (uint32_t)b_desc0;
+      constexpr uint32_t kStageStep = S::kStageBytes >> 4;
+      constexpr uint32_t kAStep = (A_MN ? kChunkBytes / kKSteps : 32u) >> 4;   // K-major: 32 bytes along the row
+      constexpr uint32_t kBStep = (B_MN ? kChunkBytes / kKSteps : 32u) >> 4;   // MN-major: kBK/4 rows of 128 bytes
+      const uint32_t idesc = p.idesc;
       for (int tile = group; ok && tile < num_tiles; tile += num_groups, ++local) {
         const uint32_t acc = local & 1u, acc_phase = (local >> 1) & 1u;
         ok = wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status);
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
+        uint32_t accumulate = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status);
-          if (!ok) break;
+          if (!ptx::mbar_try_wait(full_bar(stage), phase)) {
+            ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status);
+            if (!ok) break;
+          }
           ptx::tc_fence_after_sync();
-          const uint32_t a_src = smem_base + stage * S::kStageBytes;
-          const uint32_t b_src = a_src + S::kABytes;
+          const uint32_t a_lo = a_lo0 + stage * kStageStep, b_lo = b_lo0 + stage * kStageStep;
 #pragma unroll
           for (int k = 0; k < kKSteps; ++k) {
-            // K-major: 32 bytes further along the swizzled row.  MN-major: kBK/4 rows of 128 bytes further.
-            const uint64_t adesc = A_MN ? ptx::smem_desc_sw128(a_src + k * (kChunkBytes / kKSteps), kChunkBytes, 1024)
-                                        : ptx::smem_desc_sw128(a_src + k * 32, 16, 1024);
-            const uint64_t bdesc = B_MN ? ptx::smem_desc_sw128(b_src + k * (kChunkBytes / kKSteps), kChunkBytes, 1024)
-                                        : ptx::smem_desc_sw128(b_src + k * 32, 16, 1024);
-            if (CG == 2) ptx::mma_ss_pair<ES == 1>(d_tmem, adesc, bdesc, p.idesc, (kb | k) != 0 ? 1u : 0u);
-            else ptx::mma_ss<ES == 1>(d_tmem, adesc, bdesc, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            const uint64_t adesc = ((uint64_t)a_hi << 32) | (a_lo + k * kAStep);
+            const uint64_t bdesc = ((uint64_t)b_hi << 32) | (b_lo + k * kBStep);
+            if (CG == 2) ptx::mma_ss_pair<ES == 1>(d_tmem, adesc, bdesc, idesc, accumulate);
+            else ptx::mma_ss<ES == 1>(d_tmem, adesc, bdesc, idesc, accumulate);
+            accumulate = 1;
           }
           // stage reusable (in both CTAs of a pair) once these MMAs have read it
           if (CG == 2) ptx::mma_commit_pair(empty_bar(stage), 3); else ptx::mma_commit(empty_bar(stage));
