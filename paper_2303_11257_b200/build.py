@@ -13,7 +13,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libunitscale.so")
 SOURCES = ["host.cu", "elementwise.cu", "gemm.cu", "static_ws.cu"]
-HEADERS = ["common.cuh", "sm100.cuh", "gemm_kernel.cuh", "host.h", os.path.join("..", "..", "include", "unitscale.h")]
+# (operand bytes, A MN-major, B MN-major): forward, backward-input, backward-weight for FP8 and 16-bit operands
+GEMM_PARTS = [(1, 0, 1), (1, 0, 0), (1, 1, 1), (2, 0, 1), (2, 0, 0), (2, 1, 1)]
+HEADERS = ["common.cuh", "sm100.cuh", "gemm_kernel.cuh", "gemm_launch.h", "gemm_inst.cu", "host.h", os.path.join("..", "..", "include", "unitscale.h")]
 
 
 def _nvcc() -> str:
@@ -31,22 +33,40 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def _compile(args):
+    res = subprocess.run(args, capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("nvcc failed:\n" + " ".join(args) + "\n" + res.stdout + res.stderr)
+    return res.stderr
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the library if it is missing or older than its sources; returns its path."""
+    """Compile the library if it is missing or older than its sources; returns its path.
+
+    Every translation unit is compiled to an object in parallel (gemm_inst.cu once per operand
+    width and layout), then linked into libunitscale.so next to this file."""
     if not force and not _stale():
         return LIB
-    cmd = [
-        _nvcc(), "-std=c++17", "-O3", "-lineinfo",
-        "-gencode", "arch=compute_100a,code=sm_100a",
-        "-Xcompiler", "-fPIC", "-shared",
-        "-Xptxas", "-v" if verbose else "-O3",
-        "-o", LIB,
-    ] + [os.path.join(CSRC, f) for f in SOURCES] + ["-lcudart"]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    from concurrent.futures import ThreadPoolExecutor
+    objdir = os.path.join(HERE, "_build")
+    os.makedirs(objdir, exist_ok=True)
+    common = [_nvcc(), "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
+              "-Xcompiler", "-fPIC", "-Xptxas", "-v" if verbose else "-O3", "-c"]
+    jobs, objs = [], []
+    for f in SOURCES:
+        o = os.path.join(objdir, f.replace(".cu", ".o"))
+        objs.append(o)
+        jobs.append(common + ["-o", o, os.path.join(CSRC, f)])
+    for es, amn, bmn in GEMM_PARTS:
+        o = os.path.join(objdir, f"gemm_inst_{es}_{amn}_{bmn}.o")
+        objs.append(o)
+        jobs.append(common + [f"-DUS_INST_ES={es}", f"-DUS_INST_AMN={amn}", f"-DUS_INST_BMN={bmn}", "-o", o,
+                              os.path.join(CSRC, "gemm_inst.cu")])
+    with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 4)) as pool:
+        logs = list(pool.map(_compile, jobs))
+    _compile([_nvcc(), "-shared", "-o", LIB] + objs + ["-lcudart"])
     if verbose:
-        print(res.stderr)
+        print("\n".join(logs))
     return LIB
 
 

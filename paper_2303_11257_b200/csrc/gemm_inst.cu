@@ -1,0 +1,112 @@
+// Kernel instantiations of the unit-scaled GEMM for one (operand width, A layout, B layout)
+// combination, selected by the macros US_INST_ES, US_INST_AMN, US_INST_BMN.  The build compiles
+// this file once per combination, in parallel.
+#include <cuda.h>
+
+#include "gemm_kernel.cuh"
+#include "gemm_launch.h"
+#include "host.h"
+
+#ifndef US_INST_ES
+#error "compile with -DUS_INST_ES=<1|2> -DUS_INST_AMN=<0|1> -DUS_INST_BMN=<0|1>"
+#endif
+
+namespace us {
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+// Tensor map over a row-major matrix [rows x cols] of ES-byte elements with a 128-byte-wide,
+// 128-byte-swizzled box of `box_rows` rows.  Out-of-range parts of a box read as zero.
+static bool make_tmap(CUtensorMap* tm, const us_mat* m, int es, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const CUtensorMapDataType type = es == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                 : es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32;
+  cuuint64_t dims[2] = {(cuuint64_t)m->cols, (cuuint64_t)m->rows};
+  cuuint64_t strides[1] = {(cuuint64_t)m->ld * es};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, type, 2, m->ptr, dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int ES, bool A_MN, bool B_MN, int BN, int CG, int EPI>
+static us_status launch(const us_mat* A, const us_mat* B, const GemmParams& p, const EpiMats& em, cudaStream_t stream) {
+  constexpr int kBK = kStageKBytes / ES;
+  CUtensorMap ta, tb, t_out, t_aux, t_skip;
+  if (!make_tmap(&ta, A, ES, A_MN ? kBK : kBM)) return US_ERR_CUDA;
+  if (!make_tmap(&tb, B, ES, B_MN ? kBK : BN / CG)) return US_ERR_CUDA;
+  // epilogue boxes: 32 rows x 128 bytes; unused maps alias the output's so that every parameter is valid
+  if (!make_tmap(&t_out, em.out, dtype_size(em.out->dtype), 32)) return US_ERR_CUDA;
+  t_aux = t_out; t_skip = t_out;
+  if (EPI != kEpiLegacy && em.aux && !make_tmap(&t_aux, em.aux, dtype_size(em.aux->dtype), 32)) return US_ERR_CUDA;
+  if (EPI != kEpiLegacy && em.skip && !make_tmap(&t_skip, em.skip, dtype_size(em.skip->dtype), 32)) return US_ERR_CUDA;
+  auto kern = gemm_kernel<ES, A_MN, B_MN, BN, CG, EPI>;
+  constexpr int smem = GemmSmem<BN, CG>::kTotal;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return US_ERR_CUDA;
+  const int sms = host::sm_count();
+  if (sms <= 0) return US_ERR_CUDA;
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int groups = sms / CG;                        // one CTA per SM; pairs share a TPC
+  const int grid = CG * (tiles < groups ? tiles : groups);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CG; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, ta, tb, t_out, t_aux, t_skip, p) == cudaSuccess ? US_OK : US_ERR_CUDA;
+}
+
+template <int ES, bool A_MN, bool B_MN, int BN, int CG>
+static us_status pick_epilogue(const us_mat* A, const us_mat* B, const GemmParams& p, const EpiMats& em, int epi,
+                               cudaStream_t stream) {
+  switch (epi) {
+    case kEpiPlain:    return launch<ES, A_MN, B_MN, BN, CG, kEpiPlain>(A, B, p, em, stream);
+    case kEpiGelu:     return launch<ES, A_MN, B_MN, BN, CG, kEpiGelu>(A, B, p, em, stream);
+    case kEpiGeluGrad: return launch<ES, A_MN, B_MN, BN, CG, kEpiGeluGrad>(A, B, p, em, stream);
+    case kEpiSkip:     return launch<ES, A_MN, B_MN, BN, CG, kEpiSkip>(A, B, p, em, stream);
+    default:           return launch<ES, A_MN, B_MN, BN, CG, kEpiLegacy>(A, B, p, em, stream);
+  }
+}
+
+}  // namespace
+
+template <int ES, bool A_MN, bool B_MN>
+us_status launch_gemm(const us_mat* A, const us_mat* B, GemmParams& p, const EpiMats& em, int epi, cudaStream_t stream) {
+  // CTA pairs with 256 x 256 tiles whenever such a tile is not mostly empty; 128 x 128 tiles otherwise.
+  const bool pair = p.N > 128 && p.M > kBM;
+  const int bn = pair ? 256 : 128, cg = pair ? 2 : 1;
+  p.tiles_m = (p.M + kBM * cg - 1) / (kBM * cg);
+  p.tiles_n = (p.N + bn - 1) / bn;
+  p.idesc = (p.idesc & ~((0x3fu << 17) | (0x1fu << 24))) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((kBM * cg) >> 4) << 24);
+  return pair ? pick_epilogue<ES, A_MN, B_MN, 256, 2>(A, B, p, em, epi, stream)
+              : pick_epilogue<ES, A_MN, B_MN, 128, 1>(A, B, p, em, epi, stream);
+}
+
+template us_status launch_gemm<US_INST_ES, (US_INST_AMN != 0), (US_INST_BMN != 0)>(const us_mat*, const us_mat*, GemmParams&,
+                                                                                 const EpiMats&, int, cudaStream_t);
+
+}  // namespace us

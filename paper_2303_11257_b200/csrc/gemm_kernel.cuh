@@ -39,7 +39,6 @@ struct GemmParams {
   void* aux; int aux_dt; int64_t aux_ld;
   const void* skip; int skip_dt; int64_t skip_ld; float skip_coef, out_coef;
   unsigned int* status;
-  int staged;                               // 1: epilogue goes through shared memory and TMA (see epilogue_staged)
 };
 
 constexpr int kBM = 128;                 // tile rows = TMEM lanes
@@ -48,6 +47,15 @@ constexpr int kKSteps = 4;               // MMAs per stage (32 bytes of K each)
 constexpr int kEpilogueWarps = 8;           // two per TMEM lane quarter, each takes every other 32-column slice
 constexpr int kGemmThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kEpiWarpBytes = 8192;
+
+// What the epilogue fuses, fixed at compile time so that each kernel carries one code path only.
+enum EpiKind {
+  kEpiPlain = 0,     // scale, round, store
+  kEpiGelu = 1,      // + scaled GELU, optionally keeping the 16-bit pre-activation
+  kEpiGeluGrad = 2,  // + scaled GELU gradient from the stored pre-activation
+  kEpiSkip = 3,      // + weighted skip tensor (residual)
+  kEpiLegacy = 4     // any other combination: direct global accesses, runtime switches
+};
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr unsigned int kStatusTimeout = 1;
 
@@ -187,18 +195,18 @@ struct EpiCtx {
 // pre-activation (GELU gradient) or the skip tensor, box stores for the output and for the
 // pre-activation the GELU epilogue keeps.  TMA clips stores and zero-fills loads at the matrix
 // edges, so ragged shapes need no special path.  No cross-warp synchronisation is involved.
-template <int BN, int CG>
+template <int BN, int CG, int EPI>
 __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUtensorMap* tm_out, const CUtensorMap* tm_aux,
                                                 const CUtensorMap* tm_skip, const EpiCtx& c) {
   constexpr int kWarpCols = 128;
   const int q = c.warp & 3, half = (c.warp - 2) >> 2;
   if (half >= BN / kWarpCols) return;                       // BN = 128: one warp per lane quarter
   const int lane = c.lane;
-  const int in_kind = p.act == US_ACT_GELU_GRAD ? 1 : (p.skip ? 2 : 0);
+  constexpr int in_kind = EPI == kEpiGeluGrad ? 1 : (EPI == kEpiSkip ? 2 : 0);
   const int in_dt = in_kind == 1 ? p.aux_dt : p.skip_dt;
   const int in_es = in_kind ? dtype_size(in_dt) : 4;
   const CUtensorMap* tm_in = in_kind == 1 ? tm_aux : tm_skip;
-  const bool aux_out = p.act == US_ACT_GELU && p.aux != nullptr;
+  const bool aux_out = EPI == kEpiGelu && p.aux != nullptr;
   const int out_es = dtype_size(p.out_dt);
   const int in_box_cols = 128 / in_es, out_box_cols = 128 / out_es;
   const uint32_t buf_in = c.buf0, buf_aux = c.buf0;          // first box: input, or the kept pre-activation
@@ -294,10 +302,10 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
           }
         }
         // ---- activation and residual
-        if (p.act == US_ACT_GELU) {
+        if (EPI == kEpiGelu) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = gelu_scaled(v[i], p.act_in, p.act_out);
-        } else if (p.act == US_ACT_GELU_GRAD) {
+        } else if (EPI == kEpiGeluGrad) {
           float h[32];
           unpack16<32>(raw, in_dt, h);
 #pragma unroll
@@ -383,9 +391,10 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
 
 // ES: operand element size in bytes (1 = FP8, 2 = BF16 / F16).
 // A_MN / B_MN: operand stored MN-major ([K x M] resp. [K x N] row-major) instead of K-major.
+// EPI: the fused epilogue (EpiKind).
 // CG: 1 = every CTA computes its own 128 x BN tiles; 2 = clusters of two CTAs compute 256 x BN
 //     tiles with tcgen05.mma.cta_group::2 (the even CTA issues, both load and both run an epilogue).
-template <int ES, bool A_MN, bool B_MN, int BN, int CG>
+template <int ES, bool A_MN, bool B_MN, int BN, int CG, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_aux,
@@ -423,7 +432,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::kStages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
-    const int epi_arrivals = p.staged ? CG * 4 * (BN / 128) : CG * kEpilogueWarps;
+    const int epi_arrivals = EPI != kEpiLegacy ? CG * 4 * (BN / 128) : CG * kEpilogueWarps;
     for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full_bar(a), 1); ptx::mbar_init(acc_empty_bar(a), epi_arrivals); }
     ptx::mbar_init(drained_bar, 1);
     for (int w = 0; w < kEpilogueWarps; ++w) ptx::mbar_init(epi_in_bar(w), 1);
@@ -543,14 +552,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         for (uint32_t it = 0; it < kWaitLimit && !ptx::mbar_try_wait(drained_bar, 0); ++it) {}
       }
     }
-  } else if (p.staged) {
+  } else if (EPI != kEpiLegacy) {
     // ------------------------------------------------------------ epilogue warps, through shared memory + TMA
     EpiCtx c;
     c.tmem_base = tmem_base; c.acc_full0 = acc_full_bar(0); c.acc_empty0 = acc_empty_bar(0);
     c.in_bar = epi_in_bar(warp - 2); c.buf0 = epi_base + (warp - 2) * kEpiWarpBytes;
     c.abort_flag = abort_flag; c.warp = warp; c.lane = lane; c.rank = rank;
     c.group = group; c.num_groups = num_groups; c.num_tiles = num_tiles;
-    epilogue_staged<BN, CG>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
+    epilogue_staged<BN, CG, EPI>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
   } else {
     // ------------------------------------------------------------ epilogue warps, direct global accesses
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
