@@ -30,9 +30,11 @@ __device__ __forceinline__ uint16_t cvt_e5m2x2(float lo, float hi) {
 }
 template <bool E5>
 __device__ __forceinline__ uint32_t cvt_fp8x4(float a, float b, float c, float d) {
-  uint32_t lo = E5 ? cvt_e5m2x2(a, b) : cvt_e4m3x2(a, b);
-  uint32_t hi = E5 ? cvt_e5m2x2(c, d) : cvt_e4m3x2(c, d);
-  return lo | (hi << 16);
+  const uint32_t lo = E5 ? cvt_e5m2x2(a, b) : cvt_e4m3x2(a, b);
+  const uint32_t hi = E5 ? cvt_e5m2x2(c, d) : cvt_e4m3x2(c, d);
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, 0x5410;" : "=r"(r) : "r"(lo), "r"(hi));   // low halves of lo and hi, one instruction
+  return r;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -164,6 +166,75 @@ __device__ __forceinline__ float gelu_grad_scaled(float h, float g, float in_sca
   const float e = ex2_approx((-0.72134752044448170f * z) * z);   // exp(-z^2 / 2) = 2^(-z^2 log2(e) / 2)
   const float d = fmaf(z * 0.39894228040143268f, e, Phi);
   return (out_scale * in_scale) * d * g;
+}
+
+// ---------------------------------------------------------------- two floats per instruction
+// sm_100 executes add / mul / fma on pairs of float32 held in a 64-bit register (same IEEE
+// rounding per lane as the scalar forms); the GEMM epilogues use it to halve the number of
+// issued arithmetic instructions.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 splat2(float x) { return pack2(x, x); }
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+
+// q(|z|) for two arguments (see normal_tail).
+__device__ __forceinline__ void normal_tail2(f32x2 z, float& q0, float& q1) {
+  float z0, z1;
+  unpack2(z, z0, z1);
+  const f32x2 a = pack2(fminf(fabsf(z0), 7.5f), fminf(fabsf(z1), 7.5f));
+  f32x2 r = splat2(2.772329208e-05f);
+  r = fma2(r, a, splat2(-7.209949545e-04f));
+  r = fma2(r, a, splat2(7.917892188e-03f));
+  r = fma2(r, a, splat2(-5.315330625e-02f));
+  r = fma2(r, a, splat2(-4.589684010e-01f));
+  r = fma2(r, a, splat2(-1.151137114e+00f));
+  r = fma2(r, a, splat2(-9.999993443e-01f));
+  float r0, r1;
+  unpack2(r, r0, r1);
+  q0 = ex2_approx(r0);
+  q1 = ex2_approx(r1);
+}
+
+// gelu_scaled for two values: h holds the pre-activations, in2 / out2 the splatted scales.
+__device__ __forceinline__ void gelu_scaled2(f32x2 h, f32x2 in2, f32x2 out2, float& y0, float& y1) {
+  const f32x2 z = mul2(in2, h);
+  float q0, q1;
+  normal_tail2(z, q0, q1);
+  float oz0, oz1;
+  unpack2(mul2(out2, z), oz0, oz1);
+  y0 = fmaf(-fabsf(oz0), q0, fmaxf(oz0, 0.f));
+  y1 = fmaf(-fabsf(oz1), q1, fmaxf(oz1, 0.f));
+}
+
+// gelu_grad_scaled for two values: h = stored pre-activations, g = incoming gradients,
+// in2 = splat(in_scale), os2 = splat(out_scale * in_scale).
+__device__ __forceinline__ f32x2 gelu_grad_scaled2(f32x2 h, f32x2 g, f32x2 in2, f32x2 os2) {
+  const f32x2 z = mul2(in2, h);
+  float q0, q1, z0, z1;
+  normal_tail2(z, q0, q1);
+  unpack2(z, z0, z1);
+  const f32x2 Phi = pack2(z0 >= 0.f ? 1.0f - q0 : q0, z1 >= 0.f ? 1.0f - q1 : q1);
+  float e0, e1;
+  unpack2(mul2(mul2(splat2(-0.72134752044448170f), z), z), e0, e1);
+  const f32x2 e = pack2(ex2_approx(e0), ex2_approx(e1));
+  const f32x2 d = fma2(mul2(z, splat2(0.39894228040143268f)), e, Phi);
+  return mul2(mul2(os2, d), g);
 }
 
 }  // namespace us

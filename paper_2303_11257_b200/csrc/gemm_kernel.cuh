@@ -249,7 +249,8 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
         const int col = n_w + 32 * sl;
         if (col >= p.N) break;                               // warp-uniform
         const bool last_slice = (sl == kWarpCols / 32 - 1) || (col + 32 >= p.N);
-        // ---- fused-epilogue operand for this slice, from the input box
+        // ---- fused-epilogue operand for this slice: read it from the input box up front, so that
+        //      the box can be refilled while the slice is being computed
         uint4 raw[8];
         if (in_kind) {
           const int off = (32 * sl) % in_box_cols;
@@ -274,105 +275,107 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
             }
           }
         }
+        // ---- staging boxes that start with this slice must have been read by their last TMA store
+        const int aux_off = (32 * sl) % 64, out_off = (32 * sl) % out_box_cols;
+        if (out_off == 0 || (aux_out && aux_off == 0)) {
+          if (!in_kind && !aux_out) {                        // both boxes hold outputs, used alternately
+            buf_out = c.buf0 + (plain_toggle ? 4096u : 0u);
+            plain_toggle ^= 1;
+            if (lane == 0) ptx::bulk_wait_group_read<1>();
+          } else {
+            if (lane == 0) ptx::bulk_wait_group_read<0>();
+          }
+          __syncwarp();
+        }
         float v[32];
         ptx::tmem_ld_32x32(t_row + 32 * sl, v);
+        const f32x2 scale2 = splat2(p.scale), in2 = splat2(p.act_in), out2 = splat2(p.act_out);
+        const f32x2 os2 = splat2(p.act_out * p.act_in), skip2 = splat2(p.skip_coef), oc2 = splat2(p.out_coef);
+        const uint32_t aux_cb = (uint32_t)(aux_off * 2) >> 4, out_cb = (uint32_t)(out_off * out_es) >> 4;
+        const uint32_t dst = buf_out + row_off;
+        uint32_t held[2];                                    // first half of a 16-byte chunk of FP8 codes
+        // Eight values at a time run through the whole chain (scale, kept pre-activation, activation,
+        // residual, rounding, staging store), so that the different execution pipes overlap.
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] *= p.scale;
-        // ---- pre-activation kept for the backward pass (16-bit, two slices per box)
-        if (aux_out) {
-          const int off = (32 * sl) % 64;
-          if (off == 0) {
-            if (lane == 0) ptx::bulk_wait_group_read<0>();
-            __syncwarp();
-          }
-          const uint32_t cb = (uint32_t)(off * 2) >> 4;
+        for (int g = 0; g < 4; ++g) {
+          f32x2 x[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint32_t w[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              w[k] = p.aux_dt == US_BF16 ? pack_bf16x2(v[8 * j + 2 * k], v[8 * j + 2 * k + 1])
-                                         : pack_f16x2(v[8 * j + 2 * k], v[8 * j + 2 * k + 1]);
-            ptx::sts128(buf_aux + row_off + (((cb + j) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
-          }
-          if (off == 32 || last_slice) {
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) { ptx::tma_store_2d(tm_aux, buf_aux, col - off, row0); ptx::bulk_commit_group(); }
-          }
-        }
-        // ---- activation and residual
-        if (EPI == kEpiGelu) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = gelu_scaled(v[i], p.act_in, p.act_out);
-        } else if (EPI == kEpiGeluGrad) {
-          float h[32];
-          unpack16<32>(raw, in_dt, h);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = gelu_grad_scaled(h[i], v[i], p.act_in, p.act_out);
-        }
-        if (in_kind == 2) {
-          float sk[32];
-          if (in_dt == US_F32) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              sk[4 * i] = __uint_as_float(raw[i].x); sk[4 * i + 1] = __uint_as_float(raw[i].y);
-              sk[4 * i + 2] = __uint_as_float(raw[i].z); sk[4 * i + 3] = __uint_as_float(raw[i].w);
-            }
-          } else {
-            unpack16<32>(raw, in_dt, sk);
-          }
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = fmaf(p.skip_coef, sk[i], p.out_coef * v[i]);
-        }
-        // ---- output box
-        {
-          const int off = (32 * sl) % out_box_cols;
-          if (off == 0) {
-            if (!in_kind && !aux_out) {                      // both boxes hold outputs, used alternately
-              buf_out = c.buf0 + (plain_toggle ? 4096u : 0u);
-              plain_toggle ^= 1;
-              if (lane == 0) ptx::bulk_wait_group_read<1>();
-            } else {
-              if (lane == 0) ptx::bulk_wait_group_read<0>();
-            }
-            __syncwarp();
-          }
-          const uint32_t cb = (uint32_t)(off * out_es) >> 4;
-          const uint32_t dst = buf_out + row_off;
-          if (p.out_dt == US_F32) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-              ptx::sts128(dst + (((cb + j) ^ sw) << 4),
-                          make_uint4(__float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]),
-                                     __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3])));
-          } else if (p.out_dt == US_BF16 || p.out_dt == US_F16) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint32_t w[4];
-#pragma unroll
-              for (int k = 0; k < 4; ++k)
-                w[k] = p.out_dt == US_BF16 ? pack_bf16x2(v[8 * j + 2 * k], v[8 * j + 2 * k + 1])
-                                           : pack_f16x2(v[8 * j + 2 * k], v[8 * j + 2 * k + 1]);
-              ptx::sts128(dst + (((cb + j) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
+          for (int k = 0; k < 4; ++k) x[k] = mul2(pack2(v[8 * g + 2 * k], v[8 * g + 2 * k + 1]), scale2);
+          float y[8];
+          if (EPI == kEpiGelu) {
+            if (aux_out) {
               uint32_t w[4];
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
-                const float* e = &v[16 * j + 4 * k];
-                w[k] = p.out_dt == US_E5M2 ? cvt_fp8x4<true>(e[0], e[1], e[2], e[3]) : cvt_fp8x4<false>(e[0], e[1], e[2], e[3]);
+                float a, b;
+                unpack2(x[k], a, b);
+                w[k] = p.aux_dt == US_BF16 ? pack_bf16x2(a, b) : pack_f16x2(a, b);
               }
-              ptx::sts128(dst + (((cb + j) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+              ptx::sts128(buf_aux + row_off + (((aux_cb + g) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) gelu_scaled2(x[k], in2, out2, y[2 * k], y[2 * k + 1]);
+          } else if (EPI == kEpiGeluGrad) {
+            const uint32_t w[4] = {raw[g].x, raw[g].y, raw[g].z, raw[g].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float2 h = in_dt == US_BF16 ? unpack_bf16x2(w[k]) : unpack_f16x2(w[k]);
+              unpack2(gelu_grad_scaled2(pack2(h.x, h.y), x[k], in2, os2), y[2 * k], y[2 * k + 1]);
+            }
+          } else if (EPI == kEpiSkip) {
+            float sk[8];
+            if (in_dt == US_F32) {
+              sk[0] = __uint_as_float(raw[2 * g].x); sk[1] = __uint_as_float(raw[2 * g].y);
+              sk[2] = __uint_as_float(raw[2 * g].z); sk[3] = __uint_as_float(raw[2 * g].w);
+              sk[4] = __uint_as_float(raw[2 * g + 1].x); sk[5] = __uint_as_float(raw[2 * g + 1].y);
+              sk[6] = __uint_as_float(raw[2 * g + 1].z); sk[7] = __uint_as_float(raw[2 * g + 1].w);
+            } else {
+              const uint32_t w[4] = {raw[g].x, raw[g].y, raw[g].z, raw[g].w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float2 h = in_dt == US_BF16 ? unpack_bf16x2(w[k]) : unpack_f16x2(w[k]);
+                sk[2 * k] = h.x; sk[2 * k + 1] = h.y;
+              }
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              unpack2(fma2(skip2, pack2(sk[2 * k], sk[2 * k + 1]), mul2(oc2, x[k])), y[2 * k], y[2 * k + 1]);
+          } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) unpack2(x[k], y[2 * k], y[2 * k + 1]);
+          }
+          // ---- rounding to the output format and staging store of these eight values
+          if (p.out_dt == US_F32) {
+            ptx::sts128(dst + (((out_cb + 2 * g) ^ sw) << 4),
+                        make_uint4(__float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3])));
+            ptx::sts128(dst + (((out_cb + 2 * g + 1) ^ sw) << 4),
+                        make_uint4(__float_as_uint(y[4]), __float_as_uint(y[5]), __float_as_uint(y[6]), __float_as_uint(y[7])));
+          } else if (p.out_dt == US_BF16 || p.out_dt == US_F16) {
+            uint32_t w[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              w[k] = p.out_dt == US_BF16 ? pack_bf16x2(y[2 * k], y[2 * k + 1]) : pack_f16x2(y[2 * k], y[2 * k + 1]);
+            ptx::sts128(dst + (((out_cb + g) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+          } else {
+            const uint32_t lo = p.out_dt == US_E5M2 ? cvt_fp8x4<true>(y[0], y[1], y[2], y[3]) : cvt_fp8x4<false>(y[0], y[1], y[2], y[3]);
+            const uint32_t hi = p.out_dt == US_E5M2 ? cvt_fp8x4<true>(y[4], y[5], y[6], y[7]) : cvt_fp8x4<false>(y[4], y[5], y[6], y[7]);
+            if ((g & 1) == 0) {
+              held[0] = lo; held[1] = hi;
+            } else {
+              ptx::sts128(dst + (((out_cb + (g >> 1)) ^ sw) << 4), make_uint4(held[0], held[1], lo, hi));
             }
           }
-          if (off + 32 == out_box_cols || last_slice) {
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) { ptx::tma_store_2d(tm_out, buf_out, col - off, row0); ptx::bulk_commit_group(); }
-          }
+        }
+        // ---- boxes completed by this slice go out
+        if (aux_out && (aux_off == 32 || last_slice)) {
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) { ptx::tma_store_2d(tm_aux, buf_aux, col - aux_off, row0); ptx::bulk_commit_group(); }
+        }
+        if (out_off + 32 == out_box_cols || last_slice) {
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) { ptx::tma_store_2d(tm_out, buf_out, col - out_off, row0); ptx::bulk_commit_group(); }
         }
       }
     }
