@@ -31,36 +31,37 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map over a row-major matrix [rows x cols] of ES-byte elements with a 128-byte-wide,
-// 128-byte-swizzled box of `box_rows` rows.  Out-of-range parts of a box read as zero.
-static bool make_tmap(CUtensorMap* tm, const us_mat* m, int es, int box_rows) {
+// Tensor map over a row-major matrix [rows x cols] of ES-byte elements with a box of `box_rows` rows
+// and `box_bytes` (128, or 64) bytes per row, swizzled with the pattern of that width.  Out-of-range parts of a box read as zero.
+static bool make_tmap(CUtensorMap* tm, const us_mat* m, int es, int box_rows, int box_bytes = 128) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const CUtensorMapDataType type = es == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                                  : es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32;
   cuuint64_t dims[2] = {(cuuint64_t)m->cols, (cuuint64_t)m->rows};
   cuuint64_t strides[1] = {(cuuint64_t)m->ld * es};
-  cuuint32_t box[2] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows};
+  cuuint32_t box[2] = {(cuuint32_t)(box_bytes / es), (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(tm, type, 2, m->ptr, dims,
-                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
-template <int ES, bool A_MN, bool B_MN, int BN, int CG, int EPI>
+template <int ES, bool A_MN, bool B_MN, int BN, int CG, int EPI, int EW>
 static us_status launch(const us_mat* A, const us_mat* B, const GemmParams& p, const EpiMats& em, cudaStream_t stream) {
   constexpr int kBK = kStageKBytes / ES;
   CUtensorMap ta, tb, t_out, t_aux, t_skip;
   if (!make_tmap(&ta, A, ES, A_MN ? kBK : kBM)) return US_ERR_CUDA;
   if (!make_tmap(&tb, B, ES, B_MN ? kBK : BN / CG)) return US_ERR_CUDA;
   // epilogue boxes: 32 rows x 128 bytes; unused maps alias the output's so that every parameter is valid
-  if (!make_tmap(&t_out, em.out, dtype_size(em.out->dtype), 32)) return US_ERR_CUDA;
+  if (!make_tmap(&t_out, em.out, dtype_size(em.out->dtype), 32, EW == 16 ? 64 : 128)) return US_ERR_CUDA;
   t_aux = t_out; t_skip = t_out;
   if (EPI != kEpiLegacy && em.aux && !make_tmap(&t_aux, em.aux, dtype_size(em.aux->dtype), 32)) return US_ERR_CUDA;
   if (EPI != kEpiLegacy && em.skip && !make_tmap(&t_skip, em.skip, dtype_size(em.skip->dtype), 32)) return US_ERR_CUDA;
-  auto kern = gemm_kernel<ES, A_MN, B_MN, BN, CG, EPI>;
-  constexpr int smem = GemmSmem<BN, CG>::kTotal;
+  auto kern = gemm_kernel<ES, A_MN, B_MN, BN, CG, EPI, EW>;
+  constexpr int smem = GemmSmem<BN, CG, EW>::kTotal;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return US_ERR_CUDA;
   const int sms = host::sm_count();
   if (sms <= 0) return US_ERR_CUDA;
@@ -69,7 +70,7 @@ static us_status launch(const us_mat* A, const us_mat* B, const GemmParams& p, c
   const int grid = CG * (tiles < groups ? tiles : groups);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kGemmThreads);
+  cfg.blockDim = dim3(gemm_threads(EW));
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -83,12 +84,17 @@ static us_status launch(const us_mat* A, const us_mat* B, const GemmParams& p, c
 template <int ES, bool A_MN, bool B_MN, int BN, int CG>
 static us_status pick_epilogue(const us_mat* A, const us_mat* B, const GemmParams& p, const EpiMats& em, int epi,
                                cudaStream_t stream) {
+  // The GELU epilogues with an FP8 output (the FFN's forward and backward hidden layer) are ALU
+  // bound with eight epilogue warps; they run with sixteen.
+  const bool fp8_out = em.out->dtype == US_E4M3 || em.out->dtype == US_E5M2;
   switch (epi) {
-    case kEpiPlain:    return launch<ES, A_MN, B_MN, BN, CG, kEpiPlain>(A, B, p, em, stream);
-    case kEpiGelu:     return launch<ES, A_MN, B_MN, BN, CG, kEpiGelu>(A, B, p, em, stream);
-    case kEpiGeluGrad: return launch<ES, A_MN, B_MN, BN, CG, kEpiGeluGrad>(A, B, p, em, stream);
-    case kEpiSkip:     return launch<ES, A_MN, B_MN, BN, CG, kEpiSkip>(A, B, p, em, stream);
-    default:           return launch<ES, A_MN, B_MN, BN, CG, kEpiLegacy>(A, B, p, em, stream);
+    case kEpiPlain:    return launch<ES, A_MN, B_MN, BN, CG, kEpiPlain, 8>(A, B, p, em, stream);
+    case kEpiGelu:     return fp8_out ? launch<ES, A_MN, B_MN, BN, CG, kEpiGelu, 16>(A, B, p, em, stream)
+                                      : launch<ES, A_MN, B_MN, BN, CG, kEpiGelu, 8>(A, B, p, em, stream);
+    case kEpiGeluGrad: return fp8_out ? launch<ES, A_MN, B_MN, BN, CG, kEpiGeluGrad, 16>(A, B, p, em, stream)
+                                      : launch<ES, A_MN, B_MN, BN, CG, kEpiGeluGrad, 8>(A, B, p, em, stream);
+    case kEpiSkip:     return launch<ES, A_MN, B_MN, BN, CG, kEpiSkip, 8>(A, B, p, em, stream);
+    default:           return launch<ES, A_MN, B_MN, BN, CG, kEpiLegacy, 8>(A, B, p, em, stream);
   }
 }
 

@@ -44,9 +44,13 @@ struct GemmParams {
 constexpr int kBM = 128;                 // tile rows = TMEM lanes
 constexpr int kStageKBytes = 128;        // bytes of K per stage = one swizzle atom
 constexpr int kKSteps = 4;               // MMAs per stage (32 bytes of K each)
-constexpr int kEpilogueWarps = 8;           // two per TMEM lane quarter, each takes every other 32-column slice
-constexpr int kGemmThreads = 64 + 32 * kEpilogueWarps;
-constexpr int kEpiWarpBytes = 8192;
+constexpr int kEpilogueWarps = 8;           // default: two per TMEM lane quarter
+// Epilogue warps EW of a kernel: 8, or 16 for the ALU-heavy GELU epilogues with FP8 output (four
+// per lane quarter, 64 columns each), which need more warps in flight to keep the pipes busy.
+__host__ __device__ constexpr int gemm_threads(int ew) { return 64 + 32 * ew; }
+// Staging per epilogue warp: EW = 8: two 32-row x 128-byte boxes; EW = 16: one such box (stored
+// pre-activation in or out, 64 columns of 16 bits) and one 32-row x 64-byte box (64 FP8 outputs).
+__host__ __device__ constexpr int epi_warp_bytes(int ew) { return ew == 16 ? 4096 + 2048 : 8192; }
 
 // What the epilogue fuses, fixed at compile time so that each kernel carries one code path only.
 enum EpiKind {
@@ -61,13 +65,13 @@ constexpr unsigned int kStatusTimeout = 1;
 
 // Shared-memory plan of one CTA.  CG = CTAs cooperating on a tile (1, or 2 = cta_group::2 pair):
 // a pair computes 256 x BN, each CTA holding its 128 rows of A and its BN/2 rows of B.
-template <int BN, int CG>
+template <int BN, int CG, int EW>
 struct GemmSmem {
   static constexpr int kABytes = kBM * kStageKBytes;
   static constexpr int kBBytes = (BN / CG) * kStageKBytes;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kEpiBytes = kEpilogueWarps * kEpiWarpBytes;   // two 4 KB staging boxes per epilogue warp
-  static constexpr int kStages = (229376 - kEpiBytes) / kStageBytes; // 5 x 32 KB or 3 x 48 KB next to the 64 KB above
+  static constexpr int kEpiBytes = EW * epi_warp_bytes(EW);          // 64 KB (EW = 8) or 96 KB (EW = 16)
+  static constexpr int kStages = (229376 - kEpiBytes) / kStageBytes; // 32 KB stages: 5 (EW = 8) or 4 (EW = 16)
   static constexpr int kBarrierBytes = 512;
   static constexpr int kTotal = kStages * kStageBytes + kEpiBytes + kBarrierBytes + 1024;  // + alignment slack
 };
@@ -195,12 +199,13 @@ struct EpiCtx {
 // pre-activation (GELU gradient) or the skip tensor, box stores for the output and for the
 // pre-activation the GELU epilogue keeps.  TMA clips stores and zero-fills loads at the matrix
 // edges, so ragged shapes need no special path.  No cross-warp synchronisation is involved.
-template <int BN, int CG, int EPI>
+template <int BN, int CG, int EPI, int EW>
 __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUtensorMap* tm_out, const CUtensorMap* tm_aux,
                                                 const CUtensorMap* tm_skip, const EpiCtx& c) {
-  constexpr int kWarpCols = 128;
-  const int q = c.warp & 3, half = (c.warp - 2) >> 2;
-  if (half >= BN / kWarpCols) return;                       // BN = 128: one warp per lane quarter
+  constexpr int kWarpCols = EW == 16 ? 64 : 128;            // columns of the tile one warp handles
+  constexpr bool kNarrowOut = EW == 16;                     // FP8 output box of 64 bytes per row (64-byte swizzle)
+  const int q = c.warp & 3, half = (c.warp - 2) >> 2;       // lane quarter; which group of kWarpCols columns
+  if (half >= BN / kWarpCols) return;                       // more warps than column groups: the rest sit out
   const int lane = c.lane;
   constexpr int in_kind = EPI == kEpiGeluGrad ? 1 : (EPI == kEpiSkip ? 2 : 0);
   const int in_dt = in_kind == 1 ? p.aux_dt : p.skip_dt;
@@ -208,10 +213,13 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
   const CUtensorMap* tm_in = in_kind == 1 ? tm_aux : tm_skip;
   const bool aux_out = EPI == kEpiGelu && p.aux != nullptr;
   const int out_es = dtype_size(p.out_dt);
-  const int in_box_cols = 128 / in_es, out_box_cols = 128 / out_es;
+  const int in_box_cols = 128 / in_es, out_box_cols = kNarrowOut ? 64 : 128 / out_es;
   const uint32_t buf_in = c.buf0, buf_aux = c.buf0;          // first box: input, or the kept pre-activation
   const uint32_t row_off = (uint32_t)lane * 128u;
   const uint32_t sw = (uint32_t)(lane & 7);
+  // 64-byte output rows: pitch 64, 16-byte chunk c of row r at chunk c ^ ((r >> 1) & 3)
+  const uint32_t out_row_off = kNarrowOut ? (uint32_t)lane * 64u : row_off;
+  const uint32_t out_sw = kNarrowOut ? (uint32_t)((lane >> 1) & 3) : sw;
   uint32_t in_phase = 0;
   int plain_toggle = 0;
   uint32_t buf_out = c.buf0 + 4096u;
@@ -292,7 +300,7 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
         const f32x2 scale2 = splat2(p.scale), in2 = splat2(p.act_in), out2 = splat2(p.act_out);
         const f32x2 os2 = splat2(p.act_out * p.act_in), skip2 = splat2(p.skip_coef), oc2 = splat2(p.out_coef);
         const uint32_t aux_cb = (uint32_t)(aux_off * 2) >> 4, out_cb = (uint32_t)(out_off * out_es) >> 4;
-        const uint32_t dst = buf_out + row_off;
+        const uint32_t dst = buf_out + out_row_off;
         uint32_t held[2];                                    // first half of a 16-byte chunk of FP8 codes
         // Eight values at a time run through the whole chain (scale, kept pre-activation, activation,
         // residual, rounding, staging store), so that the different execution pipes overlap.
@@ -346,23 +354,23 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
           }
           // ---- rounding to the output format and staging store of these eight values
           if (p.out_dt == US_F32) {
-            ptx::sts128(dst + (((out_cb + 2 * g) ^ sw) << 4),
+            ptx::sts128(dst + (((out_cb + 2 * g) ^ out_sw) << 4),
                         make_uint4(__float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3])));
-            ptx::sts128(dst + (((out_cb + 2 * g + 1) ^ sw) << 4),
+            ptx::sts128(dst + (((out_cb + 2 * g + 1) ^ out_sw) << 4),
                         make_uint4(__float_as_uint(y[4]), __float_as_uint(y[5]), __float_as_uint(y[6]), __float_as_uint(y[7])));
           } else if (p.out_dt == US_BF16 || p.out_dt == US_F16) {
             uint32_t w[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k)
               w[k] = p.out_dt == US_BF16 ? pack_bf16x2(y[2 * k], y[2 * k + 1]) : pack_f16x2(y[2 * k], y[2 * k + 1]);
-            ptx::sts128(dst + (((out_cb + g) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+            ptx::sts128(dst + (((out_cb + g) ^ out_sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
           } else {
             const uint32_t lo = p.out_dt == US_E5M2 ? cvt_fp8x4<true>(y[0], y[1], y[2], y[3]) : cvt_fp8x4<false>(y[0], y[1], y[2], y[3]);
             const uint32_t hi = p.out_dt == US_E5M2 ? cvt_fp8x4<true>(y[4], y[5], y[6], y[7]) : cvt_fp8x4<false>(y[4], y[5], y[6], y[7]);
             if ((g & 1) == 0) {
               held[0] = lo; held[1] = hi;
             } else {
-              ptx::sts128(dst + (((out_cb + (g >> 1)) ^ sw) << 4), make_uint4(held[0], held[1], lo, hi));
+              ptx::sts128(dst + (((out_cb + (g >> 1)) ^ out_sw) << 4), make_uint4(held[0], held[1], lo, hi));
             }
           }
         }
@@ -394,15 +402,16 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
 
 // ES: operand element size in bytes (1 = FP8, 2 = BF16 / F16).
 // A_MN / B_MN: operand stored MN-major ([K x M] resp. [K x N] row-major) instead of K-major.
-// EPI: the fused epilogue (EpiKind).
+// EPI: the fused epilogue (EpiKind).  EW: number of epilogue warps (8 or 16).
 // CG: 1 = every CTA computes its own 128 x BN tiles; 2 = clusters of two CTAs compute 256 x BN
 //     tiles with tcgen05.mma.cta_group::2 (the even CTA issues, both load and both run an epilogue).
-template <int ES, bool A_MN, bool B_MN, int BN, int CG, int EPI>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+template <int ES, bool A_MN, bool B_MN, int BN, int CG, int EPI, int EW>
+__global__ void __launch_bounds__(gemm_threads(EW), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_aux,
             const __grid_constant__ CUtensorMap tmap_skip, const GemmParams p) {
-  using S = GemmSmem<BN, CG>;
+  using S = GemmSmem<BN, CG, EW>;
+  static_assert(EW == 8 || (EW == 16 && (EPI == kEpiGelu || EPI == kEpiGeluGrad)), "16 epilogue warps serve the GELU epilogues only");
   constexpr int kBK = kStageKBytes / ES;            // K elements per stage
   constexpr int kChunkElems = 128 / ES;             // MN elements per 128-byte row of an MN-major tile
   constexpr uint32_t kChunkBytes = kBK * 128;       // one MN-major chunk: kBK rows of 128 bytes
@@ -422,7 +431,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * S::kStages + 2 + a); };
   const uint32_t drained_bar = bars + 8u * (2 * S::kStages + 4);
   auto epi_in_bar = [&](int w) { return bars + 8u * (2 * S::kStages + 5 + w); };
-  uint8_t* tail = smem_gen + S::kStages * S::kStageBytes + S::kEpiBytes + 8 * (2 * S::kStages + 5 + kEpilogueWarps);
+  uint8_t* tail = smem_gen + S::kStages * S::kStageBytes + S::kEpiBytes + 8 * (2 * S::kStages + 5 + EW);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
 
@@ -435,10 +444,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::kStages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
-    const int epi_arrivals = EPI != kEpiLegacy ? CG * 4 * (BN / 128) : CG * kEpilogueWarps;
+    const int epi_arrivals = EPI != kEpiLegacy ? CG * 4 * (BN / (EW == 16 ? 64 : 128)) : CG * kEpilogueWarps;
     for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full_bar(a), 1); ptx::mbar_init(acc_empty_bar(a), epi_arrivals); }
     ptx::mbar_init(drained_bar, 1);
-    for (int w = 0; w < kEpilogueWarps; ++w) ptx::mbar_init(epi_in_bar(w), 1);
+    for (int w = 0; w < EW; ++w) ptx::mbar_init(epi_in_bar(w), 1);
     *abort_flag = 0;
     ptx::mbar_init_fence();
     ptx::prefetch_tensormap(&tmap_a);
@@ -559,10 +568,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     // ------------------------------------------------------------ epilogue warps, through shared memory + TMA
     EpiCtx c;
     c.tmem_base = tmem_base; c.acc_full0 = acc_full_bar(0); c.acc_empty0 = acc_empty_bar(0);
-    c.in_bar = epi_in_bar(warp - 2); c.buf0 = epi_base + (warp - 2) * kEpiWarpBytes;
+    c.in_bar = epi_in_bar(warp - 2); c.buf0 = epi_base + (warp - 2) * epi_warp_bytes(EW);
     c.abort_flag = abort_flag; c.warp = warp; c.lane = lane; c.rank = rank;
     c.group = group; c.num_groups = num_groups; c.num_tiles = num_tiles;
-    epilogue_staged<BN, CG, EPI>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
+    epilogue_staged<BN, CG, EPI, EW>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
   } else {
     // ------------------------------------------------------------ epilogue warps, direct global accesses
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
