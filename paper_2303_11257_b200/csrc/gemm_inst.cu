@@ -107,6 +107,9 @@ us_status launch_gemm(const us_mat* A, const us_mat* B, GemmParams& p, const Epi
   const int bn = pair ? 256 : 128, cg = pair ? 2 : 1;
   p.tiles_m = (p.M + kBM * cg - 1) / (kBM * cg);
   p.tiles_n = (p.N + bn - 1) / bn;
+  // A (M x K operand) is re-read by every column of tiles: keep the plain order while it fits well
+  // inside the 126 MB L2, switch to bands of 8 tile rows beyond that.
+  p.band_m = ((long long)p.M * p.K * ES <= (80ll << 20)) ? p.tiles_m : 8;
   p.idesc = (p.idesc & ~((0x3fu << 17) | (0x1fu << 24))) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((kBM * cg) >> 4) << 24);
   return pair ? pick_epilogue<ES, A_MN, B_MN, 256, 2>(A, B, p, em, epi, stream)
               : pick_epilogue<ES, A_MN, B_MN, 128, 1>(A, B, p, em, epi, stream);

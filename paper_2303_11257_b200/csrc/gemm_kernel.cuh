@@ -32,6 +32,7 @@ namespace us {
 struct GemmParams {
   int M, N, K;
   int tiles_m, tiles_n;
+  int band_m;                               // tile rows per band of the tile order (see tile_mn)
   float scale;
   uint32_t idesc;
   void* out; int out_dt; int64_t out_ld;
@@ -75,6 +76,23 @@ struct GemmSmem {
   static constexpr int kBarrierBytes = 512;
   static constexpr int kTotal = kStages * kStageBytes + kEpiBytes + kBarrierBytes + 1024;  // + alignment slack
 };
+
+// Tile order.  Tiles that run at the same time (consecutive indices) should share operand panels
+// in L2: tiles are walked in bands of band_m tile-rows, down the band first and then across.  With
+// band_m = tiles_m this is plain column-major order (all of A stays resident in L2 while B streams
+// through once); when A is too large for that the host picks band_m = 8, so that a wave of ~74
+// tiles touches 8 row panels of A and ~9 column panels of B.
+__device__ __forceinline__ void tile_mn(const GemmParams& p, int tile, int& tm, int& tn) {
+  const int band_tiles = p.band_m * p.tiles_n;
+  const int band = tile / band_tiles;
+  const int first_m = band * p.band_m;
+  const int rows = min(p.band_m, p.tiles_m - first_m);
+  const int r = tile - band * band_tiles;
+  tm = first_m + r % rows;
+  tn = r / rows;
+}
+__device__ __forceinline__ int tile_m(const GemmParams& p, int tile) { int tm, tn; tile_mn(p, tile, tm, tn); return tm; }
+__device__ __forceinline__ int tile_n(const GemmParams& p, int tile) { int tm, tn; tile_mn(p, tile, tm, tn); return tn; }
 
 // Bounded mbarrier wait.  Returns false if the CTA is aborting (this wait or another one timed out).
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
@@ -224,8 +242,8 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
   int plain_toggle = 0;
   uint32_t buf_out = c.buf0 + 4096u;
 
-  auto tile_rows = [&](int tile) { return (tile % p.tiles_m) * (kBM * CG) + c.rank * kBM + q * 32; };
-  auto tile_cols = [&](int tile) { return (tile / p.tiles_m) * BN + half * kWarpCols; };
+  auto tile_rows = [&](int tile) { return tile_m(p, tile) * (kBM * CG) + c.rank * kBM + q * 32; };
+  auto tile_cols = [&](int tile) { return tile_n(p, tile) * BN + half * kWarpCols; };
   auto next_active_tile = [&](int tile) {
     while (tile < c.num_tiles && tile_cols(tile) >= p.N) tile += c.num_groups;
     return tile;
@@ -470,8 +488,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
       for (int tile = group; ok && tile < num_tiles; tile += num_groups) {
-        const int m0 = (tile % p.tiles_m) * (kBM * CG) + rank * kBM;
-        const int n0 = (tile / p.tiles_m) * BN + rank * kBRows;
+        const int m0 = tile_m(p, tile) * (kBM * CG) + rank * kBM;
+        const int n0 = tile_n(p, tile) * BN + rank * kBRows;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
           if (!ok) break;
@@ -580,8 +598,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     bool ok = true;
     for (int tile = group; ok && tile < num_tiles; tile += num_groups, ++local) {
       const uint32_t acc = local & 1u, acc_phase = (local >> 1) & 1u;
-      const int m0 = (tile % p.tiles_m) * (kBM * CG) + rank * kBM;
-      const int n0 = (tile / p.tiles_m) * BN;
+      const int m0 = tile_m(p, tile) * (kBM * CG) + rank * kBM;
+      const int n0 = tile_n(p, tile) * BN;
       const int64_t row = m0 + q * 32 + lane;
       const bool row_ok = row < p.M;
       EpiloguePrefetch pf;
