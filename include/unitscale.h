@@ -174,6 +174,23 @@ us_status us_residual_add(const us_mat* skip, const us_mat* branch, float tau, c
                           void* stream);
 us_status us_cast_fp8(const us_mat* src, float scale, const us_mat* dst, void* stream);
 
+/* ------------------------------------------------------------ scaled softmax
+ *
+ * Row-wise scaled softmax and its gradient (table "Table of unit scaling factors", row softmax:
+ * alpha = beta = s for rows of s elements; appendix paragraph "Softmax (followed by matmul)": the
+ * output is then about one everywhere, and the following matmul uses its ordinary factor).
+ *
+ *   us_softmax_fwd   P_ij  = alpha * exp(S_ij - max_j S_ij) / sum_j exp(S_ij - max_j S_ij)
+ *   us_softmax_bwd   dS_ij = beta * p_ij * (dP_ij - sum_k p_ik dP_ik),   p = P / alpha
+ *
+ * The backward pass takes the forward pass's scaled output P (as stored) and the gradient dP of
+ * that output.  All tensors of a call have the same rows x cols; inputs F32, BF16 or F16, outputs
+ * any us_dtype; any ld >= cols (rows that start 16-byte aligned, with cols a multiple of 8, take
+ * the 128-bit path).  alpha must be positive in us_softmax_bwd.
+ */
+us_status us_softmax_fwd(const us_mat* S, float alpha, const us_mat* P, void* stream);
+us_status us_softmax_bwd(const us_mat* P, const us_mat* dP, float alpha, float beta, const us_mat* dS, void* stream);
+
 /* ---------------------------------------------------------------- host helpers
  *
  * us_scales_linear: unit-scaling factors of matmul(X[b x m], W[m x n]).

@@ -89,6 +89,24 @@ def residual_add(skip, branch, tau):
     return weighted_add(skip, branch, ca, cb)
 
 
+# --------------------------------------------------------------------------- softmax
+
+def softmax_fwd(S, alpha):
+    """alpha * softmax over the last axis (table row "softmax": alpha = s for rows of s elements)."""
+    S = np.asarray(S, np.float64)
+    e = np.exp(S - S.max(axis=-1, keepdims=True))
+    return _f32(alpha) * e / e.sum(axis=-1, keepdims=True)
+
+
+def softmax_bwd(P, dP, alpha, beta):
+    """beta * softmax_grad: dS_j = beta * p_j (dP_j - sum_k p_k dP_k), p = P / alpha = softmax(S).
+
+    P is the forward pass's scaled output as stored; dP is the gradient with respect to it."""
+    p = np.asarray(P, np.float64) / _f32(alpha)
+    dP = np.asarray(dP, np.float64)
+    return _f32(beta) * p * (dP - np.sum(p * dP, axis=-1, keepdims=True))
+
+
 # --------------------------------------------------------------------------- storage rounding
 
 def store(v, dtype: str):

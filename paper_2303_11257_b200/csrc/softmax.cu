@@ -1,0 +1,238 @@
+// Scaled softmax over the rows of a matrix, forward and backward (table "Table of unit scaling
+// factors", row softmax: alpha = beta = s for rows of s elements; appendix paragraph "Softmax
+// (followed by matmul)").  One warp per row, 128-bit loads and stores, warp-shuffle reductions;
+// rows of up to 2048 elements are held in registers between the reduction and the write.
+#include "common.cuh"
+#include "host.h"
+
+namespace us {
+
+constexpr int kSmThreads = 256;            // 8 rows per CTA
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct SmArgs {
+  const void* in0; int in0_dt; int64_t in0_ld;      // S (forward) or P (backward)
+  const void* in1; int in1_dt; int64_t in1_ld;      // dP (backward only)
+  void* out; int out_dt; int64_t out_ld;
+  int64_t rows; int cols;
+  int vec_ok;                                       // all row starts 16-byte aligned and cols % 8 == 0
+  float alpha, beta;
+};
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Eight consecutive elements starting at column `col` of a row (fill beyond the row's end).
+__device__ __forceinline__ void load8(const void* base, int dt, int64_t row_off, int col, int cols, bool vec, float fill,
+                                      float (&v)[8]) {
+  if (vec) {
+    load_vec<8>(static_cast<const char*>(base) + (row_off + col) * dtype_size(dt), dt, v);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = (col + i < cols) ? load_one(base, dt, row_off + col + i) : fill;
+  }
+}
+__device__ __forceinline__ void store8(void* base, int dt, int64_t row_off, int col, int cols, bool vec, const float (&v)[8]) {
+  if (vec) {
+    char* p = static_cast<char*>(base) + (row_off + col) * dtype_size(dt);
+    if (dt == US_E4M3 || dt == US_E5M2) {
+      const uint32_t lo = dt == US_E5M2 ? cvt_fp8x4<true>(v[0], v[1], v[2], v[3]) : cvt_fp8x4<false>(v[0], v[1], v[2], v[3]);
+      const uint32_t hi = dt == US_E5M2 ? cvt_fp8x4<true>(v[4], v[5], v[6], v[7]) : cvt_fp8x4<false>(v[4], v[5], v[6], v[7]);
+      *reinterpret_cast<uint2*>(p) = make_uint2(lo, hi);
+    } else {
+      store_vec<8>(p, dt, v);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (col + i < cols) store_one(base, dt, row_off + col + i, v[i]);
+  }
+}
+
+// NCH > 0: the row fits in NCH chunks of 8 elements per lane, kept in registers.
+// NCH == 0: any length; the row is re-read from global memory (cache) in each pass.
+template <int NCH>
+__global__ void __launch_bounds__(kSmThreads) softmax_fwd_kernel(const SmArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (kSmThreads / 32) + (threadIdx.x >> 5);
+  if (row >= a.rows) return;
+  const int64_t in_off = row * a.in0_ld, out_off = row * a.out_ld;
+  const bool vec = a.vec_ok != 0;
+  const int nch = NCH > 0 ? NCH : (a.cols + 255) / 256;
+  float x[NCH > 0 ? NCH : 1][8];
+  float m = -INFINITY;
+  for (int c = 0; c < nch; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    float t[8];
+    if (col < a.cols) {
+      load8(a.in0, a.in0_dt, in_off, col, a.cols, vec, -INFINITY, t);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = -INFINITY;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { m = fmaxf(m, t[i]); if (NCH > 0) x[c][i] = t[i]; }
+  }
+  m = warp_max(m);
+  const float mb = m * kLog2e;
+  float sum = 0.f;
+  for (int c = 0; c < nch; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    float t[8];
+    if (NCH > 0) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = x[c][i];
+    } else if (col < a.cols) {
+      load8(a.in0, a.in0_dt, in_off, col, a.cols, vec, -INFINITY, t);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = -INFINITY;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float e = ex2_approx(fmaf(t[i], kLog2e, -mb));    // exp(x - max); exp(-inf) = 0 for the padding
+      sum += e;
+      if (NCH > 0) x[c][i] = e;
+    }
+  }
+  sum = warp_sum(sum);
+  const float inv = a.alpha / sum;
+  for (int c = 0; c < nch; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    if (col >= a.cols) continue;
+    float t[8];
+    if (NCH > 0) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = x[c][i] * inv;
+    } else {
+      load8(a.in0, a.in0_dt, in_off, col, a.cols, vec, -INFINITY, t);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = ex2_approx(fmaf(t[i], kLog2e, -mb)) * inv;
+    }
+    store8(a.out, a.out_dt, out_off, col, a.cols, vec, t);
+  }
+}
+
+template <int NCH>
+__global__ void __launch_bounds__(kSmThreads) softmax_bwd_kernel(const SmArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (kSmThreads / 32) + (threadIdx.x >> 5);
+  if (row >= a.rows) return;
+  const int64_t p_off = row * a.in0_ld, g_off = row * a.in1_ld, out_off = row * a.out_ld;
+  const bool vec = a.vec_ok != 0;
+  const int nch = NCH > 0 ? NCH : (a.cols + 255) / 256;
+  const float inv_alpha = 1.0f / a.alpha;
+  float pt[NCH > 0 ? NCH : 1][8], g[NCH > 0 ? NCH : 1][8];
+  float dot = 0.f;
+  for (int c = 0; c < nch; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    float tp[8], tg[8];
+    if (col < a.cols) {
+      load8(a.in0, a.in0_dt, p_off, col, a.cols, vec, 0.f, tp);
+      load8(a.in1, a.in1_dt, g_off, col, a.cols, vec, 0.f, tg);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { tp[i] = 0.f; tg[i] = 0.f; }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      tp[i] *= inv_alpha;                                   // softmax(S) recovered from the scaled output
+      dot = fmaf(tp[i], tg[i], dot);
+      if (NCH > 0) { pt[c][i] = tp[i]; g[c][i] = tg[i]; }
+    }
+  }
+  dot = warp_sum(dot);
+  for (int c = 0; c < nch; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    if (col >= a.cols) continue;
+    float tp[8], tg[8], t[8];
+    if (NCH > 0) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { tp[i] = pt[c][i]; tg[i] = g[c][i]; }
+    } else {
+      load8(a.in0, a.in0_dt, p_off, col, a.cols, vec, 0.f, tp);
+      load8(a.in1, a.in1_dt, g_off, col, a.cols, vec, 0.f, tg);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) tp[i] *= inv_alpha;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t[i] = a.beta * tp[i] * (tg[i] - dot);
+    store8(a.out, a.out_dt, out_off, col, a.cols, vec, t);
+  }
+}
+
+static bool rows_aligned(const us_mat* m) {
+  return reinterpret_cast<uintptr_t>(m->ptr) % 16 == 0 && (m->ld * dtype_size(m->dtype)) % 16 == 0;
+}
+
+template <bool BWD>
+static us_status launch_softmax(const SmArgs& a, cudaStream_t st) {
+  if (a.rows == 0 || a.cols == 0) return US_OK;
+  const int64_t grid64 = (a.rows + kSmThreads / 32 - 1) / (kSmThreads / 32);
+  if (grid64 > 0x7fffffff) return US_ERR_INVALID_ARG;
+  const int grid = (int)grid64;
+  const int nch = (a.cols + 255) / 256;
+#define US_SM_LAUNCH(N)                                                          \
+  do {                                                                           \
+    if (BWD) softmax_bwd_kernel<N><<<grid, kSmThreads, 0, st>>>(a);              \
+    else softmax_fwd_kernel<N><<<grid, kSmThreads, 0, st>>>(a);                  \
+  } while (0)
+  if (nch <= 1) US_SM_LAUNCH(1);
+  else if (nch <= 2) US_SM_LAUNCH(2);
+  else if (nch <= 4) US_SM_LAUNCH(4);
+  else if (nch <= 8 && !BWD) US_SM_LAUNCH(8);
+  else US_SM_LAUNCH(0);
+#undef US_SM_LAUNCH
+  return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
+}
+
+static us_status check_mat(const us_mat* m, const us_mat* like, bool input) {
+  if (!m || m->rows < 0 || m->cols < 0 || m->ld < m->cols) return US_ERR_INVALID_ARG;
+  if (like && (m->rows != like->rows || m->cols != like->cols)) return US_ERR_INVALID_ARG;
+  if (m->rows * m->cols > 0 && !m->ptr) return US_ERR_INVALID_ARG;
+  if (m->cols > 0x7ffffff0) return US_ERR_INVALID_ARG;
+  if (input ? !(m->dtype == US_F32 || m->dtype == US_BF16 || m->dtype == US_F16) : !(m->dtype >= US_F32 && m->dtype <= US_E5M2))
+    return US_ERR_UNSUPPORTED;
+  if (m->ptr && reinterpret_cast<uintptr_t>(m->ptr) % dtype_size(m->dtype)) return US_ERR_ALIGNMENT;
+  return US_OK;
+}
+
+}  // namespace us
+
+using namespace us;
+
+extern "C" us_status us_softmax_fwd(const us_mat* S, float alpha, const us_mat* P, void* stream) {
+  us_status s = check_mat(S, nullptr, true);
+  if (s == US_OK) s = check_mat(P, S, false);
+  if (s != US_OK) return s;
+  SmArgs a{};
+  a.in0 = S->ptr; a.in0_dt = S->dtype; a.in0_ld = S->ld;
+  a.out = P->ptr; a.out_dt = P->dtype; a.out_ld = P->ld;
+  a.rows = S->rows; a.cols = (int)S->cols; a.alpha = alpha; a.beta = 0.f;
+  a.vec_ok = rows_aligned(S) && rows_aligned(P) && S->cols % 8 == 0;
+  return launch_softmax<false>(a, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" us_status us_softmax_bwd(const us_mat* P, const us_mat* dP, float alpha, float beta, const us_mat* dS,
+                                    void* stream) {
+  us_status s = check_mat(P, nullptr, true);
+  if (s == US_OK) s = check_mat(dP, P, true);
+  if (s == US_OK) s = check_mat(dS, P, false);
+  if (s != US_OK) return s;
+  if (!(alpha > 0.f)) return US_ERR_INVALID_ARG;
+  SmArgs a{};
+  a.in0 = P->ptr; a.in0_dt = P->dtype; a.in0_ld = P->ld;
+  a.in1 = dP->ptr; a.in1_dt = dP->dtype; a.in1_ld = dP->ld;
+  a.out = dS->ptr; a.out_dt = dS->dtype; a.out_ld = dS->ld;
+  a.rows = P->rows; a.cols = (int)P->cols; a.alpha = alpha; a.beta = beta;
+  a.vec_ok = rows_aligned(P) && rows_aligned(dP) && rows_aligned(dS) && P->cols % 8 == 0;
+  return launch_softmax<true>(a, static_cast<cudaStream_t>(stream));
+}

@@ -68,7 +68,9 @@ def _load() -> C.CDLL:
     lib.us_gelu_bwd.argtypes = [MP, MP, F, F, MP, V]
     lib.us_residual_add.argtypes = [MP, MP, F, MP, V]
     lib.us_cast_fp8.argtypes = [MP, F, MP, V]
-    for name in ("us_gelu_fwd", "us_gelu_bwd", "us_residual_add", "us_cast_fp8"):
+    lib.us_softmax_fwd.argtypes = [MP, F, MP, V]
+    lib.us_softmax_bwd.argtypes = [MP, MP, F, F, MP, V]
+    for name in ("us_gelu_fwd", "us_gelu_bwd", "us_residual_add", "us_cast_fp8", "us_softmax_fwd", "us_softmax_bwd"):
         getattr(lib, name).restype = C.c_int
     FP = C.POINTER(C.c_float)
     lib.us_scales_linear.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_int, FP, FP, FP]
@@ -191,6 +193,16 @@ def us_residual_add(skip, branch, tau, out, stream=None):
 def us_cast_fp8(src, scale, dst, stream=None):
     _check("us_cast_fp8", _lib.us_cast_fp8(C.byref(mat(src)), scale, C.byref(mat(dst)), _stream(stream)))
     return dst
+
+
+def us_softmax_fwd(S, alpha, P, stream=None):
+    _check("us_softmax_fwd", _lib.us_softmax_fwd(C.byref(mat(S)), alpha, C.byref(mat(P)), _stream(stream)))
+    return P
+
+
+def us_softmax_bwd(P, dP, alpha, beta, dS, stream=None):
+    _check("us_softmax_bwd", _lib.us_softmax_bwd(C.byref(mat(P)), C.byref(mat(dP)), alpha, beta, C.byref(mat(dS)), _stream(stream)))
+    return dS
 
 
 def us_scales_linear(b: int, m: int, n: int, constrained: bool = False):
