@@ -114,6 +114,31 @@ us_status us_linear_bwd_x(const us_mat* G, const us_mat* W, float beta_x, const 
 us_status us_linear_bwd_w(const us_mat* X, const us_mat* G, float beta_w, const us_epilogue* ep,
                           const us_mat* dW, void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * Batched forms: count[0] x count[1] independent problems of one shape in a single launch, e.g. the
+ * (sequence, head) problems of scaled dot-product attention (appendix "Unit scaling and attention":
+ * alpha = beta_1 = beta_2 = 1 / sqrt(d) for the scores; the scaled softmax output then feeds an
+ * ordinary scaled matmul).  The us_mat arguments describe problem (0, 0); problem (i, j) of an
+ * operand starts stride[0] * i + stride[1] * j elements further.  Problems may be strided views of
+ * larger tensors (a head is a 64-column slice of a [tokens x 3 d] QKV matrix: ld = 3 d, inner
+ * stride 64, outer stride = sequence length * ld).  Every stride times the element size must be a
+ * multiple of 16 bytes (US_ERR_ALIGNMENT), strides of dimensions with count > 1 must be positive.
+ * No fused epilogue; otherwise dtypes, alignment, workspace and errors as for the single forms.
+ */
+typedef struct {
+  int64_t count[2];      /* number of problems in the outer / inner batch dimension (>= 1 each) */
+  int64_t a_stride[2];   /* first operand: elements between consecutive problems, outer / inner */
+  int64_t b_stride[2];   /* second operand */
+  int64_t out_stride[2]; /* output */
+} us_batch;
+
+us_status us_linear_fwd_batched(const us_mat* X, const us_mat* W, float alpha, const us_mat* Y, const us_batch* batch,
+                                void* ws, size_t ws_bytes, void* stream);
+us_status us_linear_bwd_x_batched(const us_mat* G, const us_mat* W, float beta_x, const us_mat* dX, const us_batch* batch,
+                                  void* ws, size_t ws_bytes, void* stream);
+us_status us_linear_bwd_w_batched(const us_mat* X, const us_mat* G, float beta_w, const us_mat* dW, const us_batch* batch,
+                                  void* ws, size_t ws_bytes, void* stream);
+
 /* Bytes of device workspace the linear ops need. */
 size_t us_workspace_bytes(void);
 

@@ -21,7 +21,7 @@ enum Op { kFwd, kBwdX, kBwdW };
 
 // A, B: the two operands in call order; out [M x N].
 static us_status linear(Op op, const us_mat* A, const us_mat* B, float scale, const us_epilogue* ep, const us_mat* out,
-                        void* ws, size_t ws_bytes, void* stream) {
+                        void* ws, size_t ws_bytes, void* stream, const us_batch* batch = nullptr) {
   if (!valid_mat(A) || !valid_mat(B) || !valid_mat(out)) return US_ERR_INVALID_ARG;
   int64_t M, N, K;
   bool shapes_ok;
@@ -71,6 +71,26 @@ static us_status linear(Op op, const us_mat* A, const us_mat* B, float scale, co
   else if (p.act == US_ACT_NONE) epi = kEpiSkip;
   else if (p.act == US_ACT_GELU && !p.skip) epi = kEpiGelu;
   else if (p.act == US_ACT_GELU_GRAD && !p.skip) epi = kEpiGeluGrad;
+  BatchDesc bd;
+  if (batch) {
+    if (ep) return US_ERR_UNSUPPORTED;                  // batched problems take no fused epilogue
+    const us_mat* ms[3] = {A, B, out};
+    const int64_t* strides[3] = {batch->a_stride, batch->b_stride, batch->out_stride};
+    int64_t* dst[3] = {bd.a, bd.b, bd.out};
+    if (batch->count[0] < 1 || batch->count[1] < 1 || batch->count[0] * batch->count[1] > (1 << 20)) return US_ERR_INVALID_ARG;
+    bd.nb0 = batch->count[0]; bd.nb1 = batch->count[1];
+    for (int i = 0; i < 3; ++i) {
+      const int es = dtype_size(ms[i]->dtype);
+      for (int d = 0; d < 2; ++d) {
+        int64_t st = strides[i][d];
+        if (batch->count[d] == 1) st = ms[i]->rows * ms[i]->ld;    // unused dimension: any valid pitch
+        if (st <= 0) return US_ERR_INVALID_ARG;
+        if ((st * es) % 16) return US_ERR_ALIGNMENT;
+        dst[i][d] = st;
+      }
+    }
+    if ((long long)((M + 127) / 128) * ((N + 127) / 128) * bd.nb0 * bd.nb1 > 0x7fffffffll) return US_ERR_INVALID_ARG;
+  }
   const bool a_mn = (op == kBwdW), b_mn = (op != kBwdX);
   const int a_fmt = f8 ? (A->dtype == US_E5M2) : (A->dtype == US_BF16);
   const int b_fmt = f8 ? (B->dtype == US_E5M2) : (B->dtype == US_BF16);
@@ -78,15 +98,15 @@ static us_status linear(Op op, const us_mat* A, const us_mat* B, float scale, co
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (f8) {
     switch (op) {
-      case kFwd:  return launch_gemm<1, false, true>(A, B, p, em, epi, st);
-      case kBwdX: return launch_gemm<1, false, false>(A, B, p, em, epi, st);
-      default:    return launch_gemm<1, true, true>(A, B, p, em, epi, st);
+      case kFwd:  return launch_gemm<1, false, true>(A, B, p, em, epi, bd, st);
+      case kBwdX: return launch_gemm<1, false, false>(A, B, p, em, epi, bd, st);
+      default:    return launch_gemm<1, true, true>(A, B, p, em, epi, bd, st);
     }
   }
   switch (op) {
-    case kFwd:  return launch_gemm<2, false, true>(A, B, p, em, epi, st);
-    case kBwdX: return launch_gemm<2, false, false>(A, B, p, em, epi, st);
-    default:    return launch_gemm<2, true, true>(A, B, p, em, epi, st);
+    case kFwd:  return launch_gemm<2, false, true>(A, B, p, em, epi, bd, st);
+    case kBwdX: return launch_gemm<2, false, false>(A, B, p, em, epi, bd, st);
+    default:    return launch_gemm<2, true, true>(A, B, p, em, epi, bd, st);
   }
 }
 
@@ -103,6 +123,22 @@ extern "C" us_status us_linear_bwd_x(const us_mat* G, const us_mat* W, float bet
 extern "C" us_status us_linear_bwd_w(const us_mat* X, const us_mat* G, float beta_w, const us_epilogue* ep,
                                      const us_mat* dW, void* ws, size_t ws_bytes, void* stream) {
   return us::linear(us::kBwdW, X, G, beta_w, ep, dW, ws, ws_bytes, stream);
+}
+
+extern "C" us_status us_linear_fwd_batched(const us_mat* X, const us_mat* W, float alpha, const us_mat* Y,
+                                           const us_batch* batch, void* ws, size_t ws_bytes, void* stream) {
+  if (!batch) return US_ERR_INVALID_ARG;
+  return us::linear(us::kFwd, X, W, alpha, nullptr, Y, ws, ws_bytes, stream, batch);
+}
+extern "C" us_status us_linear_bwd_x_batched(const us_mat* G, const us_mat* W, float beta_x, const us_mat* dX,
+                                             const us_batch* batch, void* ws, size_t ws_bytes, void* stream) {
+  if (!batch) return US_ERR_INVALID_ARG;
+  return us::linear(us::kBwdX, G, W, beta_x, nullptr, dX, ws, ws_bytes, stream, batch);
+}
+extern "C" us_status us_linear_bwd_w_batched(const us_mat* X, const us_mat* G, float beta_w, const us_mat* dW,
+                                             const us_batch* batch, void* ws, size_t ws_bytes, void* stream) {
+  if (!batch) return US_ERR_INVALID_ARG;
+  return us::linear(us::kBwdW, X, G, beta_w, nullptr, dW, ws, ws_bytes, stream, batch);
 }
 
 extern "C" size_t us_workspace_bytes(void) { return 256; }

@@ -33,6 +33,7 @@ struct GemmParams {
   int M, N, K;
   int tiles_m, tiles_n;
   int band_m;                               // tile rows per band of the tile order (see tile_mn)
+  int nb0, nb1;                             // batch counts (outer, inner); 1, 1 for a single problem
   float scale;
   uint32_t idesc;
   void* out; int out_dt; int64_t out_ld;
@@ -83,6 +84,7 @@ struct GemmSmem {
 // through once); when A is too large for that the host picks band_m = 8, so that a wave of ~74
 // tiles touches 8 row panels of A and ~9 column panels of B.
 __device__ __forceinline__ void tile_mn(const GemmParams& p, int tile, int& tm, int& tn) {
+  tile %= p.tiles_m * p.tiles_n;                     // position inside its problem of the batch
   const int band_tiles = p.band_m * p.tiles_n;
   const int band = tile / band_tiles;
   const int first_m = band * p.band_m;
@@ -93,6 +95,13 @@ __device__ __forceinline__ void tile_mn(const GemmParams& p, int tile, int& tm, 
 }
 __device__ __forceinline__ int tile_m(const GemmParams& p, int tile) { int tm, tn; tile_mn(p, tile, tm, tn); return tm; }
 __device__ __forceinline__ int tile_n(const GemmParams& p, int tile) { int tm, tn; tile_mn(p, tile, tm, tn); return tn; }
+// Batched problems: consecutive groups of tiles_m * tiles_n tiles belong to consecutive problems,
+// numbered outer * nb1 + inner.
+__device__ __forceinline__ void tile_batch(const GemmParams& p, int tile, int& b0, int& b1) {
+  const int b = tile / (p.tiles_m * p.tiles_n);
+  b0 = b / p.nb1;
+  b1 = b - b0 * p.nb1;
+}
 
 // Bounded mbarrier wait.  Returns false if the CTA is aborting (this wait or another one timed out).
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
@@ -217,7 +226,7 @@ struct EpiCtx {
 // pre-activation (GELU gradient) or the skip tensor, box stores for the output and for the
 // pre-activation the GELU epilogue keeps.  TMA clips stores and zero-fills loads at the matrix
 // edges, so ragged shapes need no special path.  No cross-warp synchronisation is involved.
-template <int BN, int CG, int EPI, int EW>
+template <int BN, int CG, int EPI, int EW, bool BATCHED>
 __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUtensorMap* tm_out, const CUtensorMap* tm_aux,
                                                 const CUtensorMap* tm_skip, const EpiCtx& c) {
   constexpr int kWarpCols = EW == 16 ? 64 : 128;            // columns of the tile one warp handles
@@ -251,7 +260,7 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
   auto issue_in = [&](int col, int row0) {
     if (lane == 0) {
       ptx::mbar_expect_tx(c.in_bar, 4096);
-      ptx::tma_load_2d(buf_in, tm_in, c.in_bar, col, row0);
+      ptx::tma_load_2d(buf_in, tm_in, c.in_bar, col, row0);      // fused inputs exist for single problems only
     }
   };
   if (in_kind) {
@@ -401,7 +410,11 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
         if (out_off + 32 == out_box_cols || last_slice) {
           ptx::fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) { ptx::tma_store_2d(tm_out, buf_out, col - out_off, row0); ptx::bulk_commit_group(); }
+          if (lane == 0) {
+            if (BATCHED) { int b0, b1; tile_batch(p, tile, b0, b1); ptx::tma_store_4d(tm_out, buf_out, col - out_off, row0, b1, b0); }
+            else ptx::tma_store_2d(tm_out, buf_out, col - out_off, row0);
+            ptx::bulk_commit_group();
+          }
         }
       }
     }
@@ -423,12 +436,13 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
 // EPI: the fused epilogue (EpiKind).  EW: number of epilogue warps (8 or 16).
 // CG: 1 = every CTA computes its own 128 x BN tiles; 2 = clusters of two CTAs compute 256 x BN
 //     tiles with tcgen05.mma.cta_group::2 (the even CTA issues, both load and both run an epilogue).
-template <int ES, bool A_MN, bool B_MN, int BN, int CG, int EPI, int EW>
+template <int ES, bool A_MN, bool B_MN, int BN, int CG, int EPI, int EW, bool BATCHED>
 __global__ void __launch_bounds__(gemm_threads(EW), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_aux,
             const __grid_constant__ CUtensorMap tmap_skip, const GemmParams p) {
   using S = GemmSmem<BN, CG, EW>;
+  static_assert(!BATCHED || EPI == kEpiPlain, "batched problems take the plain epilogue");
   static_assert(EW == 8 || (EW == 16 && (EPI == kEpiGelu || EPI == kEpiGeluGrad)), "16 epilogue warps serve the GELU epilogues only");
   constexpr int kBK = kStageKBytes / ES;            // K elements per stage
   constexpr int kChunkElems = 128 / ES;             // MN elements per 128-byte row of an MN-major tile
@@ -457,7 +471,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   const int lane = threadIdx.x & 31;
   const int rank = (CG == 2) ? (int)ptx::cluster_ctarank() : 0;     // position in the pair
   const int group = blockIdx.x / CG, num_groups = gridDim.x / CG;   // tile-walking unit: CTA or pair
-  const int num_tiles = p.tiles_m * p.tiles_n;                      // tiles of (128 * CG) x BN
+  const int num_tiles = p.tiles_m * p.tiles_n * p.nb0 * p.nb1;      // tiles of (128 * CG) x BN, all problems
   const int num_kb = (p.K + kBK - 1) / kBK;
 
   if (threadIdx.x == 0) {
@@ -490,6 +504,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       for (int tile = group; ok && tile < num_tiles; tile += num_groups) {
         const int m0 = tile_m(p, tile) * (kBM * CG) + rank * kBM;
         const int n0 = tile_n(p, tile) * BN + rank * kBRows;
+        int b0 = 0, b1 = 0;
+        if (BATCHED) tile_batch(p, tile, b0, b1);
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
           if (!ok) break;
@@ -500,7 +516,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           const uint32_t fb = (CG == 2) ? ptx::in_even_cta(full_bar(stage)) : full_bar(stage);
           if (rank == 0) ptx::mbar_expect_tx(full_bar(stage), CG * S::kStageBytes);
           auto load = [&](uint32_t dst, const void* tm, int x, int y) {
-            if (CG == 2) ptx::tma_load_2d_pair(dst, tm, fb, x, y); else ptx::tma_load_2d(dst, tm, fb, x, y);
+            if (BATCHED) {
+              if (CG == 2) ptx::tma_load_4d_pair(dst, tm, fb, x, y, b1, b0); else ptx::tma_load_4d(dst, tm, fb, x, y, b1, b0);
+            } else {
+              if (CG == 2) ptx::tma_load_2d_pair(dst, tm, fb, x, y); else ptx::tma_load_2d(dst, tm, fb, x, y);
+            }
           };
           if (A_MN) {
 #pragma unroll
@@ -589,7 +609,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     c.in_bar = epi_in_bar(warp - 2); c.buf0 = epi_base + (warp - 2) * epi_warp_bytes(EW);
     c.abort_flag = abort_flag; c.warp = warp; c.lane = lane; c.rank = rank;
     c.group = group; c.num_groups = num_groups; c.num_tiles = num_tiles;
-    epilogue_staged<BN, CG, EPI, EW>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
+    epilogue_staged<BN, CG, EPI, EW, BATCHED>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
   } else {
     // ------------------------------------------------------------ epilogue warps, direct global accesses
     const int q = warp & 3;                          // TMEM lane quarter this warp may read

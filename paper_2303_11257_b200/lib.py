@@ -36,6 +36,10 @@ class us_epilogue(C.Structure):
     ]
 
 
+class us_batch(C.Structure):
+    _fields_ = [("count", C.c_int64 * 2), ("a_stride", C.c_int64 * 2), ("b_stride", C.c_int64 * 2), ("out_stride", C.c_int64 * 2)]
+
+
 class UnitScaleError(RuntimeError):
     def __init__(self, fn: str, status: int):
         self.status = status
@@ -57,6 +61,10 @@ def _load() -> C.CDLL:
     for name in ("us_linear_fwd", "us_linear_bwd_x", "us_linear_bwd_w"):
         fn = getattr(lib, name)
         fn.argtypes = [MP, MP, F, EP, MP, V, SZ, V]
+        fn.restype = C.c_int
+    for name in ("us_linear_fwd_batched", "us_linear_bwd_x_batched", "us_linear_bwd_w_batched"):
+        fn = getattr(lib, name)
+        fn.argtypes = [MP, MP, F, MP, C.POINTER(us_batch), V, SZ, V]
         fn.restype = C.c_int
     lib.us_linear_fwd_static_ws.argtypes = [MP, MP, F, EP, MP, C.POINTER(C.c_void_p), V]
     lib.us_linear_fwd_static_ws.restype = C.c_int
@@ -156,6 +164,33 @@ def us_linear_bwd_x(G, W, beta_x, dX, ws, ep=None, stream=None):
 
 def us_linear_bwd_w(X, G, beta_w, dW, ws, ep=None, stream=None):
     return _linear("us_linear_bwd_w", X, G, beta_w, ep, dW, ws, stream)
+
+
+def batch(count, a_stride, b_stride, out_stride) -> us_batch:
+    """us_batch from (outer, inner) pairs of counts and element strides."""
+    b = us_batch()
+    for i in range(2):
+        b.count[i], b.a_stride[i], b.b_stride[i], b.out_stride[i] = count[i], a_stride[i], b_stride[i], out_stride[i]
+    return b
+
+
+def _linear_batched(name, a, b, scale, out, bt, ws, stream):
+    fn = getattr(_lib, name)
+    _check(name, fn(C.byref(mat(a)), C.byref(mat(b)), scale, C.byref(mat(out)), C.byref(bt),
+                    ws.data_ptr(), ws.numel() * ws.element_size(), _stream(stream)))
+    return out
+
+
+def us_linear_fwd_batched(X, W, alpha, Y, bt, ws, stream=None):
+    return _linear_batched("us_linear_fwd_batched", X, W, alpha, Y, bt, ws, stream)
+
+
+def us_linear_bwd_x_batched(G, W, beta_x, dX, bt, ws, stream=None):
+    return _linear_batched("us_linear_bwd_x_batched", G, W, beta_x, dX, bt, ws, stream)
+
+
+def us_linear_bwd_w_batched(X, G, beta_w, dW, bt, ws, stream=None):
+    return _linear_batched("us_linear_bwd_w_batched", X, G, beta_w, dW, bt, ws, stream)
 
 
 def us_linear_fwd_static_ws(X, W, alpha, Y, ep=None, stream=None) -> int:
