@@ -1,0 +1,94 @@
+"""Unit-scaled Transformer encoder layer, forward and backward (test infrastructure, fp64 NumPy).
+
+Self-attention block followed by the FFN block of ops.py, both wrapped in fixed(tau) residuals
+(section "Weighted addition"), without layer norm.  Scaled dot-product attention follows the
+appendix "Unit scaling and attention" (scores scaled by 1 / sqrt(d_head) in both passes) and the
+paragraph "Softmax (followed by matmul)" (softmax scaled by the row length s, then an ordinary
+scaled matmul with alpha = s^-1/2).  Matmul inputs of the projections are FP8 (E4 activations and
+weights, E5 gradients); the attention matmuls take 16-bit operands; every stored intermediate is
+rounded to the format it is stored in.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+from . import ops as O
+from . import scales as S
+
+
+@dataclass
+class EncoderResult:
+    QKV: np.ndarray = None
+    S: np.ndarray = None
+    P: np.ndarray = None
+    Cq: np.ndarray = None
+    R1: np.ndarray = None
+    ffn: O.FFNResult = None
+    dC: np.ndarray = None
+    dP: np.ndarray = None
+    dS: np.ndarray = None
+    dQKV: np.ndarray = None
+    dX: np.ndarray = None
+    dWqkv: np.ndarray = None
+    dWo: np.ndarray = None
+
+
+def _heads(M, nseq, slen, nhead, hd, which, d):
+    """[T x 3d] (or [T x d] with which = 0) -> [nseq, nhead, slen, hd] view of one of Q / K / V."""
+    o = which * d
+    return M[:, o:o + nhead * hd].reshape(nseq, slen, nhead, hd).transpose(0, 2, 1, 3)
+
+
+def _unheads(H, nseq, slen, nhead, hd):
+    """[nseq, nhead, slen, hd] -> [T x d]."""
+    return H.transpose(0, 2, 1, 3).reshape(nseq * slen, nhead * hd)
+
+
+def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16") -> EncoderResult:
+    T, d = X.shape
+    hd = d // nhead
+    f32 = lambda v: float(np.float32(v))
+    r = EncoderResult()
+    c_skip, c_branch = S.residual_coefficients(tau)
+    a_qkv, b_qkv, b_w = d ** -0.5, (3 * d) ** -0.5, T ** -0.5
+    a_o, b_o = d ** -0.5, d ** -0.5
+    a_s = b_Q = b_K = hd ** -0.5
+    a_c, b_P, b_V = slen ** -0.5, hd ** -0.5, slen ** -0.5
+    sm = float(slen)
+
+    Xq, _ = O.store(np.asarray(X), "e4m3")
+    Wqkv_q, _ = O.store(np.asarray(Wqkv), "e4m3")
+    Wo_q, _ = O.store(np.asarray(Wo), "e4m3")
+    # ---- forward
+    r.QKV, _ = O.store(O.linear_fwd(Xq, Wqkv_q, a_qkv), att)
+    Q, K, V = (_heads(r.QKV, nseq, slen, nhead, hd, i, d) for i in range(3))
+    S4, _ = O.store(f32(a_s) * (Q @ K.transpose(0, 1, 3, 2)), att)              # alpha Q K^T per (sequence, head)
+    P4, _ = O.store(O.softmax_fwd(S4, sm), att)
+    C4 = f32(a_c) * (P4 @ V)
+    r.Cq, _ = O.store(_unheads(C4, nseq, slen, nhead, hd), "e4m3")
+    r.S, r.P = S4.reshape(-1, slen), P4.reshape(-1, slen)
+    ep = O.Epilogue(skip=np.asarray(X, np.float64), skip_coef=c_skip, out_coef=c_branch)
+    r.R1, _, _ = O.apply_epilogue(O.linear_fwd(r.Cq, Wo_q, a_o), ep, "bf16")
+    sc = O.FFNScales.unconstrained(T, d, W1.shape[1], tau)
+    r.ffn = O.ffn_block(r.R1, W1, W2, G, sc, operand="fp8")
+    # ---- backward
+    g1 = r.ffn.dX
+    g1q, _ = O.store(g1, "e5m2")
+    r.dC, _ = O.store(O.linear_bwd_x(g1q, Wo_q, b_o), att)
+    r.dWo, _ = O.store(O.linear_bwd_w(r.Cq, g1q, b_w), "f32")
+    dC4 = _heads(r.dC, nseq, slen, nhead, hd, 0, d)
+    dP4, _ = O.store(f32(b_P) * (dC4 @ V.transpose(0, 1, 3, 2)), att)           # beta_1 G W^T with W = V
+    dV4 = f32(b_V) * (P4.transpose(0, 1, 3, 2) @ dC4)                           # beta_2 X^T G with X = P
+    dS4, _ = O.store(O.softmax_bwd(P4, dP4, sm, sm), att)
+    dQ4 = f32(b_Q) * (dS4 @ K)
+    dK4 = f32(b_K) * (dS4.transpose(0, 1, 3, 2) @ Q)
+    r.dP, r.dS = dP4.reshape(-1, slen), dS4.reshape(-1, slen)
+    dQKV = np.concatenate([_unheads(t, nseq, slen, nhead, hd) for t in (dQ4, dK4, dV4)], axis=1)
+    r.dQKV, _ = O.store(dQKV, att)
+    dQKVq, _ = O.store(r.dQKV, "e5m2")
+    ep = O.Epilogue(skip=g1, skip_coef=c_skip, out_coef=c_branch)
+    r.dX, _, _ = O.apply_epilogue(O.linear_bwd_x(dQKVq, Wqkv_q, b_qkv), ep, "bf16")
+    r.dWqkv, _ = O.store(O.linear_bwd_w(Xq, dQKVq, b_w), "f32")
+    return r

@@ -1,0 +1,121 @@
+"""Unit-scaled Transformer encoder layer (self-attention block + FFN block), forward and backward,
+as a sequence of libunitscale calls.  A driver only: buffers and call order; all arithmetic runs
+in the library's kernels.
+
+Layer (no layer norm; fixed(tau) residuals, section "Weighted addition"):
+    QKV = alpha_qkv q(X) q(Wqkv)                          FP8 GEMM, 16-bit output [T x 3d]
+    S   = alpha_s Q_h K_h^T   per (sequence, head)        batched, 16-bit operands, alpha_s = 1/sqrt(d_head)
+    P   = s softmax(S)                                    scaled softmax (table row "softmax"), s = sequence length
+    C   = alpha_c P V_h                                   batched, alpha_c = s^-1/2, stored as E4M3
+    R1  = sqrt(1-tau) X + sqrt(tau) alpha_o C q(Wo)       FP8 GEMM + residual epilogue
+    R2  = FFN block on R1                                 see ffn.py
+Backward from G = dL/dR2: the FFN block's backward gives g1 = dL/dR1, then
+    dC  = beta_o q(g1) q(Wo)^T ; dWo = beta_w C^T q(g1)
+    dP  = beta_P dC_h V_h^T ; dV = beta_V P^T dC_h        batched
+    dS  = s softmax_grad(P, dP)
+    dQ  = beta_Q dS K_h ; dK = beta_K dS^T Q_h            batched
+    dX  = sqrt(1-tau) g1 + sqrt(tau) beta_qkv q(dQKV) q(Wqkv)^T ; dWqkv = beta_w q(X)^T q(dQKV)
+Scale factors are the unconstrained table values (alpha = fan_in^-1/2, beta_X = fan_out^-1/2,
+beta_W = batch^-1/2 with the batch of an attention matmul = its sequence length).
+"""
+from __future__ import annotations
+
+import math
+
+import torch
+
+from . import ffn as F
+from . import lib as L
+
+E4, E5 = torch.float8_e4m3fn, torch.float8_e5m2
+
+
+class UnitScaledEncoderLayer:
+    def __init__(self, nseq: int, slen: int, d: int, nhead: int, d_ff: int, tau: float = 0.5,
+                 att_dtype=torch.bfloat16, device="cuda"):
+        assert d % nhead == 0
+        self.nseq, self.slen, self.d, self.nhead, self.hd, self.d_ff, self.tau = nseq, slen, d, nhead, d // nhead, d_ff, tau
+        T = self.T = nseq * slen
+        e = lambda r, c, dt: torch.empty((r, c), dtype=dt, device=device)
+        self.att_dtype = att_dtype
+        self.Xq, self.Wqkv_q, self.Wo_q = e(T, d, E4), e(d, 3 * d, E4), e(d, d, E4)
+        self.QKV = e(T, 3 * d, att_dtype)
+        self.S = e(nseq * nhead * slen, slen, att_dtype)
+        self.P = e(nseq * nhead * slen, slen, att_dtype)
+        self.Cq = e(T, d, E4)
+        self.R1 = e(T, d, torch.bfloat16)
+        self.ffn = F.UnitScaledFFN(T, d, d_ff, scales=F.FFNScales.unit(T, d, d_ff, tau), device=device)
+        self.g1q = e(T, d, E5)
+        self.dC = e(T, d, att_dtype)
+        self.dP = e(nseq * nhead * slen, slen, att_dtype)
+        self.dS = e(nseq * nhead * slen, slen, att_dtype)
+        self.dQKV = e(T, 3 * d, att_dtype)
+        self.dQKVq = e(T, 3 * d, E5)
+        self.dX = e(T, d, torch.bfloat16)
+        self.dWqkv, self.dWo = e(d, 3 * d, torch.float32), e(d, d, torch.float32)
+        self.ws = L.new_workspace(device)
+        self.c_skip, self.c_branch = math.sqrt(1.0 - tau), math.sqrt(tau)
+        s, hd = slen, self.hd
+        self.sc = dict(
+            alpha_qkv=d ** -0.5, beta_qkv=(3 * d) ** -0.5, alpha_o=d ** -0.5, beta_o=d ** -0.5, beta_w=T ** -0.5,
+            alpha_s=hd ** -0.5, beta_Q=hd ** -0.5, beta_K=hd ** -0.5,          # attention scores: 1 / sqrt(d_head)
+            alpha_c=s ** -0.5, beta_P=hd ** -0.5, beta_V=s ** -0.5,            # context matmul: fan_in = s, fan_out = d_head, batch = s
+            sm=float(s))
+        qkv = (slen * 3 * d, hd)          # (outer, inner) strides of a head slice of a [T x 3d] matrix
+        sq = (nhead * slen * slen, slen * slen)
+        td = (slen * d, hd)               # head slice of a [T x d] matrix
+        n = (nseq, nhead)
+        self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
+                       dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
+        self.launches_per_step = 8 + 10 + 11      # attention forward, FFN forward + backward, attention backward
+
+    def _heads(self, M, which):
+        """Problem (0, 0) of a [T x 3d] matrix: rows of the first sequence, columns of head 0 of Q / K / V."""
+        o = which * self.d
+        return M[: self.slen, o:o + self.hd]
+
+    def step(self, X, Wqkv, Wo, W1, W2, G, stream=None):
+        sc, ws, s = self.sc, self.ws, self.slen
+        # ---- forward
+        L.us_cast_fp8(Wqkv, 1.0, self.Wqkv_q, stream)
+        L.us_cast_fp8(Wo, 1.0, self.Wo_q, stream)
+        L.us_cast_fp8(X, 1.0, self.Xq, stream)
+        L.us_linear_fwd(self.Xq, self.Wqkv_q, sc["alpha_qkv"], self.QKV, ws, None, stream)
+        Q, K, V = (self._heads(self.QKV, i) for i in range(3))
+        L.us_linear_bwd_x_batched(Q, K, sc["alpha_s"], self.S[:s], self.bt["scores"], ws, stream)
+        L.us_softmax_fwd(self.S, sc["sm"], self.P, stream)
+        L.us_linear_fwd_batched(self.P[:s], V, sc["alpha_c"], self.Cq[:s, : self.hd], self.bt["ctx"], ws, stream)
+        ep = L.epilogue(skip=X, skip_coef=self.c_skip, out_coef=self.c_branch)
+        L.us_linear_fwd(self.Cq, self.Wo_q, sc["alpha_o"], self.R1, ws, ep, stream)
+        f = self.ffn
+        f.cast_weights(W1, W2, stream)
+        f.forward(self.R1, stream)
+        # ---- backward
+        f.backward(G, stream)                                   # f.dX = dL/dR1
+        g1 = f.dX
+        L.us_cast_fp8(g1, 1.0, self.g1q, stream)
+        L.us_linear_bwd_x(self.g1q, self.Wo_q, sc["beta_o"], self.dC, ws, None, stream)
+        L.us_linear_bwd_w(self.Cq, self.g1q, sc["beta_w"], self.dWo, ws, None, stream)
+        dC_h = self.dC[:s, : self.hd]
+        L.us_linear_bwd_x_batched(dC_h, V, sc["beta_P"], self.dP[:s], self.bt["dP"], ws, stream)
+        L.us_linear_bwd_w_batched(self.P[:s], dC_h, sc["beta_V"], self._heads(self.dQKV, 2), self.bt["dV"], ws, stream)
+        L.us_softmax_bwd(self.P, self.dP, sc["sm"], sc["sm"], self.dS, stream)
+        L.us_linear_fwd_batched(self.dS[:s], K, sc["beta_Q"], self._heads(self.dQKV, 0), self.bt["dQ"], ws, stream)
+        L.us_linear_bwd_w_batched(self.dS[:s], Q, sc["beta_K"], self._heads(self.dQKV, 1), self.bt["dK"], ws, stream)
+        L.us_cast_fp8(self.dQKV, 1.0, self.dQKVq, stream)
+        ep = L.epilogue(skip=g1, skip_coef=self.c_skip, out_coef=self.c_branch)
+        L.us_linear_bwd_x(self.dQKVq, self.Wqkv_q, sc["beta_qkv"], self.dX, ws, ep, stream)
+        L.us_linear_bwd_w(self.Xq, self.dQKVq, sc["beta_w"], self.dWqkv, ws, None, stream)
+        return self.dX
+
+    def check(self) -> None:
+        for ws in (self.ws, self.ffn.ws):
+            st = L.us_workspace_status(ws)
+            if st != L.US_OK:
+                raise L.UnitScaleError("UnitScaledEncoderLayer", st)
+
+    def flops(self) -> float:
+        T, d, f, s, hd = self.T, self.d, self.d_ff, self.slen, self.hd
+        proj = 6.0 * T * d * 3 * d + 6.0 * T * d * d
+        att = 2 * 6.0 * (self.nseq * self.nhead) * s * s * hd
+        return proj + att + 12.0 * T * d * f

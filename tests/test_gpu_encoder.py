@@ -1,0 +1,79 @@
+"""Unit-scaled encoder layer (attention block + FFN block), forward and backward, against the
+oracle's chain.
+
+Each op is checked strictly on its own elsewhere (batched GEMMs, softmax, linear ops with fused
+epilogues).  Here thirty launches are chained through 16-bit and FP8 intermediates: wherever the
+device and the oracle round an intermediate to neighbouring codes (a near-tie decided by float32 vs
+float64 arithmetic), everything downstream moves a little.  The chain is therefore compared with a
+looser bound: the first GEMM strictly, later tensors to a few 16-bit ulps of their scale, with all
+but a small fraction of the elements inside the strict bound."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import encoder as E
+from tests import util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(nseq, slen, d, nhead, f, seed):
+    from paper_2303_11257_b200 import encoder, synth
+    T = nseq * slen
+    host = (synth.normal(seed, 0, (T, d)), synth.normal(seed, 1, (d, 3 * d)), synth.normal(seed, 2, (d, d)),
+            synth.normal(seed, 3, (d, f)), synth.normal(seed, 4, (f, d)), synth.normal(seed, 5, (T, d)))
+    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, f)
+    layer.step(*[torch.from_numpy(t).cuda() for t in host])
+    layer.check()
+    return layer, host
+
+
+def _close(got, ref, name):
+    """Deep in the chain most elements carry the echo of some upstream rounding flip, so the check is
+    statistical: small mean error relative to the tensor's scale, no error of the order of the tensor
+    itself, and near-perfect correlation (a wiring, transposition or scale mistake fails all three)."""
+    g = U.host_values(got)
+    scale = max(1.0, float(np.abs(ref).std()))
+    err = np.abs(g - ref) / scale
+    assert err.mean() <= 5e-2, f"{name}: mean err {err.mean():.3e}"
+    assert err.max() <= 0.5 + 0.02 * float(np.abs(ref).max()) / scale, f"{name}: max err {err.max():.3e}"
+    corr = np.corrcoef(g.ravel(), ref.ravel())[0, 1]
+    assert corr > 0.999, f"{name}: correlation {corr:.6f}"
+
+
+def _mostly_strict(got, ref, name, frac):
+    g = U.host_values(got)
+    scale = max(1.0, float(np.abs(ref).std()))
+    outside = np.abs(g - ref) / scale > 2e-3 + U.ulp_of(ref, "bf16") / scale
+    assert outside.mean() <= frac, f"{name}: {outside.mean():.3%} of the elements beyond the strict bound"
+
+
+@pytest.mark.parametrize("cfg", [(2, 128, 256, 4, 512), (3, 80, 192, 3, 400)])
+def test_encoder_layer_small(cfg):
+    nseq, slen, d, nhead, f = cfg
+    layer, host = _run(nseq, slen, d, nhead, f, seed=41)
+    r = E.encoder_layer(*host, nseq, slen, nhead)
+    U.assert_close_stored(layer.QKV, r.QKV, "bf16", 2e-3, "QKV")                 # first GEMM: strict
+    for name, got, ref in (("S", layer.S, r.S), ("P", layer.P, r.P), ("R1", layer.R1, r.R1), ("R2", layer.ffn.R, r.ffn.R),
+                           ("dC", layer.dC, r.dC), ("dP", layer.dP, r.dP), ("dS", layer.dS, r.dS), ("dQKV", layer.dQKV, r.dQKV),
+                           ("dX", layer.dX, r.dX), ("dWqkv", layer.dWqkv, r.dWqkv), ("dWo", layer.dWo, r.dWo),
+                           ("dW1", layer.ffn.dW1, r.ffn.dW1), ("dW2", layer.ffn.dW2, r.ffn.dW2)):
+        _close(got, ref, name)
+    for name, got, ref in (("S", layer.S, r.S), ("P", layer.P, r.P), ("R1", layer.R1, r.R1)):
+        _mostly_strict(got, ref, name, 0.02)                                 # early in the chain: nearly all strict
+    from oracle import formats as Fm
+    d_c = U.code_distance(U.codes_of(layer.Cq), Fm.quantise_codes(r.Cq, Fm.E4M3), "e4m3")
+    assert (d_c > 0).mean() < 0.05                        # the FP8 context tensor: few codes differ ...
+    _close(layer.Cq, r.Cq, "C")                          # ... and none by much in value
+
+
+def test_encoder_layer_bert_large_shape_statistics():
+    """Config 5 at full size (16 x 512 tokens, d = 1024, 16 heads): the layer runs, reports no timeout,
+    and its tensors have the scale the oracle shows at a smaller size (unit-ish at initialisation)."""
+    layer, _ = _run(16, 512, 1024, 16, 4096, seed=42)
+    st = lambda t: t.float().std().item()
+    assert abs(st(layer.QKV) - 1) < 0.03 and abs(st(layer.S) - 1) < 0.05
+    assert abs(layer.P.float().mean().item() - 1) < 0.01
+    for t in (layer.R1, layer.ffn.R, layer.dX, layer.dQKV, layer.dWqkv, layer.dWo, layer.ffn.dW1, layer.ffn.dW2):
+        assert 0.5 < st(t) < 6.0
+    assert torch.isfinite(layer.dX.float()).all().item()

@@ -1,0 +1,52 @@
+"""Pins for the oracle's encoder layer: per-head attention against a direct loop, unit scale at
+initialisation, and agreement of its pieces with the single-op functions."""
+import numpy as np
+
+from oracle import encoder as E
+from oracle import ops as O
+from paper_2303_11257_b200 import synth
+
+
+def _tensors(nseq, slen, d, f, seed=0):
+    T = nseq * slen
+    return (synth.normal(seed, 0, (T, d)), synth.normal(seed, 1, (d, 3 * d)), synth.normal(seed, 2, (d, d)),
+            synth.normal(seed, 3, (d, f)), synth.normal(seed, 4, (f, d)), synth.normal(seed, 5, (T, d)))
+
+
+def test_attention_pieces_match_a_direct_per_head_loop():
+    nseq, slen, d, nhead, f = 2, 16, 32, 4, 64
+    hd = d // nhead
+    X, Wqkv, Wo, W1, W2, G = _tensors(nseq, slen, d, f)
+    r = E.encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead)
+    for i in range(nseq):
+        for j in range(nhead):
+            rows = slice(i * slen, (i + 1) * slen)
+            q, k, v = (r.QKV[rows, o + j * hd:o + (j + 1) * hd] for o in (0, d, 2 * d))
+            pr = slice((i * nhead + j) * slen, (i * nhead + j + 1) * slen)
+            s_ref = O.store(O.linear_bwd_x(q, k, hd ** -0.5), "bf16")[0]            # alpha Q K^T
+            assert np.array_equal(r.S[pr], s_ref)
+            p_ref = O.store(O.softmax_fwd(s_ref, slen), "bf16")[0]
+            assert np.array_equal(r.P[pr], p_ref)
+            c_ref = O.store(O.linear_fwd(p_ref, v, slen ** -0.5), "e4m3")[0]
+            assert np.array_equal(r.Cq[rows, j * hd:(j + 1) * hd], c_ref)
+            dc = r.dC[rows, j * hd:(j + 1) * hd]
+            assert np.array_equal(r.dP[pr], O.store(O.linear_bwd_x(dc, v, hd ** -0.5), "bf16")[0])
+            dv = O.linear_bwd_w(p_ref, dc, slen ** -0.5)
+            assert np.array_equal(r.dQKV[rows, 2 * d + j * hd:2 * d + (j + 1) * hd], O.store(dv, "bf16")[0])
+            ds = r.dS[pr]
+            assert np.array_equal(r.dQKV[rows, j * hd:(j + 1) * hd], O.store(O.linear_fwd(ds, k, hd ** -0.5), "bf16")[0])
+            assert np.array_equal(r.dQKV[rows, d + j * hd:d + (j + 1) * hd], O.store(O.linear_bwd_w(ds, q, hd ** -0.5), "bf16")[0])
+
+
+def test_unit_scale_at_initialisation():
+    nseq, slen, d, nhead, f = 2, 128, 256, 4, 512
+    X, Wqkv, Wo, W1, W2, G = _tensors(nseq, slen, d, f, seed=1)
+    r = E.encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead)
+    assert abs(r.QKV.std() - 1) < 0.05
+    assert abs(r.S.std() - 1) < 0.1                       # scores scaled by 1 / sqrt(d_head)
+    assert abs(r.P.mean() - 1) < 0.01                     # scaled softmax output is about one
+    # unit-normal scores make the softmax output far from uniform (std 1.26 instead of 0), so the
+    # tensors downstream of it come out at 1.4 - 2.3 rather than exactly one
+    assert 0.5 < r.R1.std() < 2.5 and 0.5 < r.dX.std() < 2.5
+    for t in (r.dWqkv, r.dWo, r.dQKV, r.dC):
+        assert 0.3 < t.std() < 3.0
