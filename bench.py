@@ -9,7 +9,8 @@ epilogues (10 kernel launches, replayed as one CUDA graph).  Prints ONE JSON lin
   value      matmul TFLOP/s (12 T d f FLOP per step) with all inputs resident in HBM,
              K steps timed with CUDA events after W warm-ups, max over ranks.
   e2e        same metric through the public call with host buffers: every step copies
-             X, W1, W2, G from pinned host memory and reads R, dX, dW1, dW2 back.
+             X, W1, W2, G from pinned host memory and reads R, dX, dW1, dW2 back (copies of
+             neighbouring steps overlap the compute on separate streams).
   roofline   the GEMM kernel: achieved FLOP/s per launch (timing events between the launches of
              the step graph, separate pass) against the measured tensor peak.
   cpu_baseline / --impl reference: the fp64 NumPy oracle on the host cores, on a bounded
@@ -371,15 +372,35 @@ def run_ours(args, rank: int, world: int, local: int):
     h2d = sum(t.numel() * t.element_size() for t in pinned[0])
     d2h = sum(t.numel() * t.element_size() for t in outs[0])
 
+    # Three streams pipeline the steps: while step i computes, step i+1's inputs are being copied
+    # in and step i-1's results are being read back (two buffer sets; events keep a set's copies
+    # and its graph replay in order).
+    cur = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in sets]      # inputs of the set are on the device
+    ev_done = [torch.cuda.Event() for _ in sets]    # the set's step has finished
+    ev_out = [torch.cuda.Event() for _ in sets]     # the set's results have been read back
+
     def e2e_step(i):
         s = i % 2
-        for dst, src in zip(sets[s], pinned[s]):
-            dst.copy_(src, non_blocking=True)
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(ev_done[s])             # the previous step on this set no longer reads its inputs
+            for dst, src in zip(sets[s], pinned[s]):
+                dst.copy_(src, non_blocking=True)
+            ev_in[s].record(s_in)
+        cur.wait_event(ev_in[s])
+        cur.wait_event(ev_out[s])                   # its previous results have been copied out
         graphs[s].replay()
-        for dst, src in zip(outs[s], (blocks[s].R, blocks[s].dX, blocks[s].dW1, blocks[s].dW2)):
-            dst.copy_(src, non_blocking=True)
+        ev_done[s].record(cur)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_done[s])
+            for dst, src in zip(outs[s], (blocks[s].R, blocks[s].dX, blocks[s].dW1, blocks[s].dW2)):
+                dst.copy_(src, non_blocking=True)
+            ev_out[s].record(s_out)
 
-    for i in range(3):
+    for ev in ev_done + ev_out:
+        ev.record(cur)
+    for i in range(4):
         e2e_step(i)
     torch.cuda.synchronize()
     barrier(world)
@@ -387,6 +408,7 @@ def run_ours(args, rank: int, world: int, local: int):
     e0.record()
     for i in range(n_e2e):
         e2e_step(i)
+    cur.wait_stream(s_out)
     e1.record()
     torch.cuda.synchronize()
     windows.append((w0, time.time()))
