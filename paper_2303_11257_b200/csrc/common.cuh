@@ -129,24 +129,36 @@ __device__ __forceinline__ void store_one(void* base, int dt, int64_t idx, float
 }
 
 // ---------------------------------------------------------------- scaled GELU
-// Lower normal tail q(a) = Phi(-a), a = |z|, as 2^R(a) with R a degree-6 polynomial fitted to
-// log2 Phi(-a) on [0, 7.5] (fit_normal_tail.py regenerates the coefficients): one ex2 and six FMAs,
-// |q error| <= 2.7e-7, |a q error| <= 1.5e-7 in float32.  Beyond 7.5 the tail is below 4e-14 and a
-// is clamped.  Phi(z) = z >= 0 ? 1 - q : q, and gelu(z) = z Phi(z) = max(z, 0) - |z| q(|z|).
+// Lower normal tail q(a) = Phi(-a), a = |z|, as 2^R(t) with t = min(a / 7.5, 1) and R a degree-6
+// polynomial fitted to log2 Phi(-7.5 t) on [0, 1] (fit_normal_tail.py regenerates the coefficients):
+// one saturating multiply, six FMAs and one ex2; |q error| <= 2.7e-7, |a q error| <= 1.5e-7 in
+// float32.  Beyond a = 7.5 the tail is below 4e-14 and t stays at 1.  Phi(z) = z >= 0 ? 1 - q : q,
+// and gelu(z) = z Phi(z) = max(z, 0) - |z| q(|z|).
+constexpr float kTailRange = 7.5f;
+constexpr float kTailC0 = -9.999993443e-01f, kTailC1 = -8.633527756e+00f, kTailC2 = -2.581697273e+01f,
+                kTailC3 = -2.242405128e+01f, kTailC4 = 2.505270767e+01f, kTailC5 = -1.710954857e+01f,
+                kTailC6 = 4.934150219e+00f;
+
 __device__ __forceinline__ float ex2_approx(float x) {
   float r;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
   return r;
 }
+// min(|x| k, 1) for k > 0 in one instruction of the FMA pipe (the clamp is the multiply's saturation).
+__device__ __forceinline__ float sat_mul_abs(float x, float k) {
+  float r;
+  asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(r) : "f"(fabsf(x)), "f"(k));
+  return r;
+}
 __device__ __forceinline__ float normal_tail(float z) {
-  const float a = fminf(fabsf(z), 7.5f);
-  float r = 2.772329208e-05f;
-  r = fmaf(r, a, -7.209949545e-04f);
-  r = fmaf(r, a, 7.917892188e-03f);
-  r = fmaf(r, a, -5.315330625e-02f);
-  r = fmaf(r, a, -4.589684010e-01f);
-  r = fmaf(r, a, -1.151137114e+00f);
-  r = fmaf(r, a, -9.999993443e-01f);
+  const float t = sat_mul_abs(z, 1.0f / kTailRange);
+  float r = kTailC6;
+  r = fmaf(r, t, kTailC5);
+  r = fmaf(r, t, kTailC4);
+  r = fmaf(r, t, kTailC3);
+  r = fmaf(r, t, kTailC2);
+  r = fmaf(r, t, kTailC1);
+  r = fmaf(r, t, kTailC0);
   return ex2_approx(r);
 }
 
@@ -193,33 +205,47 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
   return r;
 }
 
-// q(|z|) for two arguments (see normal_tail).
-__device__ __forceinline__ void normal_tail2(f32x2 z, float& q0, float& q1) {
-  float z0, z1;
-  unpack2(z, z0, z1);
-  const f32x2 a = pack2(fminf(fabsf(z0), 7.5f), fminf(fabsf(z1), 7.5f));
-  f32x2 r = splat2(2.772329208e-05f);
-  r = fma2(r, a, splat2(-7.209949545e-04f));
-  r = fma2(r, a, splat2(7.917892188e-03f));
-  r = fma2(r, a, splat2(-5.315330625e-02f));
-  r = fma2(r, a, splat2(-4.589684010e-01f));
-  r = fma2(r, a, splat2(-1.151137114e+00f));
-  r = fma2(r, a, splat2(-9.999993443e-01f));
+// q for two arguments given t = min(|z| / 7.5, 1) of each (see normal_tail).
+__device__ __forceinline__ void normal_tail2(float t0, float t1, float& q0, float& q1) {
+  const f32x2 t = pack2(t0, t1);
+  f32x2 r = splat2(kTailC6);
+  r = fma2(r, t, splat2(kTailC5));
+  r = fma2(r, t, splat2(kTailC4));
+  r = fma2(r, t, splat2(kTailC3));
+  r = fma2(r, t, splat2(kTailC2));
+  r = fma2(r, t, splat2(kTailC1));
+  r = fma2(r, t, splat2(kTailC0));
   float r0, r1;
   unpack2(r, r0, r1);
   q0 = ex2_approx(r0);
   q1 = ex2_approx(r1);
 }
 
-// gelu_scaled for two values: h holds the pre-activations, in2 / out2 the splatted scales.
-__device__ __forceinline__ void gelu_scaled2(f32x2 h, f32x2 in2, f32x2 out2, float& y0, float& y1) {
-  const f32x2 z = mul2(in2, h);
-  float q0, q1;
-  normal_tail2(z, q0, q1);
-  float oz0, oz1;
-  unpack2(mul2(out2, z), oz0, oz1);
-  y0 = fmaf(-fabsf(oz0), q0, fmaxf(oz0, 0.f));
-  y1 = fmaf(-fabsf(oz1), q1, fmaxf(oz1, 0.f));
+// out_scale * gelu(in_scale * x) for two values.  x holds the pre-activations, k = in_scale / 7.5,
+// oi = out_scale * in_scale.  The arithmetic is laid out for the instruction mix of the GEMM
+// epilogue: comparisons and min / max issue at half rate and do not overlap the packed FMAs there,
+// so the clamp is a saturating multiply and, with CANCEL, max(.) is replaced by
+//     gelu = h + |h| (1 - 2 q),  h = x / 2,
+// which for negative x subtracts nearly equal numbers: the absolute error stays below
+// 2^-24 |out_scale x|, harmless in front of a rounding to 8 or 16 bits but not for a float32 output,
+// which takes the form max(x, 0) - |x| q instead (CANCEL = false).
+template <bool CANCEL>
+__device__ __forceinline__ void gelu_scaled2(f32x2 x, float k, float oi, float& y0, float& y1) {
+  float x0, x1, q0, q1;
+  unpack2(x, x0, x1);
+  normal_tail2(sat_mul_abs(x0, k), sat_mul_abs(x1, k), q0, q1);
+  if (CANCEL) {
+    float h0, h1, w0, w1;
+    unpack2(mul2(splat2(0.5f * oi), x), h0, h1);
+    unpack2(fma2(pack2(q0, q1), splat2(-2.0f), splat2(1.0f)), w0, w1);
+    y0 = fmaf(fabsf(h0), w0, h0);
+    y1 = fmaf(fabsf(h1), w1, h1);
+  } else {
+    float o0, o1;
+    unpack2(mul2(splat2(oi), x), o0, o1);
+    y0 = fmaf(-fabsf(o0), q0, fmaxf(o0, 0.f));
+    y1 = fmaf(-fabsf(o1), q1, fmaxf(o1, 0.f));
+  }
 }
 
 // gelu_grad_scaled for two values: h = stored pre-activations, g = incoming gradients,
@@ -227,8 +253,8 @@ __device__ __forceinline__ void gelu_scaled2(f32x2 h, f32x2 in2, f32x2 out2, flo
 __device__ __forceinline__ f32x2 gelu_grad_scaled2(f32x2 h, f32x2 g, f32x2 in2, f32x2 os2) {
   const f32x2 z = mul2(in2, h);
   float q0, q1, z0, z1;
-  normal_tail2(z, q0, q1);
   unpack2(z, z0, z1);
+  normal_tail2(sat_mul_abs(z0, 1.0f / kTailRange), sat_mul_abs(z1, 1.0f / kTailRange), q0, q1);
   const f32x2 Phi = pack2(z0 >= 0.f ? 1.0f - q0 : q0, z1 >= 0.f ? 1.0f - q1 : q1);
   float e0, e1;
   unpack2(mul2(mul2(splat2(-0.72134752044448170f), z), z), e0, e1);

@@ -128,6 +128,12 @@ us_status launch_gemm(const us_mat* A, const us_mat* B, GemmParams& p, const Epi
   // A (M x K operand) is re-read by every column of tiles: keep the plain order while it fits well
   // inside the 126 MB L2, switch to bands of 8 tile rows beyond that.
   p.band_m = ((long long)p.M * p.K * ES <= (80ll << 20)) ? p.tiles_m : 8;
+  p.full_bands = p.tiles_m / p.band_m;
+  p.d_problem = make_fast_div(p.tiles_m * p.tiles_n);
+  p.d_band = make_fast_div(p.band_m * p.tiles_n);
+  p.d_rows = make_fast_div(p.band_m);
+  p.d_rows_last = make_fast_div(p.tiles_m % p.band_m ? p.tiles_m % p.band_m : 1);
+  p.d_nb1 = make_fast_div(p.nb1);
   p.idesc = (p.idesc & ~((0x3fu << 17) | (0x1fu << 24))) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)((kBM * cg) >> 4) << 24);
   return pair ? pick_epilogue<ES, A_MN, B_MN, 256, 2>(A, B, p, em, epi, bd, stream)
               : pick_epilogue<ES, A_MN, B_MN, 128, 1>(A, B, p, em, epi, bd, stream);

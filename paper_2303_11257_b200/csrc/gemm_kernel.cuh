@@ -29,11 +29,30 @@
 
 namespace us {
 
+// Division of a non-negative int below 2^31 by a divisor fixed at launch: one multiply-high, one
+// add and one shift instead of the ~30-instruction sequence of a hardware-less integer divide, which
+// every epilogue warp would otherwise run several times per tile.  mul = floor(2^32 (2^shift - d) / d) + 1,
+// shift = ceil(log2 d); floor(n / d) = (mulhi(n, mul) + n) >> shift.
+struct FastDiv {
+  uint32_t mul, shift;
+  __device__ __forceinline__ int div(int n) const { return (int)((__umulhi((uint32_t)n, mul) + (uint32_t)n) >> shift); }
+};
+inline FastDiv make_fast_div(int d) {
+  FastDiv f;
+  uint32_t l = 0;
+  while ((1ll << l) < d) ++l;
+  f.shift = l;
+  f.mul = (uint32_t)((((1ull << l) - (uint64_t)d) << 32) / (uint64_t)d + 1ull);
+  return f;
+}
+
 struct GemmParams {
   int M, N, K;
   int tiles_m, tiles_n;
   int band_m;                               // tile rows per band of the tile order (see tile_mn)
   int nb0, nb1;                             // batch counts (outer, inner); 1, 1 for a single problem
+  int full_bands;                           // bands that have band_m tile rows; a last, shorter one may follow
+  FastDiv d_problem, d_band, d_rows, d_rows_last, d_nb1;   // by tiles_m * tiles_n, band_m * tiles_n, band_m, tiles_m % band_m, nb1
   float scale;
   uint32_t idesc;
   void* out; int out_dt; int64_t out_ld;
@@ -84,26 +103,28 @@ struct GemmSmem {
 // through once); when A is too large for that the host picks band_m = 8, so that a wave of ~74
 // tiles touches 8 row panels of A and ~9 column panels of B.
 __device__ __forceinline__ void tile_mn(const GemmParams& p, int tile, int& tm, int& tn) {
-  tile %= p.tiles_m * p.tiles_n;                     // position inside its problem of the batch
-  const int band_tiles = p.band_m * p.tiles_n;
-  const int band = tile / band_tiles;
+  tile -= p.d_problem.div(tile) * (p.tiles_m * p.tiles_n);   // position inside its problem of the batch
+  const int band = p.d_band.div(tile);
   const int first_m = band * p.band_m;
-  const int rows = min(p.band_m, p.tiles_m - first_m);
-  const int r = tile - band * band_tiles;
-  tm = first_m + r % rows;
-  tn = r / rows;
+  const bool last = band >= p.full_bands;
+  const int rows = last ? p.tiles_m - first_m : p.band_m;
+  const int r = tile - band * (p.band_m * p.tiles_n);
+  tn = last ? p.d_rows_last.div(r) : p.d_rows.div(r);
+  tm = first_m + r - tn * rows;
 }
 __device__ __forceinline__ int tile_m(const GemmParams& p, int tile) { int tm, tn; tile_mn(p, tile, tm, tn); return tm; }
 __device__ __forceinline__ int tile_n(const GemmParams& p, int tile) { int tm, tn; tile_mn(p, tile, tm, tn); return tn; }
 // Batched problems: consecutive groups of tiles_m * tiles_n tiles belong to consecutive problems,
 // numbered outer * nb1 + inner.
 __device__ __forceinline__ void tile_batch(const GemmParams& p, int tile, int& b0, int& b1) {
-  const int b = tile / (p.tiles_m * p.tiles_n);
-  b0 = b / p.nb1;
+  const int b = p.d_problem.div(tile);
+  b0 = p.d_nb1.div(b);
   b1 = b - b0 * p.nb1;
 }
 
 // Bounded mbarrier wait.  Returns false if the CTA is aborting (this wait or another one timed out).
+// (Each attempt already suspends the thread in hardware for a while, so polling costs few issue
+// slots: pausing between attempts made no measurable difference.)
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                              unsigned int* status) {
   for (uint32_t it = 0; it < kWaitLimit; ++it) {
@@ -263,6 +284,16 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
       ptx::tma_load_2d(buf_in, tm_in, c.in_bar, col, row0);      // fused inputs exist for single problems only
     }
   };
+  // This warp is done reading accumulator a: its values are in registers, so the buffer is handed
+  // back to the MMA warp before the arithmetic and the stores of the last slice, not after them.
+  auto release_acc = [&](uint32_t a) {
+    ptx::tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) {
+      if (CG == 2) ptx::mbar_arrive_cluster(ptx::in_even_cta(c.acc_empty0 + 8u * a));
+      else ptx::mbar_arrive(c.acc_empty0 + 8u * a);
+    }
+  };
   if (in_kind) {
     const int t0 = next_active_tile(c.group);
     if (t0 < c.num_tiles) issue_in(tile_cols(t0), tile_rows(t0));
@@ -278,6 +309,7 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
     if (!ok) break;
     ptx::tc_fence_after_sync();
     const uint32_t t_row = c.tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + half * kWarpCols;
+    bool released = false;
     if (n_w < p.N) {
 #pragma unroll 1
       for (int sl = 0; sl < kWarpCols / 32; ++sl) {
@@ -288,7 +320,7 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
         //      the box can be refilled while the slice is being computed
         uint4 raw[8];
         if (in_kind) {
-          const int off = (32 * sl) % in_box_cols;
+          const int off = (32 * sl) & (in_box_cols - 1);       // box widths are powers of two
           if (off == 0) {
             ok = wait_bounded(c.in_bar, in_phase, c.abort_flag, p.status);
             ok = __all_sync(0xffffffffu, ok);
@@ -311,7 +343,7 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
           }
         }
         // ---- staging boxes that start with this slice must have been read by their last TMA store
-        const int aux_off = (32 * sl) % 64, out_off = (32 * sl) % out_box_cols;
+        const int aux_off = (32 * sl) & 63, out_off = (32 * sl) & (out_box_cols - 1);
         if (out_off == 0 || (aux_out && aux_off == 0)) {
           if (!in_kind && !aux_out) {                        // both boxes hold outputs, used alternately
             buf_out = c.buf0 + (plain_toggle ? 4096u : 0u);
@@ -324,7 +356,9 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
         }
         float v[32];
         ptx::tmem_ld_32x32(t_row + 32 * sl, v);
-        const f32x2 scale2 = splat2(p.scale), in2 = splat2(p.act_in), out2 = splat2(p.act_out);
+        if (last_slice) { release_acc(acc); released = true; }   // the MMA warp may refill it while this slice is worked on
+        const f32x2 scale2 = splat2(p.scale), in2 = splat2(p.act_in);
+        const float tail_k = fabsf(p.act_in) * (1.0f / kTailRange), act_oi = p.act_out * p.act_in;
         const f32x2 os2 = splat2(p.act_out * p.act_in), skip2 = splat2(p.skip_coef), oc2 = splat2(p.out_coef);
         const uint32_t aux_cb = (uint32_t)(aux_off * 2) >> 4, out_cb = (uint32_t)(out_off * out_es) >> 4;
         const uint32_t dst = buf_out + out_row_off;
@@ -349,7 +383,7 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
               ptx::sts128(buf_aux + row_off + (((aux_cb + g) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
             }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) gelu_scaled2(x[k], in2, out2, y[2 * k], y[2 * k + 1]);
+            for (int k = 0; k < 4; ++k) gelu_scaled2<kNarrowOut>(x[k], tail_k, act_oi, y[2 * k], y[2 * k + 1]);
           } else if (EPI == kEpiGeluGrad) {
             const uint32_t w[4] = {raw[g].x, raw[g].y, raw[g].z, raw[g].w};
 #pragma unroll
@@ -420,12 +454,7 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
     }
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) break;
-    ptx::tc_fence_before_sync();
-    __syncwarp();
-    if (lane == 0) {
-      if (CG == 2) ptx::mbar_arrive_cluster(ptx::in_even_cta(c.acc_empty0 + 8u * acc));
-      else ptx::mbar_arrive(c.acc_empty0 + 8u * acc);
-    }
+    if (!released) release_acc(acc);                           // tile without columns for this warp
   }
   if (lane == 0) ptx::bulk_wait_group_read<0>();             // stores have left shared memory before the CTA may exit
   __syncwarp();
