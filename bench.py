@@ -313,7 +313,7 @@ def run_ours(args, rank: int, world: int, local: int):
     ms_per_step = ms_total / args.steps
     value = aggregate_throughput(flops_step * args.steps, world, ms_total * 1e-3) / 1e12
 
-    # ---- per-launch timing pass: the same ten launches captured in one graph with a timing event
+    # ---- per-launch timing pass: the same launches captured in one graph with a timing event
     #      (event-record node) between consecutive launches, replayed after a warm-up
     blk, tensors = blocks[0], sets[0]
     stage_list = blk.stages(*tensors)
@@ -356,6 +356,7 @@ def run_ours(args, rank: int, world: int, local: int):
         "flops_per_launch": flops_launch, "us_per_launch": gemm_us,
     }
     cast_bytes = {"cast_W1": d * f * 5, "cast_W2": d * f * 5, "cast_X": T * d * 5, "cast_G": T * d * 5}
+    cast_bytes["cast_all"] = sum(cast_bytes.values())
     if args.operand != "fp8":
         cast_bytes = {k: v // 5 * 6 for k, v in cast_bytes.items()}
     kernels = []

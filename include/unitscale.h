@@ -189,8 +189,18 @@ us_status us_linear_fwd_static_ws(const us_mat* X, const us_mat* W, float alpha,
  *                  paragraph "Quantisation error"); the product is one float32
  *                  multiply.  NaN stays NaN.
  *
- * Inputs may be F32, BF16 or F16; outputs any us_dtype (us_cast_fp8: E4M3 or E5M2
- * only).  0 <= tau <= 1.
+ * us_cast_fp8_multi  count (1..8) casts dst[i] = q(scale[i] * src[i]) as ONE kernel launch: the
+ *                  same arithmetic as count calls of us_cast_fp8 (bit-identical results), for
+ *                  the casts that open a training step (weights, activations and the incoming
+ *                  gradient all go to FP8 before the first matmul needs them, figure "PyTorch
+ *                  examples": every matmul input is quantised), where four short launches cost
+ *                  more than the bytes they move.  src, scale, dst: host arrays of count
+ *                  elements.  Every tensor must be free of row padding (ld == cols) and start
+ *                  on a 16-byte boundary: US_ERR_UNSUPPORTED / US_ERR_ALIGNMENT otherwise, and
+ *                  nothing is launched.  Tensors must not overlap.
+ *
+ * Inputs may be F32, BF16 or F16; outputs any us_dtype (us_cast_fp8, us_cast_fp8_multi: E4M3
+ * or E5M2 only).  0 <= tau <= 1.
  */
 us_status us_gelu_fwd(const us_mat* H, float s_in, float alpha, const us_mat* A, void* stream);
 us_status us_gelu_bwd(const us_mat* H, const us_mat* dA, float s_in, float beta, const us_mat* dH,
@@ -198,6 +208,8 @@ us_status us_gelu_bwd(const us_mat* H, const us_mat* dA, float s_in, float beta,
 us_status us_residual_add(const us_mat* skip, const us_mat* branch, float tau, const us_mat* out,
                           void* stream);
 us_status us_cast_fp8(const us_mat* src, float scale, const us_mat* dst, void* stream);
+us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, const us_mat* dst,
+                            void* stream);
 
 /* ------------------------------------------------------------ scaled softmax
  *

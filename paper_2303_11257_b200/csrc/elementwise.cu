@@ -61,6 +61,42 @@ __global__ void __launch_bounds__(kThreads) ew_kernel(const EwArgs p) {
   }
 }
 
+// Several casts in one launch: the chunks of all tensors are numbered consecutively and a thread finds
+// the tensor of its chunk by scanning the (at most kMultiMax) cumulative counts.  Tensors are contiguous
+// and 16-byte aligned (checked on the host), so every chunk but a tensor's last takes the vector path.
+constexpr int kMultiMax = 8;
+struct MultiCastArgs {
+  const void* src[kMultiMax];
+  void* dst[kMultiMax];
+  int64_t elems[kMultiMax];
+  int64_t chunk_end[kMultiMax];   // cumulative chunk counts
+  float scale[kMultiMax];
+  int src_dt[kMultiMax], dst_dt[kMultiMax];
+  int count;
+};
+
+__global__ void __launch_bounds__(kThreads) multi_cast_kernel(const MultiCastArgs p) {
+  const int64_t total = p.chunk_end[p.count - 1];
+  for (int64_t c = blockIdx.x * (int64_t)kThreads + threadIdx.x; c < total; c += (int64_t)gridDim.x * kThreads) {
+    int t = 0;
+    while (c >= p.chunk_end[t]) ++t;
+    const int64_t e0 = (c - (t ? p.chunk_end[t - 1] : 0)) * kVec;
+    const int sdt = p.src_dt[t], ddt = p.dst_dt[t];
+    const char* src = static_cast<const char*>(p.src[t]) + e0 * dtype_size(sdt);
+    char* dst = static_cast<char*>(p.dst[t]) + e0;                       // FP8: one byte per element
+    const float sc = p.scale[t];
+    if (e0 + kVec <= p.elems[t]) {
+      float a[kVec];
+      load_vec<kVec>(src, sdt, a);
+#pragma unroll
+      for (int i = 0; i < kVec; ++i) a[i] *= sc;
+      store_vec<kVec>(dst, ddt, a);
+    } else {
+      for (int64_t i = 0; e0 + i < p.elems[t]; ++i) store_one(p.dst[t], ddt, e0 + i, sc * load_one(p.src[t], sdt, e0 + i));
+    }
+  }
+}
+
 static bool row_starts_aligned(const us_mat* m, bool contiguous) {
   const int es = dtype_size(m->dtype);
   if (reinterpret_cast<uintptr_t>(m->ptr) % 16) return false;
@@ -119,6 +155,36 @@ extern "C" us_status us_cast_fp8(const us_mat* src, float scale, const us_mat* d
   if (s != US_OK) return s;
   if (dst->dtype != US_E4M3 && dst->dtype != US_E5M2) return US_ERR_UNSUPPORTED;
   return ew_launch<kCast>(src, nullptr, dst, scale, 0.f, stream);
+}
+
+extern "C" us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, const us_mat* dst, void* stream) {
+  if (count < 1 || count > kMultiMax || !src || !scale || !dst) return US_ERR_INVALID_ARG;
+  MultiCastArgs p{};
+  int64_t chunks = 0;
+  int used = 0;
+  for (int i = 0; i < count; ++i) {
+    us_status s = check_ew(&src[i], nullptr, &dst[i]);
+    if (s != US_OK) return s;
+    if (dst[i].dtype != US_E4M3 && dst[i].dtype != US_E5M2) return US_ERR_UNSUPPORTED;
+    const int64_t n = src[i].rows * src[i].cols;
+    if (n == 0) continue;
+    const bool dense = (src[i].ld == src[i].cols && dst[i].ld == dst[i].cols) || src[i].rows == 1;
+    if (!dense) return US_ERR_UNSUPPORTED;                               // padded rows: use us_cast_fp8
+    if (reinterpret_cast<uintptr_t>(src[i].ptr) % 16 || reinterpret_cast<uintptr_t>(dst[i].ptr) % 16) return US_ERR_ALIGNMENT;
+    p.src[used] = src[i].ptr; p.dst[used] = dst[i].ptr; p.elems[used] = n; p.scale[used] = scale[i];
+    p.src_dt[used] = src[i].dtype; p.dst_dt[used] = dst[i].dtype;
+    chunks += (n + kVec - 1) / kVec;
+    p.chunk_end[used] = chunks;
+    ++used;
+  }
+  if (used == 0) return US_OK;
+  p.count = used;
+  const int sms = host::sm_count();
+  if (sms <= 0) return US_ERR_CUDA;
+  const int64_t want = (chunks + kThreads - 1) / kThreads;
+  const int64_t cap = (int64_t)sms * 8;
+  multi_cast_kernel<<<(int)(want < cap ? want : cap), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }
 
 extern "C" us_status us_gelu_fwd(const us_mat* H, float s_in, float alpha, const us_mat* A, void* stream) {

@@ -4,7 +4,8 @@ A driver only: it owns the device buffers and issues the C-ABI calls in order; e
 of the computation happens in the library's kernels.
 
 Forward (Figure "PyTorch examples", scaled FFN; section "Weighted addition"):
-    Xq = q(X); W1q = q(W1); W2q = q(W2)                                   us_cast_fp8
+    Xq = q(X); W1q = q(W1); W2q = q(W2)                                   us_cast_fp8 (step(): one us_cast_fp8_multi
+                                                                          launch for these three and Gq)
     H  = alpha1 Xq W1q ; A = q(alpha_g gelu(s_in H)), H kept in 16 bit    us_linear_fwd + GELU epilogue
     R  = sqrt(1-tau) X + sqrt(tau) alpha2 A W2q                           us_linear_fwd + residual epilogue
 Backward, G = dL/dR (the branch output receives G unscaled):
@@ -73,7 +74,10 @@ class UnitScaledFFN:
         self.ws = L.new_workspace(device)
         c_skip, c_branch = math.sqrt(1.0 - self.sc.tau), math.sqrt(self.sc.tau)
         self._c = (c_skip, c_branch)
-        self.launches_per_step = 10
+        # step() has all four tensors to quantise at hand when it starts, so in FP8 mode it casts them
+        # with one launch; forward() / backward() on their own cast what they are given.
+        self.fused_casts = operand == "fp8"
+        self.launches_per_step = 7 if self.fused_casts else 10
 
     def _cast(self, src, dst, stream):
         if dst.dtype in (torch.float8_e4m3fn, torch.float8_e5m2):
@@ -82,23 +86,31 @@ class UnitScaledFFN:
             # 16-bit operand mode: rounding fp32 -> bf16/fp16 is the residual kernel with tau = 0
             L.us_residual_add(src, src, 0.0, dst, stream)
 
-    def stages(self, X, W1, W2, G):
-        """The ten launches of one pass, in order, as (name, kind, callable(stream)) triples.
+    def stages(self, X, W1, W2, G, fused_casts: bool | None = None):
+        """The launches of one pass, in order, as (name, kind, callable(stream)) triples.
 
-        kind is "cast" or "gemm"; forward(), backward() and step() run exactly these."""
+        kind is "cast" or "gemm"; step() runs exactly these (seven with the casts fused into one
+        launch, ten otherwise); forward() and backward() run the unfused ones they need."""
         sc, (c_skip, c_branch) = self.sc, self._c
+        fused = self.fused_casts if fused_casts is None else fused_casts
         ep1 = L.epilogue(act=L.US_ACT_GELU, act_in_scale=sc.s_in, act_out_scale=sc.alpha_g, aux=self.H)
         ep2 = L.epilogue(skip=X, skip_coef=c_skip, out_coef=c_branch)
         ep3 = L.epilogue(act=L.US_ACT_GELU_GRAD, act_in_scale=sc.s_in, act_out_scale=sc.beta_g, aux=self.H)
         ep5 = L.epilogue(skip=G, skip_coef=c_skip, out_coef=c_branch)
         ws = self.ws
-        return [
-            ("cast_W1", "cast", lambda st=None: self._cast(W1, self.W1q, st)),
-            ("cast_W2", "cast", lambda st=None: self._cast(W2, self.W2q, st)),
-            ("cast_X", "cast", lambda st=None: self._cast(X, self.Xq, st)),
+        if fused:
+            casts = [("cast_all", "cast", lambda st=None: L.us_cast_fp8_multi(
+                [W1, W2, X, G], [1.0] * 4, [self.W1q, self.W2q, self.Xq, self.Gq], st))]
+            cast_g = []
+        else:
+            casts = [("cast_W1", "cast", lambda st=None: self._cast(W1, self.W1q, st)),
+                     ("cast_W2", "cast", lambda st=None: self._cast(W2, self.W2q, st)),
+                     ("cast_X", "cast", lambda st=None: self._cast(X, self.Xq, st))]
+            cast_g = [("cast_G", "cast", lambda st=None: self._cast(G, self.Gq, st))]
+        return casts + [
             ("fwd1_gelu", "gemm", lambda st=None: L.us_linear_fwd(self.Xq, self.W1q, sc.alpha1, self.Aq, ws, ep1, st)),
             ("fwd2_residual", "gemm", lambda st=None: L.us_linear_fwd(self.Aq, self.W2q, sc.alpha2, self.R, ws, ep2, st)),
-            ("cast_G", "cast", lambda st=None: self._cast(G, self.Gq, st)),
+        ] + cast_g + [
             ("bwd_x2_gelu_grad", "gemm", lambda st=None: L.us_linear_bwd_x(self.Gq, self.W2q, sc.beta_x2, self.dHq, ws, ep3, st)),
             ("bwd_w2", "gemm", lambda st=None: L.us_linear_bwd_w(self.Aq, self.Gq, sc.beta_w, self.dW2, ws, None, st)),
             ("bwd_x1_residual", "gemm", lambda st=None: L.us_linear_bwd_x(self.dHq, self.W1q, sc.beta_x1, self.dX, ws, ep5, st)),
@@ -110,17 +122,17 @@ class UnitScaledFFN:
         self._cast(W2, self.W2q, stream)
 
     def forward(self, X, stream=None):
-        for name, _, fn in self.stages(X, None, None, None)[2:5]:
+        for name, _, fn in self.stages(X, None, None, None, fused_casts=False)[2:5]:
             fn(stream)
         return self.R
 
     def backward(self, G, stream=None):
-        for name, _, fn in self.stages(None, None, None, G)[5:]:
+        for name, _, fn in self.stages(None, None, None, G, fused_casts=False)[5:]:
             fn(stream)
         return self.dX, self.dW1, self.dW2
 
     def step(self, X, W1, W2, G, stream=None):
-        """One pass of the whole path: weight casts, forward, backward (10 kernel launches)."""
+        """One pass of the whole path: casts, forward, backward (launches_per_step kernel launches)."""
         for name, _, fn in self.stages(X, W1, W2, G):
             fn(stream)
         return self.dX, self.dW1, self.dW2

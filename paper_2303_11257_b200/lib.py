@@ -76,9 +76,10 @@ def _load() -> C.CDLL:
     lib.us_gelu_bwd.argtypes = [MP, MP, F, F, MP, V]
     lib.us_residual_add.argtypes = [MP, MP, F, MP, V]
     lib.us_cast_fp8.argtypes = [MP, F, MP, V]
+    lib.us_cast_fp8_multi.argtypes = [C.c_int, MP, C.POINTER(C.c_float), MP, V]
     lib.us_softmax_fwd.argtypes = [MP, F, MP, V]
     lib.us_softmax_bwd.argtypes = [MP, MP, F, F, MP, V]
-    for name in ("us_gelu_fwd", "us_gelu_bwd", "us_residual_add", "us_cast_fp8", "us_softmax_fwd", "us_softmax_bwd"):
+    for name in ("us_gelu_fwd", "us_gelu_bwd", "us_residual_add", "us_cast_fp8", "us_cast_fp8_multi", "us_softmax_fwd", "us_softmax_bwd"):
         getattr(lib, name).restype = C.c_int
     FP = C.POINTER(C.c_float)
     lib.us_scales_linear.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_int, FP, FP, FP]
@@ -228,6 +229,16 @@ def us_residual_add(skip, branch, tau, out, stream=None):
 def us_cast_fp8(src, scale, dst, stream=None):
     _check("us_cast_fp8", _lib.us_cast_fp8(C.byref(mat(src)), scale, C.byref(mat(dst)), _stream(stream)))
     return dst
+
+
+def us_cast_fp8_multi(srcs, scales, dsts, stream=None):
+    """One launch for len(srcs) casts; scales: one float per tensor."""
+    n = len(srcs)
+    sm = (us_mat * n)(*[mat(t) for t in srcs])
+    dm = (us_mat * n)(*[mat(t) for t in dsts])
+    sc = (C.c_float * n)(*[float(x) for x in scales])
+    _check("us_cast_fp8_multi", _lib.us_cast_fp8_multi(n, sm, sc, dm, _stream(stream)))
+    return dsts
 
 
 def us_softmax_fwd(S, alpha, P, stream=None):

@@ -2,7 +2,7 @@
 
     python -m paper_2303_11257_b200.profile_case [--tokens 8192] [--passes 2] [--operand fp8]
 
-Each pass is the ten launches of UnitScaledFFN.step at d_model = 1024, d_ff = 4096.  At the default
+Each pass is the launches of UnitScaledFFN.step (one fused cast, six GEMMs) at d_model = 1024, d_ff = 4096.  At the default
 size the process holds well under 2 GB on the device and a pass lasts a fraction of a millisecond.
 """
 from __future__ import annotations

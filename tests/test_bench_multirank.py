@@ -1,6 +1,7 @@
 """The N > 1 plumbing of bench.py on CPU: two gloo ranks, barrier + max-over-ranks timing,
 whole-job aggregation under weak scaling, and the reference arm's rank-0-only rule."""
 import json
+import re
 import os
 import subprocess
 import sys
@@ -33,7 +34,7 @@ def test_two_gloo_ranks_reduce_time_and_aggregate(tmp_path):
          "--master-addr", "127.0.0.1", "--master-port", "29731", str(script)],
         capture_output=True, text=True, env=env, timeout=300)
     assert out.returncode == 0, out.stderr[-2000:]
-    rows = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    rows = [json.loads(m) for m in re.findall(r"\{[^{}]*\}", out.stdout)]   # ranks may interleave their lines
     assert sorted(r["rank"] for r in rows) == [0, 1]
     for r in rows:
         assert r["world"] == 2 and r["max"] == 2.0 and r["total"] == 10.0 * 2 / 2.0

@@ -81,3 +81,50 @@ def test_cast_empty_and_errors():
     with pytest.raises(L.UnitScaleError) as e:
         L.us_cast_fp8(torch.zeros((4, 8), device="cuda"), 1.0, U.empty(4, 9, "e4m3"))
     assert e.value.status == 1
+
+
+def test_cast_multi_matches_oracle_and_single_casts():
+    """Mixed source types, formats, scales and ragged sizes in one launch: codes equal the oracle's and
+    those of separate us_cast_fp8 calls; neighbours of each destination stay untouched."""
+    from paper_2303_11257_b200 import synth
+    L = _lib()
+    specs = [((64, 48), "f32", "e4m3", 1.0), ((1, 1), "f32", "e5m2", 0.5), ((300, 257), "bf16", "e5m2", 3.0),
+             ((37, 19), "fp16", "e4m3", 2.0 ** -3), ((0, 8), "f32", "e4m3", 1.0), ((1024, 1024), "f32", "e4m3", 1 / 3),
+             ((5, 16), "bf16", "e4m3", 1000.0), ((2, 7), "f32", "e5m2", 1.0)]
+    srcs, dsts, wants, singles, scales = [], [], [], [], []
+    for i, (shape, st, fmt, scale) in enumerate(specs):
+        x = synth.normal(21 + i, 0, shape, 4.0)
+        xs = F.quantise(x, F.FORMATS[st]).astype(np.float32) if st != "f32" else x
+        srcs.append(U.to_device(xs, st) if x.size else torch.zeros(shape, device="cuda"))
+        dsts.append(U.empty(shape[0], shape[1], fmt))
+        singles.append(U.empty(shape[0], shape[1], fmt))
+        wants.append(F.scaled_cast(xs, scale, F.FORMATS[fmt]))
+        scales.append(scale)
+    L.us_cast_fp8_multi(srcs, scales, dsts)
+    for src, scale, one in zip(srcs, scales, singles):
+        L.us_cast_fp8(src, scale, one)
+    for dst, one, want in zip(dsts, singles, wants):
+        assert np.array_equal(U.codes_of(dst), want)
+        assert np.array_equal(U.codes_of(dst), U.codes_of(one))
+
+
+def test_cast_multi_errors_launch_nothing():
+    L = _lib()
+    a, b = torch.ones((4, 16), device="cuda"), torch.ones((4, 16), device="cuda")
+    da, db = U.empty(4, 16, "e4m3"), U.empty(4, 16, "e4m3")
+    da.view(torch.uint8).zero_()
+    padded = U.empty(4, 16, "e4m3", 32)
+    with pytest.raises(L.UnitScaleError) as e:                       # row padding: not for the fused launch
+        L.us_cast_fp8_multi([a, b], [1.0, 1.0], [da, padded])
+    assert e.value.status == 2
+    with pytest.raises(L.UnitScaleError) as e:                       # shape mismatch
+        L.us_cast_fp8_multi([a, b], [1.0, 1.0], [da, U.empty(4, 8, "e4m3")])
+    assert e.value.status == 1
+    with pytest.raises(L.UnitScaleError) as e:                       # more tensors than one launch takes
+        L.us_cast_fp8_multi([a] * 9, [1.0] * 9, [da] * 9)
+    assert e.value.status == 1
+    with pytest.raises(L.UnitScaleError) as e:                       # misaligned start
+        L.us_cast_fp8_multi([a.view(-1)[1:33].view(2, 16)], [1.0], [U.empty(2, 16, "e4m3")])
+    assert e.value.status == 3
+    torch.cuda.synchronize()
+    assert not da.view(torch.uint8).any()                            # the valid first tensor was not written either
