@@ -75,24 +75,53 @@ struct MultiCastArgs {
   int count;
 };
 
+struct MultiChunk {
+  const char* src; char* dst; float scale; int sdt, ddt, t; int64_t e0; bool full;
+};
+__device__ __forceinline__ MultiChunk multi_locate(const MultiCastArgs& p, int64_t c) {
+  MultiChunk m;
+  int t = 0;
+  while (c >= p.chunk_end[t]) ++t;
+  m.t = t;
+  m.e0 = (c - (t ? p.chunk_end[t - 1] : 0)) * kVec;
+  m.sdt = p.src_dt[t]; m.ddt = p.dst_dt[t];
+  m.src = static_cast<const char*>(p.src[t]) + m.e0 * dtype_size(m.sdt);
+  m.dst = static_cast<char*>(p.dst[t]) + m.e0;                          // FP8: one byte per element
+  m.scale = p.scale[t];
+  m.full = m.e0 + kVec <= p.elems[t];
+  return m;
+}
+__device__ __forceinline__ void multi_tail(const MultiCastArgs& p, const MultiChunk& m) {
+  for (int64_t i = 0; m.e0 + i < p.elems[m.t]; ++i)
+    store_one(p.dst[m.t], m.ddt, m.e0 + i, m.scale * load_one(p.src[m.t], m.sdt, m.e0 + i));
+}
+
+// Two chunks per thread and iteration, both loaded before either is stored, to keep more loads in flight.
 __global__ void __launch_bounds__(kThreads) multi_cast_kernel(const MultiCastArgs p) {
   const int64_t total = p.chunk_end[p.count - 1];
-  for (int64_t c = blockIdx.x * (int64_t)kThreads + threadIdx.x; c < total; c += (int64_t)gridDim.x * kThreads) {
-    int t = 0;
-    while (c >= p.chunk_end[t]) ++t;
-    const int64_t e0 = (c - (t ? p.chunk_end[t - 1] : 0)) * kVec;
-    const int sdt = p.src_dt[t], ddt = p.dst_dt[t];
-    const char* src = static_cast<const char*>(p.src[t]) + e0 * dtype_size(sdt);
-    char* dst = static_cast<char*>(p.dst[t]) + e0;                       // FP8: one byte per element
-    const float sc = p.scale[t];
-    if (e0 + kVec <= p.elems[t]) {
-      float a[kVec];
-      load_vec<kVec>(src, sdt, a);
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  for (int64_t c = blockIdx.x * (int64_t)kThreads + threadIdx.x; c < total; c += 2 * stride) {
+    const MultiChunk m0 = multi_locate(p, c);
+    const bool two = c + stride < total;
+    const MultiChunk m1 = two ? multi_locate(p, c + stride) : m0;
+    float a[kVec], b[kVec];
+    if (m0.full) load_vec<kVec>(m0.src, m0.sdt, a);
+    if (two && m1.full) load_vec<kVec>(m1.src, m1.sdt, b);
+    if (m0.full) {
 #pragma unroll
-      for (int i = 0; i < kVec; ++i) a[i] *= sc;
-      store_vec<kVec>(dst, ddt, a);
+      for (int i = 0; i < kVec; ++i) a[i] *= m0.scale;
+      store_vec<kVec>(m0.dst, m0.ddt, a);
     } else {
-      for (int64_t i = 0; e0 + i < p.elems[t]; ++i) store_one(p.dst[t], ddt, e0 + i, sc * load_one(p.src[t], sdt, e0 + i));
+      multi_tail(p, m0);
+    }
+    if (two) {
+      if (m1.full) {
+#pragma unroll
+        for (int i = 0; i < kVec; ++i) b[i] *= m1.scale;
+        store_vec<kVec>(m1.dst, m1.ddt, b);
+      } else {
+        multi_tail(p, m1);
+      }
     }
   }
 }
