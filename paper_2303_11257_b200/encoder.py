@@ -67,7 +67,7 @@ class UnitScaledEncoderLayer:
         n = (nseq, nhead)
         self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
                        dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
-        self.launches_per_step = 8 + 10 + 11      # attention forward, FFN forward + backward, attention backward
+        self.launches_per_step = 1 + 5 + 7 + 11   # fused cast, attention forward, FFN forward + backward, attention backward
 
     def _heads(self, M, which):
         """Problem (0, 0) of a [T x 3d] matrix: rows of the first sequence, columns of head 0 of Q / K / V."""
@@ -77,9 +77,10 @@ class UnitScaledEncoderLayer:
     def step(self, X, Wqkv, Wo, W1, W2, G, stream=None):
         sc, ws, s = self.sc, self.ws, self.slen
         # ---- forward
-        L.us_cast_fp8(Wqkv, 1.0, self.Wqkv_q, stream)
-        L.us_cast_fp8(Wo, 1.0, self.Wo_q, stream)
-        L.us_cast_fp8(X, 1.0, self.Xq, stream)
+        f = self.ffn
+        # every tensor that is known when the step starts goes to FP8 in one launch
+        L.us_cast_fp8_multi([Wqkv, Wo, X, W1, W2, G], [1.0] * 6,
+                            [self.Wqkv_q, self.Wo_q, self.Xq, f.W1q, f.W2q, f.Gq], stream)
         L.us_linear_fwd(self.Xq, self.Wqkv_q, sc["alpha_qkv"], self.QKV, ws, None, stream)
         Q, K, V = (self._heads(self.QKV, i) for i in range(3))
         L.us_linear_bwd_x_batched(Q, K, sc["alpha_s"], self.S[:s], self.bt["scores"], ws, stream)
@@ -87,11 +88,9 @@ class UnitScaledEncoderLayer:
         L.us_linear_fwd_batched(self.P[:s], V, sc["alpha_c"], self.Cq[:s, : self.hd], self.bt["ctx"], ws, stream)
         ep = L.epilogue(skip=X, skip_coef=self.c_skip, out_coef=self.c_branch)
         L.us_linear_fwd(self.Cq, self.Wo_q, sc["alpha_o"], self.R1, ws, ep, stream)
-        f = self.ffn
-        f.cast_weights(W1, W2, stream)
         f.forward(self.R1, stream)
         # ---- backward
-        f.backward(G, stream)                                   # f.dX = dL/dR1
+        f.backward(G, stream, cast_g=False)                     # f.dX = dL/dR1
         g1 = f.dX
         L.us_cast_fp8(g1, 1.0, self.g1q, stream)
         L.us_linear_bwd_x(self.g1q, self.Wo_q, sc["beta_o"], self.dC, ws, None, stream)

@@ -126,8 +126,10 @@ class UnitScaledFFN:
             fn(stream)
         return self.R
 
-    def backward(self, G, stream=None):
-        for name, _, fn in self.stages(None, None, None, G, fused_casts=False)[5:]:
+    def backward(self, G, stream=None, cast_g: bool = True):
+        """Backward pass from G = dL/dR.  cast_g=False: self.Gq already holds q(G) (a caller that
+        quantised G together with other tensors in one us_cast_fp8_multi launch)."""
+        for name, _, fn in self.stages(None, None, None, G, fused_casts=False)[5 if cast_g else 6:]:
             fn(stream)
         return self.dX, self.dW1, self.dW2
 
