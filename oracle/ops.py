@@ -107,6 +107,46 @@ def softmax_bwd(P, dP, alpha, beta):
     return _f32(beta) * p * (dP - np.sum(p * dP, axis=-1, keepdims=True))
 
 
+# --------------------------------------------------------------------------- layer norm
+
+def layer_norm_fwd(X, w, c, eps=0.0):
+    """layer_norm(X, w, c)_ij = c_j + w_j (X_ij - mu_i) / sigma_i over the last axis, with
+    mu_i the row mean and sigma_i^2 = mean_j X_ij^2 - mu_i^2 (table row "layer_norm"; alpha = 1).
+
+    eps is added to sigma_i^2 (the table's formula has none: eps = 0 reproduces it)."""
+    X = np.asarray(X, np.float64)
+    mu = X.mean(axis=-1, keepdims=True)
+    var = (X * X).mean(axis=-1, keepdims=True) - mu * mu
+    xhat = (X - mu) / np.sqrt(var + eps)
+    return np.asarray(c, np.float64) + np.asarray(w, np.float64) * xhat
+
+
+def layer_norm_bwd(X, w, G, eps=0.0, beta_x=1.0, beta_wc=None):
+    """Gradients of layer_norm for an incoming G = dL/dY, scaled as the table row "layer_norm" says:
+    beta_x = 1 for the input, beta_w = beta_c = b^-1/2 for the b x n input's weight and bias
+    (appendix: weights are cut-edges, so they may take their own factors).
+
+        xhat = (X - mu) / sigma,  u = G * w
+        dX_ij = beta_x / sigma_i * (u_ij - mean_j u_ij - xhat_ij mean_j(u_ij xhat_ij))
+        dw_j  = beta_wc sum_i G_ij xhat_ij,   dc_j = beta_wc sum_i G_ij
+    Returns (dX, dw, dc)."""
+    X = np.asarray(X, np.float64)
+    G = np.asarray(G, np.float64)
+    w = np.asarray(w, np.float64)
+    b = X.shape[0]
+    if beta_wc is None:
+        beta_wc = _f32(b ** -0.5)
+    mu = X.mean(axis=-1, keepdims=True)
+    var = (X * X).mean(axis=-1, keepdims=True) - mu * mu
+    rstd = 1.0 / np.sqrt(var + eps)
+    xhat = (X - mu) * rstd
+    u = G * w
+    dX = _f32(beta_x) * rstd * (u - u.mean(axis=-1, keepdims=True) - xhat * (u * xhat).mean(axis=-1, keepdims=True))
+    dw = _f32(beta_wc) * (G * xhat).sum(axis=0)
+    dc = _f32(beta_wc) * G.sum(axis=0)
+    return dX, dw, dc
+
+
 # --------------------------------------------------------------------------- storage rounding
 
 def store(v, dtype: str):

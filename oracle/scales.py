@@ -102,3 +102,9 @@ def residual_coefficients(tau: float):
 def rescale_flop_ratio(b: int, m: int, n: int) -> float:
     """FLOP_rescaling / FLOP_matmul = (1/6)(1/b + 1/m + 1/n) (appendix "Computational overhead")."""
     return (b * n + n * m + b * m) / (6.0 * b * n * m)
+
+
+def layer_norm_scales(b: int):
+    """(alpha, beta_x, beta_w, beta_c) of layer_norm on a b x n input (table row "layer_norm"):
+    alpha = 1, beta_x = 1, beta_w = beta_c = b^-1/2."""
+    return 1.0, 1.0, b ** -0.5, b ** -0.5
