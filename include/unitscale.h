@@ -228,6 +228,34 @@ us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, co
 us_status us_softmax_fwd(const us_mat* S, float alpha, const us_mat* P, void* stream);
 us_status us_softmax_bwd(const us_mat* P, const us_mat* dP, float alpha, float beta, const us_mat* dS, void* stream);
 
+/* ------------------------------------------------------------ scaled layer norm
+ *
+ * layer_norm(X, w, c)_ij = c_j + w_j (X_ij - mu_i) / sigma_i over the rows of X [b x n], mu_i the row
+ * mean and sigma_i^2 = mean_j X_ij^2 - mu_i^2 (+ eps; the table's formula has no eps, pass 0 for it),
+ * with the factors of table "Table of unit scaling factors", row layer_norm: alpha = 1, beta_x = 1,
+ * beta_w = beta_c = b^-1/2 (appendix: the weight and bias are cut-edges and take their own factors).
+ *
+ * us_layer_norm_fwd   Y = c + w * xhat.
+ * us_layer_norm_bwd   dX_ij = beta_x / sigma_i * (u_ij - mean_j u_ij - xhat_ij * mean_j(u_ij xhat_ij)),
+ *                     u = G * w;  dw_j = beta_wc * sum_i G_ij xhat_ij;  dc_j = beta_wc * sum_i G_ij.
+ *                     xhat and sigma are recomputed from X (nothing is saved by the forward call).
+ *                     The column sums are formed without atomics, in a fixed order: the result does
+ *                     not depend on scheduling.  Two launches.
+ *
+ * X, G: F32 / BF16 / F16, any ld >= cols.  w, c: 1 x n vectors, F32 / BF16 / F16.  Y, dX: any
+ * us_dtype; dw, dc: 1 x n, F32 / BF16 / F16.  Arithmetic in float32; the variance is accumulated
+ * about the mean.  Backward: n <= 4096 (US_ERR_UNSUPPORTED beyond) and a device workspace of
+ * us_layer_norm_bwd_workspace_bytes(b, n) bytes, 16-byte aligned, owned by the caller, which must
+ * not be used by another call that may run at the same time (US_ERR_WORKSPACE if too small).
+ * The size depends on the current device's SM count.  eps >= 0.
+ */
+us_status us_layer_norm_fwd(const us_mat* X, const us_mat* w, const us_mat* c, float eps, const us_mat* Y,
+                            void* stream);
+size_t us_layer_norm_bwd_workspace_bytes(int64_t rows, int64_t cols);
+us_status us_layer_norm_bwd(const us_mat* X, const us_mat* w, const us_mat* G, float eps, float beta_x,
+                            float beta_wc, const us_mat* dX, const us_mat* dw, const us_mat* dc, void* ws,
+                            size_t ws_bytes, void* stream);
+
 /* ---------------------------------------------------------------- host helpers
  *
  * us_scales_linear: unit-scaling factors of matmul(X[b x m], W[m x n]).

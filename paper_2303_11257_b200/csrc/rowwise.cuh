@@ -1,0 +1,47 @@
+// Helpers of the row-wise kernels (softmax, layer norm): one warp per row, eight consecutive
+// elements per lane and step, warp-shuffle reductions.
+#pragma once
+
+#include "common.cuh"
+
+namespace us {
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Eight consecutive elements starting at column `col` of a row (fill beyond the row's end).
+__device__ __forceinline__ void load8(const void* base, int dt, int64_t row_off, int col, int cols, bool vec, float fill,
+                                      float (&v)[8]) {
+  if (vec) {
+    load_vec<8>(static_cast<const char*>(base) + (row_off + col) * dtype_size(dt), dt, v);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = (col + i < cols) ? load_one(base, dt, row_off + col + i) : fill;
+  }
+}
+__device__ __forceinline__ void store8(void* base, int dt, int64_t row_off, int col, int cols, bool vec, const float (&v)[8]) {
+  if (vec) {
+    char* p = static_cast<char*>(base) + (row_off + col) * dtype_size(dt);
+    if (dt == US_E4M3 || dt == US_E5M2) {
+      const uint32_t lo = dt == US_E5M2 ? cvt_fp8x4<true>(v[0], v[1], v[2], v[3]) : cvt_fp8x4<false>(v[0], v[1], v[2], v[3]);
+      const uint32_t hi = dt == US_E5M2 ? cvt_fp8x4<true>(v[4], v[5], v[6], v[7]) : cvt_fp8x4<false>(v[4], v[5], v[6], v[7]);
+      *reinterpret_cast<uint2*>(p) = make_uint2(lo, hi);
+    } else {
+      store_vec<8>(p, dt, v);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (col + i < cols) store_one(base, dt, row_off + col + i, v[i]);
+  }
+}
+
+}  // namespace us

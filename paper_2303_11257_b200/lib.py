@@ -79,6 +79,11 @@ def _load() -> C.CDLL:
     lib.us_cast_fp8_multi.argtypes = [C.c_int, MP, C.POINTER(C.c_float), MP, V]
     lib.us_softmax_fwd.argtypes = [MP, F, MP, V]
     lib.us_softmax_bwd.argtypes = [MP, MP, F, F, MP, V]
+    lib.us_layer_norm_fwd.argtypes = [MP, MP, MP, F, MP, V]
+    lib.us_layer_norm_bwd.argtypes = [MP, MP, MP, F, F, F, MP, MP, MP, V, SZ, V]
+    lib.us_layer_norm_fwd.restype = lib.us_layer_norm_bwd.restype = C.c_int
+    lib.us_layer_norm_bwd_workspace_bytes.argtypes = [C.c_int64, C.c_int64]
+    lib.us_layer_norm_bwd_workspace_bytes.restype = SZ
     for name in ("us_gelu_fwd", "us_gelu_bwd", "us_residual_add", "us_cast_fp8", "us_cast_fp8_multi", "us_softmax_fwd", "us_softmax_bwd"):
         getattr(lib, name).restype = C.c_int
     FP = C.POINTER(C.c_float)
@@ -249,6 +254,29 @@ def us_softmax_fwd(S, alpha, P, stream=None):
 def us_softmax_bwd(P, dP, alpha, beta, dS, stream=None):
     _check("us_softmax_bwd", _lib.us_softmax_bwd(C.byref(mat(P)), C.byref(mat(dP)), alpha, beta, C.byref(mat(dS)), _stream(stream)))
     return dS
+
+
+def _vec(t: torch.Tensor) -> us_mat:
+    """A 1-D parameter tensor as a 1 x n us_mat."""
+    return mat(t.view(1, -1))
+
+
+def us_layer_norm_fwd(X, w, c, eps, Y, stream=None):
+    _check("us_layer_norm_fwd", _lib.us_layer_norm_fwd(C.byref(mat(X)), C.byref(_vec(w)), C.byref(_vec(c)), eps,
+                                                       C.byref(mat(Y)), _stream(stream)))
+    return Y
+
+
+def us_layer_norm_bwd_workspace_bytes(rows: int, cols: int) -> int:
+    return int(_lib.us_layer_norm_bwd_workspace_bytes(rows, cols))
+
+
+def us_layer_norm_bwd(X, w, G, eps, beta_x, beta_wc, dX, dw, dc, ws, stream=None):
+    """ws: a uint8 CUDA tensor of at least us_layer_norm_bwd_workspace_bytes(rows, cols) bytes."""
+    _check("us_layer_norm_bwd", _lib.us_layer_norm_bwd(
+        C.byref(mat(X)), C.byref(_vec(w)), C.byref(mat(G)), eps, beta_x, beta_wc, C.byref(mat(dX)), C.byref(_vec(dw)),
+        C.byref(_vec(dc)), ws.data_ptr(), ws.numel() * ws.element_size(), _stream(stream)))
+    return dX, dw, dc
 
 
 def us_scales_linear(b: int, m: int, n: int, constrained: bool = False):

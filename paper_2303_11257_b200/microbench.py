@@ -1,4 +1,4 @@
-"""Secondary measurements: the unfused elementwise kernels and the scaled softmax against the HBM
+"""Secondary measurements: the unfused elementwise kernels, the scaled softmax and layer norm against the HBM
 roofline, and one encoder-layer step (config 5).  `python -m paper_2303_11257_b200.microbench`.
 
 Each kernel is timed with CUDA events over graph replays that rotate among buffer sets larger than
@@ -49,6 +49,15 @@ def elementwise(rows=8192, cols=4096, nsets=4):
          lambda: (torch.randn(rows * 8, 512, device=dev).to(torch.bfloat16), torch.empty(rows * 8, 512, device=dev, dtype=torch.bfloat16)), 4),
         ("us_softmax_bwd bf16,bf16->bf16 (rows of 512)", lambda a, b, o: L.us_softmax_bwd(a, b, 512.0, 512.0, o),
          lambda: tuple(torch.randn(rows * 8, 512, device=dev).abs().to(torch.bfloat16) for _ in range(2)) + (torch.empty(rows * 8, 512, device=dev, dtype=torch.bfloat16),), 6),
+        ("us_layer_norm_fwd bf16->bf16 (rows of 1024)", lambda a, w, c, o: L.us_layer_norm_fwd(a, w, c, 1e-5, o),
+         lambda: (torch.randn(rows * 4, 1024, device=dev).to(torch.bfloat16), torch.ones(1024, device=dev), torch.zeros(1024, device=dev),
+                  torch.empty(rows * 4, 1024, device=dev, dtype=torch.bfloat16)), 4),
+        ("us_layer_norm_bwd bf16,bf16->bf16 (rows of 1024, two launches)",
+         lambda a, w, g, o, dw, dc, ws: L.us_layer_norm_bwd(a, w, g, 1e-5, 1.0, (rows * 4) ** -0.5, o, dw, dc, ws),
+         lambda: (torch.randn(rows * 4, 1024, device=dev).to(torch.bfloat16), torch.ones(1024, device=dev),
+                  torch.randn(rows * 4, 1024, device=dev).to(torch.bfloat16), torch.empty(rows * 4, 1024, device=dev, dtype=torch.bfloat16),
+                  torch.empty(1024, device=dev), torch.empty(1024, device=dev),
+                  torch.empty(L.us_layer_norm_bwd_workspace_bytes(rows * 4, 1024), dtype=torch.uint8, device=dev)), 6),
     ]
     for name, fn, make, bytes_per_elt in cases:
         sets = [make() for _ in range(nsets)]
