@@ -221,8 +221,8 @@ us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, co
  *   us_softmax_bwd   dS_ij = beta * p_ij * (dP_ij - sum_k p_ik dP_ik),   p = P / alpha
  *
  * The backward pass takes the forward pass's scaled output P (as stored) and the gradient dP of
- * that output.  All tensors of a call have the same rows x cols; inputs F32, BF16 or F16, outputs
- * any us_dtype; any ld >= cols (rows that start 16-byte aligned, with cols a multiple of 8, take
+ * that output.  All tensors of a call have the same rows x cols; inputs F32, BF16 or F16 (P of
+ * us_softmax_bwd may also be E4M3 / E5M2: an output stored for an FP8 matmul), outputs any us_dtype; any ld >= cols (rows that start 16-byte aligned, with cols a multiple of 8, take
  * the 128-bit path).  alpha must be positive in us_softmax_bwd.
  */
 us_status us_softmax_fwd(const us_mat* S, float alpha, const us_mat* P, void* stream);

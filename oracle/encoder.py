@@ -5,8 +5,11 @@ Self-attention block followed by the FFN block of ops.py, both wrapped in fixed(
 appendix "Unit scaling and attention" (scores scaled by 1 / sqrt(d_head) in both passes) and the
 paragraph "Softmax (followed by matmul)" (softmax scaled by the row length s, then an ordinary
 scaled matmul with alpha = s^-1/2).  Matmul inputs of the projections are FP8 (E4 activations and
-weights, E5 gradients); the attention matmuls take 16-bit operands; every stored intermediate is
-rounded to the format it is stored in.
+weights, E5 gradients); the attention matmuls take 16-bit operands (att = "bf16" / "fp16") or, with
+att = "fp8", FP8 operands like every other matmul (section "Experiments": all matmul inputs are
+quantised): Q, K, V and the softmax output P as E4, the gradients dC, dS and dQ, dK, dV as E5, while
+the softmax input S and the gradient dP of its output, which feed no matmul, stay in BF16.  Every
+stored intermediate is rounded to the format it is stored in.
 """
 from __future__ import annotations
 
@@ -57,15 +60,17 @@ def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16"
     a_s = b_Q = b_K = hd ** -0.5
     a_c, b_P, b_V = slen ** -0.5, hd ** -0.5, slen ** -0.5
     sm = float(slen)
+    # storage formats of the attention tensors: matmul operands (activations, gradients) and the rest
+    f_act, f_grad, f_wide = ("e4m3", "e5m2", "bf16") if att == "fp8" else (att, att, att)
 
     Xq, _ = O.store(np.asarray(X), "e4m3")
     Wqkv_q, _ = O.store(np.asarray(Wqkv), "e4m3")
     Wo_q, _ = O.store(np.asarray(Wo), "e4m3")
     # ---- forward
-    r.QKV, _ = O.store(O.linear_fwd(Xq, Wqkv_q, a_qkv), att)
+    r.QKV, _ = O.store(O.linear_fwd(Xq, Wqkv_q, a_qkv), f_act)
     Q, K, V = (_heads(r.QKV, nseq, slen, nhead, hd, i, d) for i in range(3))
-    S4, _ = O.store(f32(a_s) * (Q @ K.transpose(0, 1, 3, 2)), att)              # alpha Q K^T per (sequence, head)
-    P4, _ = O.store(O.softmax_fwd(S4, sm), att)
+    S4, _ = O.store(f32(a_s) * (Q @ K.transpose(0, 1, 3, 2)), f_wide)              # alpha Q K^T per (sequence, head)
+    P4, _ = O.store(O.softmax_fwd(S4, sm), f_act)
     C4 = f32(a_c) * (P4 @ V)
     r.Cq, _ = O.store(_unheads(C4, nseq, slen, nhead, hd), "e4m3")
     r.S, r.P = S4.reshape(-1, slen), P4.reshape(-1, slen)
@@ -76,17 +81,17 @@ def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16"
     # ---- backward
     g1 = r.ffn.dX
     g1q, _ = O.store(g1, "e5m2")
-    r.dC, _ = O.store(O.linear_bwd_x(g1q, Wo_q, b_o), att)
+    r.dC, _ = O.store(O.linear_bwd_x(g1q, Wo_q, b_o), f_grad)
     r.dWo, _ = O.store(O.linear_bwd_w(r.Cq, g1q, b_w), "f32")
     dC4 = _heads(r.dC, nseq, slen, nhead, hd, 0, d)
-    dP4, _ = O.store(f32(b_P) * (dC4 @ V.transpose(0, 1, 3, 2)), att)           # beta_1 G W^T with W = V
+    dP4, _ = O.store(f32(b_P) * (dC4 @ V.transpose(0, 1, 3, 2)), f_wide)           # beta_1 G W^T with W = V
     dV4 = f32(b_V) * (P4.transpose(0, 1, 3, 2) @ dC4)                           # beta_2 X^T G with X = P
-    dS4, _ = O.store(O.softmax_bwd(P4, dP4, sm, sm), att)
+    dS4, _ = O.store(O.softmax_bwd(P4, dP4, sm, sm), f_grad)
     dQ4 = f32(b_Q) * (dS4 @ K)
     dK4 = f32(b_K) * (dS4.transpose(0, 1, 3, 2) @ Q)
     r.dP, r.dS = dP4.reshape(-1, slen), dS4.reshape(-1, slen)
     dQKV = np.concatenate([_unheads(t, nseq, slen, nhead, hd) for t in (dQ4, dK4, dV4)], axis=1)
-    r.dQKV, _ = O.store(dQKV, att)
+    r.dQKV, _ = O.store(dQKV, f_grad)
     dQKVq, _ = O.store(r.dQKV, "e5m2")
     ep = O.Epilogue(skip=g1, skip_coef=c_skip, out_coef=c_branch)
     r.dX, _, _ = O.apply_epilogue(O.linear_bwd_x(dQKVq, Wqkv_q, b_qkv), ep, "bf16")

@@ -52,6 +52,14 @@ __device__ __forceinline__ float2 unpack_f16x2(uint32_t u) {
   return __half22float2(*reinterpret_cast<__half2*>(&u));
 }
 
+// Two FP8 codes (low byte first) widened to float; exact.
+__device__ __forceinline__ float2 unpack_fp8x2(uint16_t u, bool e5) {
+  uint32_t h;
+  if (e5) asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(h) : "h"(u));
+  else asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h) : "h"(u));
+  return unpack_f16x2(h);
+}
+
 // ---------------------------------------------------------------- row fragments
 // Load N consecutive elements (N a multiple of 16 / element size) starting at a
 // 16-byte aligned address and widen them to float.
@@ -115,7 +123,8 @@ __device__ __forceinline__ void store_vec(void* p, int dt, const float (&v)[N]) 
 __device__ __forceinline__ float load_one(const void* base, int dt, int64_t idx) {
   if (dt == US_F32) return reinterpret_cast<const float*>(base)[idx];
   if (dt == US_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(base)[idx]);
-  return __half2float(reinterpret_cast<const __half*>(base)[idx]);
+  if (dt == US_F16) return __half2float(reinterpret_cast<const __half*>(base)[idx]);
+  return unpack_fp8x2(reinterpret_cast<const uint8_t*>(base)[idx], dt == US_E5M2).x;
 }
 
 __device__ __forceinline__ void store_one(void* base, int dt, int64_t idx, float v) {

@@ -20,7 +20,15 @@ __device__ __forceinline__ float warp_sum(float v) {
 // Eight consecutive elements starting at column `col` of a row (fill beyond the row's end).
 __device__ __forceinline__ void load8(const void* base, int dt, int64_t row_off, int col, int cols, bool vec, float fill,
                                       float (&v)[8]) {
-  if (vec) {
+  if (vec && (dt == US_E4M3 || dt == US_E5M2)) {
+    const uint2 r = __ldg(reinterpret_cast<const uint2*>(static_cast<const char*>(base) + row_off + col));
+    const uint32_t w[2] = {r.x, r.y};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = unpack_fp8x2((uint16_t)(w[j >> 1] >> (16 * (j & 1))), dt == US_E5M2);
+      v[2 * j] = f.x; v[2 * j + 1] = f.y;
+    }
+  } else if (vec) {
     load_vec<8>(static_cast<const char*>(base) + (row_off + col) * dtype_size(dt), dt, v);
   } else {
 #pragma unroll

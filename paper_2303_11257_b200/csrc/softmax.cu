@@ -157,12 +157,14 @@ static us_status launch_softmax(const SmArgs& a, cudaStream_t st) {
   return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }
 
-static us_status check_mat(const us_mat* m, const us_mat* like, bool input) {
+// input: a tensor the kernel reads (float formats; FP8 too where fp8_in says so).
+static us_status check_mat(const us_mat* m, const us_mat* like, bool input, bool fp8_in = false) {
   if (!m || m->rows < 0 || m->cols < 0 || m->ld < m->cols) return US_ERR_INVALID_ARG;
   if (like && (m->rows != like->rows || m->cols != like->cols)) return US_ERR_INVALID_ARG;
   if (m->rows * m->cols > 0 && !m->ptr) return US_ERR_INVALID_ARG;
   if (m->cols > 0x7ffffff0) return US_ERR_INVALID_ARG;
-  if (input ? !(m->dtype == US_F32 || m->dtype == US_BF16 || m->dtype == US_F16) : !(m->dtype >= US_F32 && m->dtype <= US_E5M2))
+  const bool is_fp8 = m->dtype == US_E4M3 || m->dtype == US_E5M2;
+  if (input ? !(m->dtype == US_F32 || m->dtype == US_BF16 || m->dtype == US_F16 || (fp8_in && is_fp8)) : !(m->dtype >= US_F32 && m->dtype <= US_E5M2))
     return US_ERR_UNSUPPORTED;
   if (m->ptr && reinterpret_cast<uintptr_t>(m->ptr) % dtype_size(m->dtype)) return US_ERR_ALIGNMENT;
   return US_OK;
@@ -186,7 +188,7 @@ extern "C" us_status us_softmax_fwd(const us_mat* S, float alpha, const us_mat* 
 
 extern "C" us_status us_softmax_bwd(const us_mat* P, const us_mat* dP, float alpha, float beta, const us_mat* dS,
                                     void* stream) {
-  us_status s = check_mat(P, nullptr, true);
+  us_status s = check_mat(P, nullptr, true, true);           // the stored forward output may be FP8
   if (s == US_OK) s = check_mat(dP, P, true);
   if (s == US_OK) s = check_mat(dS, P, false);
   if (s != US_OK) return s;

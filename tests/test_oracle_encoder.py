@@ -13,35 +13,44 @@ def _tensors(nseq, slen, d, f, seed=0):
             synth.normal(seed, 3, (d, f)), synth.normal(seed, 4, (f, d)), synth.normal(seed, 5, (T, d)))
 
 
-def test_attention_pieces_match_a_direct_per_head_loop():
+import pytest
+
+
+@pytest.mark.parametrize("att", ["bf16", "fp8"])
+def test_attention_pieces_match_a_direct_per_head_loop(att):
     nseq, slen, d, nhead, f = 2, 16, 32, 4, 64
     hd = d // nhead
     X, Wqkv, Wo, W1, W2, G = _tensors(nseq, slen, d, f)
-    r = E.encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead)
+    r = E.encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, att=att)
+    act, grad, wide = ("e4m3", "e5m2", "bf16") if att == "fp8" else ("bf16",) * 3
+    from oracle import formats as F
+    for t, fmt in ((r.QKV, act), (r.P, act), (r.dC, grad), (r.dS, grad), (r.dQKV, grad), (r.S, wide), (r.dP, wide)):
+        assert np.array_equal(F.quantise(t, F.FORMATS[fmt]), t)          # every stored tensor is on its format's grid
     for i in range(nseq):
         for j in range(nhead):
             rows = slice(i * slen, (i + 1) * slen)
             q, k, v = (r.QKV[rows, o + j * hd:o + (j + 1) * hd] for o in (0, d, 2 * d))
             pr = slice((i * nhead + j) * slen, (i * nhead + j + 1) * slen)
-            s_ref = O.store(O.linear_bwd_x(q, k, hd ** -0.5), "bf16")[0]            # alpha Q K^T
+            s_ref = O.store(O.linear_bwd_x(q, k, hd ** -0.5), wide)[0]            # alpha Q K^T
             assert np.array_equal(r.S[pr], s_ref)
-            p_ref = O.store(O.softmax_fwd(s_ref, slen), "bf16")[0]
+            p_ref = O.store(O.softmax_fwd(s_ref, slen), act)[0]
             assert np.array_equal(r.P[pr], p_ref)
             c_ref = O.store(O.linear_fwd(p_ref, v, slen ** -0.5), "e4m3")[0]
             assert np.array_equal(r.Cq[rows, j * hd:(j + 1) * hd], c_ref)
             dc = r.dC[rows, j * hd:(j + 1) * hd]
-            assert np.array_equal(r.dP[pr], O.store(O.linear_bwd_x(dc, v, hd ** -0.5), "bf16")[0])
+            assert np.array_equal(r.dP[pr], O.store(O.linear_bwd_x(dc, v, hd ** -0.5), wide)[0])
             dv = O.linear_bwd_w(p_ref, dc, slen ** -0.5)
-            assert np.array_equal(r.dQKV[rows, 2 * d + j * hd:2 * d + (j + 1) * hd], O.store(dv, "bf16")[0])
+            assert np.array_equal(r.dQKV[rows, 2 * d + j * hd:2 * d + (j + 1) * hd], O.store(dv, grad)[0])
             ds = r.dS[pr]
-            assert np.array_equal(r.dQKV[rows, j * hd:(j + 1) * hd], O.store(O.linear_fwd(ds, k, hd ** -0.5), "bf16")[0])
-            assert np.array_equal(r.dQKV[rows, d + j * hd:d + (j + 1) * hd], O.store(O.linear_bwd_w(ds, q, hd ** -0.5), "bf16")[0])
+            assert np.array_equal(r.dQKV[rows, j * hd:(j + 1) * hd], O.store(O.linear_fwd(ds, k, hd ** -0.5), grad)[0])
+            assert np.array_equal(r.dQKV[rows, d + j * hd:d + (j + 1) * hd], O.store(O.linear_bwd_w(ds, q, hd ** -0.5), grad)[0])
 
 
-def test_unit_scale_at_initialisation():
+@pytest.mark.parametrize("att", ["bf16", "fp8"])
+def test_unit_scale_at_initialisation(att):
     nseq, slen, d, nhead, f = 2, 128, 256, 4, 512
     X, Wqkv, Wo, W1, W2, G = _tensors(nseq, slen, d, f, seed=1)
-    r = E.encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead)
+    r = E.encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, att=att)
     assert abs(r.QKV.std() - 1) < 0.05
     assert abs(r.S.std() - 1) < 0.1                       # scores scaled by 1 / sqrt(d_head)
     assert abs(r.P.mean() - 1) < 0.01                     # scaled softmax output is about one
@@ -50,3 +59,18 @@ def test_unit_scale_at_initialisation():
     assert 0.5 < r.R1.std() < 2.5 and 0.5 < r.dX.std() < 2.5
     for t in (r.dWqkv, r.dWo, r.dQKV, r.dC):
         assert 0.3 < t.std() < 3.0
+
+
+def test_fp8_attention_stays_close_to_16_bit_attention():
+    """FP8 operands change every attention tensor by quantisation noise only (E5M2 gradients carry two
+    mantissa bits, so a few percent per rounding): no tensor of the layer moves by more than a fraction
+    of its scale on average, and the two runs stay almost perfectly correlated (a wiring or format mix-up
+    in either mode would break both)."""
+    nseq, slen, d, nhead, f = 2, 128, 256, 4, 512
+    t = _tensors(nseq, slen, d, f, seed=2)
+    a = E.encoder_layer(*t, nseq, slen, nhead, att="bf16")
+    b = E.encoder_layer(*t, nseq, slen, nhead, att="fp8")
+    for name in ("S", "P", "R1", "dC", "dP", "dS", "dQKV", "dX", "dWqkv", "dWo"):
+        x, y = getattr(a, name), getattr(b, name)
+        assert np.abs(x - y).mean() < 0.25 * max(1.0, np.abs(x).std()), name
+        assert np.corrcoef(x.ravel(), y.ravel())[0, 1] > 0.985, name
