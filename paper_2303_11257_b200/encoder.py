@@ -17,6 +17,12 @@ Backward from G = dL/dR2: the FFN block's backward gives g1 = dL/dR1, then
     dX  = sqrt(1-tau) g1 + sqrt(tau) beta_qkv q(dQKV) q(Wqkv)^T ; dWqkv = beta_w q(X)^T q(dQKV)
 Scale factors are the unconstrained table values (alpha = fan_in^-1/2, beta_X = fan_out^-1/2,
 beta_W = batch^-1/2 with the batch of an attention matmul = its sequence length).
+
+attention = "bf16" / "fp16": the attention matmuls take 16-bit operands.  attention = "fp8": they take
+FP8 operands like the projections (section "Experiments": all matmul inputs are quantised): the QKV
+GEMM writes Q, K, V as E4M3, the softmax writes P as E4M3, the gradients dC and dS are written as E5M2
+and the batched GEMMs write dQ, dK, dV straight into the E5M2 operand of the QKV backward GEMMs (one
+cast launch fewer); S and dP, which feed no matmul, stay in BF16.
 """
 from __future__ import annotations
 
@@ -32,25 +38,29 @@ E4, E5 = torch.float8_e4m3fn, torch.float8_e5m2
 
 class UnitScaledEncoderLayer:
     def __init__(self, nseq: int, slen: int, d: int, nhead: int, d_ff: int, tau: float = 0.5,
-                 att_dtype=torch.bfloat16, device="cuda"):
+                 attention: str = "bf16", device="cuda"):
         assert d % nhead == 0
+        self.attention = attention
+        if attention == "fp8":
+            act_dt, grad_dt, wide_dt = E4, E5, torch.bfloat16
+        else:
+            act_dt = grad_dt = wide_dt = {"bf16": torch.bfloat16, "fp16": torch.float16}[attention]
         self.nseq, self.slen, self.d, self.nhead, self.hd, self.d_ff, self.tau = nseq, slen, d, nhead, d // nhead, d_ff, tau
         T = self.T = nseq * slen
         e = lambda r, c, dt: torch.empty((r, c), dtype=dt, device=device)
-        self.att_dtype = att_dtype
         self.Xq, self.Wqkv_q, self.Wo_q = e(T, d, E4), e(d, 3 * d, E4), e(d, d, E4)
-        self.QKV = e(T, 3 * d, att_dtype)
-        self.S = e(nseq * nhead * slen, slen, att_dtype)
-        self.P = e(nseq * nhead * slen, slen, att_dtype)
+        self.QKV = e(T, 3 * d, act_dt)
+        self.S = e(nseq * nhead * slen, slen, wide_dt)
+        self.P = e(nseq * nhead * slen, slen, act_dt)
         self.Cq = e(T, d, E4)
         self.R1 = e(T, d, torch.bfloat16)
         self.ffn = F.UnitScaledFFN(T, d, d_ff, scales=F.FFNScales.unit(T, d, d_ff, tau), device=device)
         self.g1q = e(T, d, E5)
-        self.dC = e(T, d, att_dtype)
-        self.dP = e(nseq * nhead * slen, slen, att_dtype)
-        self.dS = e(nseq * nhead * slen, slen, att_dtype)
-        self.dQKV = e(T, 3 * d, att_dtype)
+        self.dC = e(T, d, grad_dt)
+        self.dP = e(nseq * nhead * slen, slen, wide_dt)
+        self.dS = e(nseq * nhead * slen, slen, grad_dt)
         self.dQKVq = e(T, 3 * d, E5)
+        self.dQKV = self.dQKVq if attention == "fp8" else e(T, 3 * d, grad_dt)   # FP8: written as E5M2 directly
         self.dX = e(T, d, torch.bfloat16)
         self.dWqkv, self.dWo = e(d, 3 * d, torch.float32), e(d, d, torch.float32)
         self.ws = L.new_workspace(device)
@@ -67,7 +77,8 @@ class UnitScaledEncoderLayer:
         n = (nseq, nhead)
         self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
                        dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
-        self.launches_per_step = 1 + 5 + 7 + 11   # fused cast, attention forward, FFN forward + backward, attention backward
+        # fused cast, attention forward, FFN forward + backward, attention backward (one cast fewer with FP8 attention)
+        self.launches_per_step = 1 + 5 + 7 + (10 if attention == "fp8" else 11)
 
     def _heads(self, M, which):
         """Problem (0, 0) of a [T x 3d] matrix: rows of the first sequence, columns of head 0 of Q / K / V."""
@@ -101,7 +112,8 @@ class UnitScaledEncoderLayer:
         L.us_softmax_bwd(self.P, self.dP, sc["sm"], sc["sm"], self.dS, stream)
         L.us_linear_fwd_batched(self.dS[:s], K, sc["beta_Q"], self._heads(self.dQKV, 0), self.bt["dQ"], ws, stream)
         L.us_linear_bwd_w_batched(self.dS[:s], Q, sc["beta_K"], self._heads(self.dQKV, 1), self.bt["dK"], ws, stream)
-        L.us_cast_fp8(self.dQKV, 1.0, self.dQKVq, stream)
+        if self.dQKV is not self.dQKVq:
+            L.us_cast_fp8(self.dQKV, 1.0, self.dQKVq, stream)
         ep = L.epilogue(skip=g1, skip_coef=self.c_skip, out_coef=self.c_branch)
         L.us_linear_bwd_x(self.dQKVq, self.Wqkv_q, sc["beta_qkv"], self.dX, ws, ep, stream)
         L.us_linear_bwd_w(self.Xq, self.dQKVq, sc["beta_w"], self.dWqkv, ws, None, stream)

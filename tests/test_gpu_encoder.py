@@ -17,12 +17,12 @@ from tests import util as U
 pytestmark = pytest.mark.gpu
 
 
-def _run(nseq, slen, d, nhead, f, seed):
+def _run(nseq, slen, d, nhead, f, seed, attention="bf16"):
     from paper_2303_11257_b200 import encoder, synth
     T = nseq * slen
     host = (synth.normal(seed, 0, (T, d)), synth.normal(seed, 1, (d, 3 * d)), synth.normal(seed, 2, (d, d)),
             synth.normal(seed, 3, (d, f)), synth.normal(seed, 4, (f, d)), synth.normal(seed, 5, (T, d)))
-    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, f)
+    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, f, attention=attention)
     layer.step(*[torch.from_numpy(t).cuda() for t in host])
     layer.check()
     return layer, host
@@ -77,3 +77,33 @@ def test_encoder_layer_bert_large_shape_statistics():
     for t in (layer.R1, layer.ffn.R, layer.dX, layer.dQKV, layer.dWqkv, layer.dWo, layer.ffn.dW1, layer.ffn.dW2):
         assert 0.5 < st(t) < 6.0
     assert torch.isfinite(layer.dX.float()).all().item()
+
+
+@pytest.mark.parametrize("cfg", [(2, 128, 256, 4, 512), (3, 80, 192, 3, 400)])
+def test_encoder_layer_fp8_attention(cfg):
+    """FP8 operands for the attention matmuls (Q, K, V, P as E4M3; dC, dS, dQ, dK, dV as E5M2).  The first
+    GEMM's FP8 output is within one code of the oracle's; the rest of the chain is compared statistically,
+    with wider bounds than the 16-bit mode because a one-code difference is 6 % (E4M3) or 12 % (E5M2) of a value."""
+    nseq, slen, d, nhead, f = cfg
+    layer, host = _run(nseq, slen, d, nhead, f, seed=43, attention="fp8")
+    r = E.encoder_layer(*host, nseq, slen, nhead, att="fp8")
+    U.assert_close_stored(layer.QKV, r.QKV, "e4m3", 2e-3, "QKV")
+    assert layer.dQKV is layer.dQKVq and layer.launches_per_step == 23
+
+    def close(got, ref, name, mean_tol):
+        g = U.host_values(got)
+        scale = max(1.0, float(np.abs(ref).std()))
+        err = np.abs(g - ref) / scale
+        assert err.mean() <= mean_tol, f"{name}: mean err {err.mean():.3e}"
+        assert np.corrcoef(g.ravel(), ref.ravel())[0, 1] > 0.995, name
+
+    for name, got, ref in (("S", layer.S, r.S), ("P", layer.P, r.P), ("C", layer.Cq, r.Cq), ("R1", layer.R1, r.R1)):
+        close(got, ref, name, 2e-2)
+    for name, got, ref in (("R2", layer.ffn.R, r.ffn.R), ("dC", layer.dC, r.dC), ("dP", layer.dP, r.dP), ("dS", layer.dS, r.dS),
+                           ("dQKV", layer.dQKV, r.dQKV), ("dX", layer.dX, r.dX), ("dWqkv", layer.dWqkv, r.dWqkv),
+                           ("dWo", layer.dWo, r.dWo), ("dW1", layer.ffn.dW1, r.ffn.dW1), ("dW2", layer.ffn.dW2, r.ffn.dW2)):
+        close(got, ref, name, 8e-2)
+    # where the chain has not yet diverged the FP8 tensors agree code for code almost everywhere
+    from oracle import formats as Fm
+    d_p = U.code_distance(U.codes_of(layer.P), Fm.quantise_codes(r.P, Fm.E4M3), "e4m3")
+    assert d_p.max() <= 2 and (d_p > 0).mean() < 0.08

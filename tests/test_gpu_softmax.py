@@ -45,6 +45,24 @@ def test_softmax_fwd_bwd(shape, ld, in_fmt, out_fmt):
     U.assert_close_stored(dS, refb, fmt_b, 3e-6 * scale * max(1.0, cols / 512), "softmax bwd")
 
 
+@pytest.mark.parametrize("shape,ld", [((5, 8), None), ((33, 512), None), ((130, 200), 208), ((7, 100), 112), ((4, 2056), None)])
+def test_softmax_bwd_from_an_fp8_stored_output(shape, ld):
+    """P as the E4M3 tensor an FP8 matmul consumes, dP in BF16, dS written as E5M2."""
+    L, synth = _mods()
+    rows, cols = shape
+    alpha = beta = float(cols)
+    p_host = O.softmax_fwd(synth.normal(23, 0, shape, 1.0).astype(np.float64), alpha).astype(np.float32)
+    g = synth.normal(23, 1, shape)
+    Pt, Gt = U.to_device(p_host, "e4m3", ld), U.to_device(g, "bf16", ld)
+    gv, pv = U.values_of(g, "bf16"), U.values_of(p_host, "e4m3")
+    refb = O.softmax_bwd(pv, gv, alpha, beta)
+    scale = np.abs(refb).max() + np.abs(gv).max()
+    for out_fmt in ("f32", "e5m2"):
+        dS = U.empty(rows, cols, out_fmt, ld)
+        L.us_softmax_bwd(Pt, Gt, alpha, beta, dS)
+        U.assert_close_stored(dS, refb, out_fmt, 3e-6 * scale * max(1.0, cols / 512), "softmax bwd from FP8 P")
+
+
 def test_attention_shape_statistics():
     """16 x 16 x 512 rows of 512 scores would be 67 M elements; a 1/16 sample keeps the test quick."""
     L, synth = _mods()
