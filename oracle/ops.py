@@ -71,6 +71,35 @@ def gelu_bwd(H, dA, s_in, beta_g):
     return _f32(beta_g) * _f32(s_in) * (_Phi(z) + z * _phi(z)) * np.asarray(dA, np.float64)
 
 
+# --------------------------------------------------------------------------- other activations
+
+def _act(fn: str):
+    """(f, f') of a table activation ("Activations": relu, gelu, tanh, sigmoid), float64."""
+    if fn == "relu":
+        return (lambda z: np.maximum(z, 0.0)), (lambda z: (z > 0) * 1.0)
+    if fn == "gelu":
+        return (lambda z: z * _Phi(z)), (lambda z: _Phi(z) + z * _phi(z))
+    if fn == "tanh":
+        return np.tanh, (lambda z: 1.0 - np.tanh(z) ** 2)
+    if fn == "sigmoid":
+        from scipy.special import expit                              # (1 + e^-z)^-1 without overflow
+        return expit, (lambda z: expit(z) * expit(-z))
+    raise ValueError(fn)
+
+
+def activation_fwd(fn, H, s_in, alpha):
+    """A = alpha * f(s_in * H) for a table activation f."""
+    f, _ = _act(fn)
+    return _f32(alpha) * f(_f32(s_in) * np.asarray(H, np.float64))
+
+
+def activation_bwd(fn, H, dA, s_in, beta):
+    """dH = beta * s_in * f'(s_in * H) * dA."""
+    _, df = _act(fn)
+    z = _f32(s_in) * np.asarray(H, np.float64)
+    return _f32(beta) * _f32(s_in) * df(z) * np.asarray(dA, np.float64)
+
+
 # --------------------------------------------------------------------------- residual
 
 def weighted_add(a, b, coef_a, coef_b):
