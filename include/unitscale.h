@@ -173,6 +173,9 @@ us_status us_workspace_status(const void* ws, void* stream);
 us_status us_linear_fwd_static_ws(const us_mat* X, const us_mat* W, float alpha, const us_epilogue* ep,
                                   const us_mat* Y, void** ws_out, void* stream);
 
+/* Activations of the table "Table of unit scaling factors", section Activations. */
+typedef enum { US_FN_GELU = 0, US_FN_RELU = 1, US_FN_TANH = 2, US_FN_SIGMOID = 3 } us_fn;
+
 /* ------------------------------------------------------------ elementwise ops
  *
  * Unfused forms of the ops between the GEMMs.  All tensors of a call have the
@@ -184,6 +187,10 @@ us_status us_linear_fwd_static_ws(const us_mat* X, const us_mat* W, float alpha,
  * us_residual_add  out = sqrt(1 - tau) * skip + sqrt(tau) * branch  (section "Weighted
  *                  addition", scheme fixed(tau)); serves the backward pass too: there
  *                  skip = incoming gradient, branch = gradient at the branch entry.
+ * us_activation_fwd  A  = alpha * f(s_in * H) for f = relu(x) = max(x, 0), tanh, sigmoid(x) = (1 + e^-x)^-1
+ *                  or gelu (table rows relu / gelu / tanh / sigmoid: alpha = 1 / std f(Z), Z ~ N(0,1));
+ * us_activation_bwd  dH = beta * s_in * f'(s_in * H) * dA (beta = 1 / rms f'(Z)); relu'(0) = 0.
+ *                  US_FN_GELU gives the same values as us_gelu_fwd / us_gelu_bwd.
  * us_cast_fp8      dst = q(scale * src), q = nearest value of the FP8 format, ties to
  *                  even, saturating (section "Floating-point formats for deep learning",
  *                  paragraph "Quantisation error"); the product is one float32
@@ -205,6 +212,9 @@ us_status us_linear_fwd_static_ws(const us_mat* X, const us_mat* W, float alpha,
 us_status us_gelu_fwd(const us_mat* H, float s_in, float alpha, const us_mat* A, void* stream);
 us_status us_gelu_bwd(const us_mat* H, const us_mat* dA, float s_in, float beta, const us_mat* dH,
                       void* stream);
+us_status us_activation_fwd(us_fn fn, const us_mat* H, float s_in, float alpha, const us_mat* A, void* stream);
+us_status us_activation_bwd(us_fn fn, const us_mat* H, const us_mat* dA, float s_in, float beta,
+                            const us_mat* dH, void* stream);
 us_status us_residual_add(const us_mat* skip, const us_mat* branch, float tau, const us_mat* out,
                           void* stream);
 us_status us_cast_fp8(const us_mat* src, float scale, const us_mat* dst, void* stream);
@@ -263,11 +273,14 @@ us_status us_layer_norm_bwd(const us_mat* X, const us_mat* w, const us_mat* G, f
  *   constrained != 0: alpha = beta_x = (m n)^-1/4 (geometric mean, section "Example").
  * us_scales_gelu: 1/std of gelu(z) and 1/rms of gelu'(z) for z ~ N(0,1) (the table prints
  *   them as 1.701 / 1.481); constrained: both equal their geometric mean.
+ * us_scales_activation: the same pair for any us_fn (relu: sqrt(2 / (1 - 1/pi)), sqrt 2; tanh
+ *   1.593 / 1.467; sigmoid 4.802 / 4.722 as printed, carried here to float precision).
  * Pure host arithmetic; output pointers must be non-NULL.
  */
 us_status us_scales_linear(int64_t b, int64_t m, int64_t n, int constrained, float* alpha,
                            float* beta_x, float* beta_w);
 us_status us_scales_gelu(int constrained, float* alpha, float* beta);
+us_status us_scales_activation(us_fn fn, int constrained, float* alpha, float* beta);
 
 const char* us_status_string(us_status s);
 int us_version(void);

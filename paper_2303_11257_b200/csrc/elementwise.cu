@@ -22,12 +22,37 @@ struct EwArgs {
   int64_t chunks_per_row;  // ceil(cols / kVec)
   int vec_ok;              // every row start of every tensor is 16-byte aligned
   float c0, c1, c2;        // op constants
+  int fn;                  // us_fn of the activation ops
 };
 
-enum EwOp { kCast = 0, kGeluFwd = 1, kGeluBwd = 2, kResidual = 3 };
+enum EwOp { kCast = 0, kGeluFwd = 1, kGeluBwd = 2, kResidual = 3, kActFwd = 4, kActBwd = 5 };
+
+// relu, tanh and sigmoid of the table "Activations" and their derivatives.  exp through ex2.approx and a
+// correctly rounded division: absolute error about 2e-7 for the bounded functions.
+__device__ __forceinline__ float sigmoid_f(float z) {
+  const float e = ex2_approx(-1.4426950408889634f * fabsf(z));     // e^-|z| in (0, 1]
+  const float r = __fdiv_rn(1.0f, 1.0f + e);
+  return z >= 0.f ? r : e * r;
+}
+__device__ __forceinline__ float act_value(int fn, float z) {
+  if (fn == US_FN_RELU) return fmaxf(z, 0.f);
+  if (fn == US_FN_TANH) return 2.0f * sigmoid_f(2.0f * z) - 1.0f;
+  if (fn == US_FN_SIGMOID) return sigmoid_f(z);
+  return 0.f;   // gelu is dispatched before this point
+}
+__device__ __forceinline__ float act_slope(int fn, float z) {
+  if (fn == US_FN_RELU) return z > 0.f ? 1.0f : 0.f;
+  if (fn == US_FN_TANH) { const float s = sigmoid_f(2.0f * z), m = sigmoid_f(-2.0f * z); return 4.0f * s * m; }   // 1 - tanh^2
+  if (fn == US_FN_SIGMOID) return sigmoid_f(z) * sigmoid_f(-z);
+  return 0.f;
+}
 
 template <int OP>
 __device__ __forceinline__ float ew_apply(float a, float b, const EwArgs& p) {
+  if (OP == kActFwd)                                                          // c0 = s_in, c1 = alpha
+    return p.fn == US_FN_GELU ? gelu_scaled(a, p.c0, p.c1) : p.c1 * act_value(p.fn, p.c0 * a);
+  if (OP == kActBwd)                                                          // a = H, b = dA, c1 = beta
+    return p.fn == US_FN_GELU ? gelu_grad_scaled(a, b, p.c0, p.c1) : (p.c1 * p.c0) * act_slope(p.fn, p.c0 * a) * b;
   if (OP == kCast) return p.c0 * a;                                   // scale * x, then the store rounds
   if (OP == kGeluFwd) return gelu_scaled(a, p.c0, p.c1);              // c0 = s_in, c1 = alpha
   if (OP == kGeluBwd) return gelu_grad_scaled(a, b, p.c0, p.c1);      // a = H, b = dA, c1 = beta
@@ -36,7 +61,7 @@ __device__ __forceinline__ float ew_apply(float a, float b, const EwArgs& p) {
 
 template <int OP>
 __global__ void __launch_bounds__(kThreads) ew_kernel(const EwArgs p) {
-  constexpr bool kTwoInputs = (OP == kGeluBwd || OP == kResidual);
+  constexpr bool kTwoInputs = (OP == kGeluBwd || OP == kResidual || OP == kActBwd);
   const int64_t total = p.rows * p.chunks_per_row;
   for (int64_t c = blockIdx.x * (int64_t)kThreads + threadIdx.x; c < total;
        c += (int64_t)gridDim.x * kThreads) {
@@ -134,8 +159,9 @@ static bool row_starts_aligned(const us_mat* m, bool contiguous) {
 
 template <int OP>
 static us_status ew_launch(const us_mat* in0, const us_mat* in1, const us_mat* out, float c0, float c1,
-                           void* stream) {
+                           void* stream, int fn = 0) {
   EwArgs p{};
+  p.fn = fn;
   // A tensor set without row padding is one long row: chunking then never straddles a row end.
   const bool contiguous = in0->ld == in0->cols && (!in1 || in1->ld == in1->cols) && out->ld == out->cols;
   p.rows = contiguous ? 1 : in0->rows;
@@ -228,6 +254,21 @@ extern "C" us_status us_gelu_bwd(const us_mat* H, const us_mat* dA, float s_in, 
   us_status s = check_ew(H, dA, dH);
   if (s != US_OK) return s;
   return ew_launch<kGeluBwd>(H, dA, dH, s_in, beta, stream);
+}
+
+extern "C" us_status us_activation_fwd(us_fn fn, const us_mat* H, float s_in, float alpha, const us_mat* A, void* stream) {
+  if (fn < US_FN_GELU || fn > US_FN_SIGMOID) return US_ERR_INVALID_ARG;
+  us_status s = check_ew(H, nullptr, A);
+  if (s != US_OK) return s;
+  return ew_launch<kActFwd>(H, nullptr, A, s_in, alpha, stream, fn);
+}
+
+extern "C" us_status us_activation_bwd(us_fn fn, const us_mat* H, const us_mat* dA, float s_in, float beta,
+                                       const us_mat* dH, void* stream) {
+  if (fn < US_FN_GELU || fn > US_FN_SIGMOID || !dA) return US_ERR_INVALID_ARG;
+  us_status s = check_ew(H, dA, dH);
+  if (s != US_OK) return s;
+  return ew_launch<kActBwd>(H, dA, dH, s_in, beta, stream, fn);
 }
 
 extern "C" us_status us_residual_add(const us_mat* skip, const us_mat* branch, float tau, const us_mat* out,

@@ -44,6 +44,24 @@ extern "C" us_status us_scales_gelu(int constrained, float* alpha, float* beta) 
   return US_OK;
 }
 
+extern "C" us_status us_scales_activation(us_fn fn, int constrained, float* alpha, float* beta) {
+  if (!alpha || !beta) return US_ERR_INVALID_ARG;
+  // 1 / std f(Z) and 1 / rms f'(Z) for Z ~ N(0, 1): relu in closed form (sqrt(2 / (1 - 1/pi)), sqrt 2),
+  // the others by numerical integration to the digits kept here (the table prints three of them).
+  double a, b;
+  switch (fn) {
+    case US_FN_GELU: a = kGeluAlpha; b = kGeluBeta; break;
+    case US_FN_RELU: a = 1.7128585504496627; b = 1.4142135623730951; break;
+    case US_FN_TANH: a = 1.5925374197228314; b = 1.4674135916307951; break;
+    case US_FN_SIGMOID: a = 4.8013133720399622; b = 4.7226460859379743; break;
+    default: return US_ERR_INVALID_ARG;
+  }
+  if (constrained) a = b = sqrt(a * b);
+  *alpha = (float)a;
+  *beta = (float)b;
+  return US_OK;
+}
+
 extern "C" const char* us_status_string(us_status s) {
   switch (s) {
     case US_OK: return "ok";

@@ -18,6 +18,8 @@ STATUS_NAMES = {
 }
 US_F32, US_BF16, US_F16, US_E4M3, US_E5M2 = range(5)
 US_ACT_NONE, US_ACT_GELU, US_ACT_GELU_GRAD = range(3)
+US_FN_GELU, US_FN_RELU, US_FN_TANH, US_FN_SIGMOID = range(4)
+FN_BY_NAME = {"gelu": US_FN_GELU, "relu": US_FN_RELU, "tanh": US_FN_TANH, "sigmoid": US_FN_SIGMOID}
 
 _TORCH_DTYPES = {
     torch.float32: US_F32, torch.bfloat16: US_BF16, torch.float16: US_F16,
@@ -76,6 +78,9 @@ def _load() -> C.CDLL:
     lib.us_gelu_bwd.argtypes = [MP, MP, F, F, MP, V]
     lib.us_residual_add.argtypes = [MP, MP, F, MP, V]
     lib.us_cast_fp8.argtypes = [MP, F, MP, V]
+    lib.us_activation_fwd.argtypes = [C.c_int, MP, F, F, MP, V]
+    lib.us_activation_bwd.argtypes = [C.c_int, MP, MP, F, F, MP, V]
+    lib.us_activation_fwd.restype = lib.us_activation_bwd.restype = C.c_int
     lib.us_cast_fp8_multi.argtypes = [C.c_int, MP, C.POINTER(C.c_float), MP, V]
     lib.us_softmax_fwd.argtypes = [MP, F, MP, V]
     lib.us_softmax_bwd.argtypes = [MP, MP, F, F, MP, V]
@@ -90,6 +95,8 @@ def _load() -> C.CDLL:
     lib.us_scales_linear.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_int, FP, FP, FP]
     lib.us_scales_linear.restype = C.c_int
     lib.us_scales_gelu.argtypes = [C.c_int, FP, FP]
+    lib.us_scales_activation.argtypes = [C.c_int, C.c_int, FP, FP]
+    lib.us_scales_activation.restype = C.c_int
     lib.us_scales_gelu.restype = C.c_int
     lib.us_status_string.argtypes = [C.c_int]
     lib.us_status_string.restype = C.c_char_p
@@ -224,6 +231,23 @@ def us_gelu_fwd(H, s_in, alpha, A, stream=None):
 def us_gelu_bwd(H, dA, s_in, beta, dH, stream=None):
     _check("us_gelu_bwd", _lib.us_gelu_bwd(C.byref(mat(H)), C.byref(mat(dA)), s_in, beta, C.byref(mat(dH)), _stream(stream)))
     return dH
+
+
+def us_activation_fwd(fn, H, s_in, alpha, A, stream=None):
+    _check("us_activation_fwd", _lib.us_activation_fwd(FN_BY_NAME.get(fn, fn), C.byref(mat(H)), s_in, alpha, C.byref(mat(A)), _stream(stream)))
+    return A
+
+
+def us_activation_bwd(fn, H, dA, s_in, beta, dH, stream=None):
+    _check("us_activation_bwd", _lib.us_activation_bwd(FN_BY_NAME.get(fn, fn), C.byref(mat(H)), C.byref(mat(dA)), s_in, beta,
+                                                       C.byref(mat(dH)), _stream(stream)))
+    return dH
+
+
+def us_scales_activation(fn, constrained: bool = False):
+    a, b = C.c_float(), C.c_float()
+    _check("us_scales_activation", _lib.us_scales_activation(FN_BY_NAME.get(fn, fn), int(constrained), C.byref(a), C.byref(b)))
+    return a.value, b.value
 
 
 def us_residual_add(skip, branch, tau, out, stream=None):

@@ -49,6 +49,14 @@ def test_scale_helpers_match_closed_forms(lib):
     assert round(lib.us_scales_gelu()[0], 3) == 1.701 and round(lib.us_scales_gelu()[1], 3) == 1.481
     with pytest.raises(lib.UnitScaleError):
         lib.us_scales_linear(0, 1, 1)
+    import math
+    for fn, want in (("relu", S.relu_scales()), ("tanh", S.tanh_scales()), ("sigmoid", S.sigmoid_scales()), ("gelu", S.gelu_scales())):
+        a, b = lib.us_scales_activation(fn)
+        assert abs(a - want[0]) < 5e-7 * want[0] and abs(b - want[1]) < 5e-7 * want[1]
+        c = lib.us_scales_activation(fn, True)
+        assert abs(c[0] - math.sqrt(want[0] * want[1])) < 1e-6 and c[0] == c[1]
+    with pytest.raises(lib.UnitScaleError):
+        lib.us_scales_activation(7)
 
 
 def test_status_strings_and_version(lib):

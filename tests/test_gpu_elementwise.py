@@ -82,3 +82,46 @@ def test_elementwise_argument_errors():
     with pytest.raises(L.UnitScaleError) as e:
         L.us_gelu_bwd(a, torch.zeros((4, 7), device="cuda"), 1.0, 1.0, a)
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("fn", ["relu", "tanh", "sigmoid", "gelu"])
+@pytest.mark.parametrize("in_fmt,out_fmt", [("f32", "f32"), ("bf16", "bf16"), ("fp16", "e4m3"), ("bf16", "e5m2")])
+@pytest.mark.parametrize("shape,ld", [((257, 1000), None), ((33, 48), 64)])
+def test_activation_fwd_bwd(fn, in_fmt, out_fmt, shape, ld):
+    """relu / tanh / sigmoid (and gelu through the same entry) with the table's scale factors.  exp goes
+    through ex2.approx in float32: 1e-6 absolute for the bounded functions, times the scale factor."""
+    L, synth = _lib()
+    alpha, beta = L.us_scales_activation(fn)
+    s_in = 0.875
+    h = synth.normal(6, 0, shape, 1.5)
+    h[0, :8] = [0.0, -0.0, 6.0, -6.0, 30.0, -30.0, 1e-8, -100.0]
+    g = synth.normal(6, 1, shape)
+    Ht, Gt = U.to_device(h, in_fmt, ld), U.to_device(g, in_fmt, ld)
+    hv, gv = U.values_of(h, in_fmt), U.values_of(g, in_fmt)
+    out = U.empty(shape[0], shape[1], out_fmt, ld)
+    L.us_activation_fwd(fn, Ht, s_in, alpha, out)
+    ref = O.activation_fwd(fn, hv, s_in, alpha)
+    U.assert_close_stored(out, ref, out_fmt, ABS * alpha * max(1.0, float(np.abs(ref).max()) / alpha / 8), "act fwd " + fn)
+    L.us_activation_bwd(fn, Ht, Gt, s_in, beta, out)
+    refb = O.activation_bwd(fn, hv, gv, s_in, beta)
+    U.assert_close_stored(out, refb, out_fmt, ABS * beta * np.abs(gv).max(), "act bwd " + fn)
+
+
+def test_activation_gelu_entry_equals_gelu_calls_and_unit_scale():
+    L, synth = _lib()
+    z = torch.from_numpy(synth.normal(7, 0, (1024, 2048))).cuda()
+    g = torch.from_numpy(synth.normal(7, 1, (1024, 2048))).cuda()
+    a, b = torch.empty_like(z), torch.empty_like(z)
+    L.us_activation_fwd("gelu", z, 1.0, 1.7, a); L.us_gelu_fwd(z, 1.0, 1.7, b)
+    assert torch.equal(a, b)
+    L.us_activation_bwd("gelu", z, g, 1.0, 1.48, a); L.us_gelu_bwd(z, g, 1.0, 1.48, b)
+    assert torch.equal(a, b)
+    for fn in ("relu", "tanh", "sigmoid"):
+        alpha, beta = L.us_scales_activation(fn)
+        L.us_activation_fwd(fn, z, 1.0, alpha, a)
+        assert abs(a.std().item() - 1) < 5e-3, fn
+        L.us_activation_bwd(fn, z, g, 1.0, beta, a)
+        assert abs(a.std().item() - 1) < 5e-3, fn
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_activation_fwd(9, z, 1.0, 1.0, a)
+    assert e.value.status == 1
