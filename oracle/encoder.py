@@ -10,6 +10,10 @@ att = "fp8", FP8 operands like every other matmul (section "Experiments": all ma
 quantised): Q, K, V and the softmax output P as E4, the gradients dC, dS and dQ, dK, dV as E5, while
 the softmax input S and the gradient dP of its output, which feed no matmul, stay in BF16.  Every
 stored intermediate is rounded to the format it is stored in.
+
+norm = "post" adds the post-norm arrangement of the appendix "Model architectures"
+(res^PostNorm(f, z) = layernorm(interp(z, f(z)))): each of the two residual sums goes through a scaled
+layer norm (table row layer_norm: alpha = 1, beta_x = 1, beta_w = beta_c = T^-1/2 for T tokens).
 """
 from __future__ import annotations
 
@@ -36,6 +40,13 @@ class EncoderResult:
     dX: np.ndarray = None
     dWqkv: np.ndarray = None
     dWo: np.ndarray = None
+    # post-norm only: the residual sums before each layer norm, the layer output, and the gradients of the norms
+    U1: np.ndarray = None
+    R2: np.ndarray = None
+    dU2: np.ndarray = None
+    dU1: np.ndarray = None
+    dln1: tuple = None          # (dw, dc) of the norm after the attention block
+    dln2: tuple = None          # (dw, dc) of the norm after the FFN block
 
 
 def _heads(M, nseq, slen, nhead, hd, which, d):
@@ -49,7 +60,10 @@ def _unheads(H, nseq, slen, nhead, hd):
     return H.transpose(0, 2, 1, 3).reshape(nseq * slen, nhead * hd)
 
 
-def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16") -> EncoderResult:
+def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16", norm=None, ln=None,
+                  eps=1e-5) -> EncoderResult:
+    """norm = None: R2 = res(ffn, res(attention, X)), G = dL/dR2 (the FFN block's output r.ffn.R).
+    norm = "post": ln = (w1, c1, w2, c2), each [d]; R1 = LN1(U1), R2 = LN2(U2) with U the residual sums."""
     T, d = X.shape
     hd = d // nhead
     f32 = lambda v: float(np.float32(v))
@@ -77,9 +91,26 @@ def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16"
     ep = O.Epilogue(skip=np.asarray(X, np.float64), skip_coef=c_skip, out_coef=c_branch)
     r.R1, _, _ = O.apply_epilogue(O.linear_fwd(r.Cq, Wo_q, a_o), ep, "bf16")
     sc = O.FFNScales.unconstrained(T, d, W1.shape[1], tau)
-    r.ffn = O.ffn_block(r.R1, W1, W2, G, sc, operand="fp8")
+    if norm == "post":
+        w1, c1, w2, c2 = (np.asarray(v, np.float64).reshape(1, d) for v in ln)
+        b_ln = f32(T ** -0.5)
+        r.U1 = r.R1
+        r.R1, _ = O.store(O.layer_norm_fwd(r.U1, w1, c1, f32(eps)), "bf16")
+        fwd = O.ffn_block(r.R1, W1, W2, np.zeros_like(np.asarray(G, np.float64)), sc, operand="fp8")   # forward part only
+        r.R2, _ = O.store(O.layer_norm_fwd(fwd.R, w2, c2, f32(eps)), "bf16")
+        # ---- backward through the second norm, the FFN block, the first norm
+        dU2, dw2, dc2 = O.layer_norm_bwd(fwd.R, w2, np.asarray(G, np.float64), f32(eps), 1.0, b_ln)
+        r.dU2, _ = O.store(dU2, "bf16")
+        r.dln2 = (O.store(dw2, "f32")[0], O.store(dc2, "f32")[0])
+        r.ffn = O.ffn_block(r.R1, W1, W2, r.dU2, sc, operand="fp8")
+        dU1, dw1, dc1 = O.layer_norm_bwd(r.U1, w1, r.ffn.dX, f32(eps), 1.0, b_ln)
+        r.dU1, _ = O.store(dU1, "bf16")
+        r.dln1 = (O.store(dw1, "f32")[0], O.store(dc1, "f32")[0])
+        g1 = r.dU1
+    else:
+        r.ffn = O.ffn_block(r.R1, W1, W2, G, sc, operand="fp8")
+        g1 = r.ffn.dX
     # ---- backward
-    g1 = r.ffn.dX
     g1q, _ = O.store(g1, "e5m2")
     r.dC, _ = O.store(O.linear_bwd_x(g1q, Wo_q, b_o), f_grad)
     r.dWo, _ = O.store(O.linear_bwd_w(r.Cq, g1q, b_w), "f32")

@@ -74,3 +74,27 @@ def test_fp8_attention_stays_close_to_16_bit_attention():
         x, y = getattr(a, name), getattr(b, name)
         assert np.abs(x - y).mean() < 0.25 * max(1.0, np.abs(x).std()), name
         assert np.corrcoef(x.ravel(), y.ravel())[0, 1] > 0.985, name
+
+
+def test_post_norm_layer_chains_the_single_op_functions_and_normalises_its_outputs():
+    nseq, slen, d, nhead, f = 2, 32, 64, 4, 128
+    t = _tensors(nseq, slen, d, f, seed=3)
+    rng = np.random.default_rng(3)
+    ln = (1 + 0.2 * rng.standard_normal(d), 0.1 * rng.standard_normal(d), 1 + 0.2 * rng.standard_normal(d), 0.1 * rng.standard_normal(d))
+    r = E.encoder_layer(*t, nseq, slen, nhead, norm="post", ln=ln)
+    plain = E.encoder_layer(*t, nseq, slen, nhead)
+    assert np.array_equal(r.U1, plain.R1)                                   # same attention block in front of the norm
+    eps = float(np.float32(1e-5))
+    assert np.array_equal(r.R1, O.store(O.layer_norm_fwd(r.U1, ln[0], ln[1], eps), "bf16")[0])
+    assert np.array_equal(r.R2, O.store(O.layer_norm_fwd(r.ffn.R, ln[2], ln[3], eps), "bf16")[0])
+    G = t[5]
+    dU2, dw2, dc2 = O.layer_norm_bwd(r.ffn.R, ln[2], G, eps)
+    assert np.array_equal(r.dU2, O.store(dU2, "bf16")[0]) and np.allclose(r.dln2[0], dw2, rtol=1e-6) and np.allclose(r.dln2[1], dc2, rtol=1e-6, atol=1e-7)
+    dU1, dw1, _ = O.layer_norm_bwd(r.U1, ln[0], r.ffn.dX, eps)
+    assert np.array_equal(r.dU1, O.store(dU1, "bf16")[0]) and np.allclose(r.dln1[0], dw1, rtol=1e-6)
+    # with unit weight and zero bias every token of the layer output has zero mean and unit variance
+    ones, zeros = np.ones(d), np.zeros(d)
+    u = E.encoder_layer(*t, nseq, slen, nhead, norm="post", ln=(ones, zeros, ones, zeros))
+    assert np.abs(u.R2.mean(axis=1)).max() < 0.02 and np.abs(u.R2.std(axis=1) - 1).max() < 0.02
+    # the norm gradients carry beta = T^-1/2: unit-ish scale
+    assert 0.3 < r.dln2[0].std() < 3 and 0.3 < r.dln1[0].std() < 3
