@@ -38,9 +38,9 @@ E4, E5 = torch.float8_e4m3fn, torch.float8_e5m2
 
 class UnitScaledEncoderLayer:
     def __init__(self, nseq: int, slen: int, d: int, nhead: int, d_ff: int, tau: float = 0.5,
-                 attention: str = "bf16", device="cuda"):
-        assert d % nhead == 0
-        self.attention = attention
+                 attention: str = "bf16", norm: str | None = None, eps: float = 1e-5, device="cuda"):
+        assert d % nhead == 0 and norm in (None, "post")
+        self.attention, self.norm, self.eps = attention, norm, eps
         if attention == "fp8":
             act_dt, grad_dt, wide_dt = E4, E5, torch.bfloat16
         else:
@@ -64,6 +64,13 @@ class UnitScaledEncoderLayer:
         self.dX = e(T, d, torch.bfloat16)
         self.dWqkv, self.dWo = e(d, 3 * d, torch.float32), e(d, d, torch.float32)
         self.ws = L.new_workspace(device)
+        if norm == "post":
+            # post-norm (appendix "Model architectures"): a scaled layer norm after each residual sum
+            self.U1, self.R2 = e(T, d, torch.bfloat16), e(T, d, torch.bfloat16)
+            self.dU1, self.dU2 = e(T, d, torch.bfloat16), e(T, d, torch.bfloat16)
+            self.dln = [torch.empty(d, dtype=torch.float32, device=device) for _ in range(4)]      # dw1, dc1, dw2, dc2
+            self.ln_ws = torch.empty(max(16, L.us_layer_norm_bwd_workspace_bytes(T, d)), dtype=torch.uint8, device=device)
+            self.beta_ln = T ** -0.5
         self.c_skip, self.c_branch = math.sqrt(1.0 - tau), math.sqrt(tau)
         s, hd = slen, self.hd
         self.sc = dict(
@@ -78,31 +85,44 @@ class UnitScaledEncoderLayer:
         self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
                        dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
         # fused cast, attention forward, FFN forward + backward, attention backward (one cast fewer with FP8 attention)
-        self.launches_per_step = 1 + 5 + 7 + (10 if attention == "fp8" else 11)
+        self.launches_per_step = 1 + 5 + 7 + (10 if attention == "fp8" else 11) + (7 if norm == "post" else 0)
 
     def _heads(self, M, which):
         """Problem (0, 0) of a [T x 3d] matrix: rows of the first sequence, columns of head 0 of Q / K / V."""
         o = which * self.d
         return M[: self.slen, o:o + self.hd]
 
-    def step(self, X, Wqkv, Wo, W1, W2, G, stream=None):
+    def step(self, X, Wqkv, Wo, W1, W2, G, stream=None, ln=None):
+        """One forward + backward pass.  G is the gradient of the layer output; with norm = "post",
+        ln = (w1, c1, w2, c2) are the weights and biases of the two layer norms ([d] each)."""
         sc, ws, s = self.sc, self.ws, self.slen
+        post = self.norm == "post"
         # ---- forward
         f = self.ffn
-        # every tensor that is known when the step starts goes to FP8 in one launch
-        L.us_cast_fp8_multi([Wqkv, Wo, X, W1, W2, G], [1.0] * 6,
-                            [self.Wqkv_q, self.Wo_q, self.Xq, f.W1q, f.W2q, f.Gq], stream)
+        # every tensor that is known when the step starts goes to FP8 in one launch (with post-norm the FFN
+        # block's incoming gradient is produced by the second norm's backward pass and is cast there)
+        L.us_cast_fp8_multi([Wqkv, Wo, X, W1, W2] + ([] if post else [G]), [1.0] * (5 if post else 6),
+                            [self.Wqkv_q, self.Wo_q, self.Xq, f.W1q, f.W2q] + ([] if post else [f.Gq]), stream)
         L.us_linear_fwd(self.Xq, self.Wqkv_q, sc["alpha_qkv"], self.QKV, ws, None, stream)
         Q, K, V = (self._heads(self.QKV, i) for i in range(3))
         L.us_linear_bwd_x_batched(Q, K, sc["alpha_s"], self.S[:s], self.bt["scores"], ws, stream)
         L.us_softmax_fwd(self.S, sc["sm"], self.P, stream)
         L.us_linear_fwd_batched(self.P[:s], V, sc["alpha_c"], self.Cq[:s, : self.hd], self.bt["ctx"], ws, stream)
         ep = L.epilogue(skip=X, skip_coef=self.c_skip, out_coef=self.c_branch)
-        L.us_linear_fwd(self.Cq, self.Wo_q, sc["alpha_o"], self.R1, ws, ep, stream)
+        L.us_linear_fwd(self.Cq, self.Wo_q, sc["alpha_o"], self.U1 if post else self.R1, ws, ep, stream)
+        if post:
+            L.us_layer_norm_fwd(self.U1, ln[0], ln[1], self.eps, self.R1, stream)
         f.forward(self.R1, stream)
         # ---- backward
-        f.backward(G, stream, cast_g=False)                     # f.dX = dL/dR1
-        g1 = f.dX
+        if post:
+            L.us_layer_norm_fwd(f.R, ln[2], ln[3], self.eps, self.R2, stream)
+            L.us_layer_norm_bwd(f.R, ln[2], G, self.eps, 1.0, self.beta_ln, self.dU2, self.dln[2], self.dln[3], self.ln_ws, stream)
+            f.backward(self.dU2, stream)                            # f.dX = dL/dR1
+            L.us_layer_norm_bwd(self.U1, ln[0], f.dX, self.eps, 1.0, self.beta_ln, self.dU1, self.dln[0], self.dln[1], self.ln_ws, stream)
+            g1 = self.dU1
+        else:
+            f.backward(G, stream, cast_g=False)                     # f.dX = dL/dR1
+            g1 = f.dX
         L.us_cast_fp8(g1, 1.0, self.g1q, stream)
         L.us_linear_bwd_x(self.g1q, self.Wo_q, sc["beta_o"], self.dC, ws, None, stream)
         L.us_linear_bwd_w(self.Cq, self.g1q, sc["beta_w"], self.dWo, ws, None, stream)

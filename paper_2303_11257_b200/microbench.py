@@ -66,17 +66,18 @@ def elementwise(rows=8192, cols=4096, nsets=4):
     return out
 
 
-def encoder_step(nseq=16, slen=512, d=1024, nhead=16, d_ff=4096, iters=10, attention="bf16"):
+def encoder_step(nseq=16, slen=512, d=1024, nhead=16, d_ff=4096, iters=10, attention="bf16", norm=None):
     T = nseq * slen
     host = (synth.normal(0, 0, (T, d)), synth.normal(0, 1, (d, 3 * d)), synth.normal(0, 2, (d, d)),
             synth.normal(0, 3, (d, d_ff)), synth.normal(0, 4, (d_ff, d)), synth.normal(0, 5, (T, d)))
     dev = [torch.from_numpy(t).cuda() for t in host]
-    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, d_ff, attention=attention)
-    layer.step(*dev)
+    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, d_ff, attention=attention, norm=norm)
+    ln = [torch.ones(d, device="cuda"), torch.zeros(d, device="cuda")] * 2 if norm else None
+    layer.step(*dev, ln=ln)
     layer.check()
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
-        layer.step(*dev)
+        layer.step(*dev, ln=ln)
     for _ in range(3):
         g.replay()
     torch.cuda.synchronize()
@@ -88,10 +89,11 @@ def encoder_step(nseq=16, slen=512, d=1024, nhead=16, d_ff=4096, iters=10, atten
     torch.cuda.synchronize()
     layer.check()
     t = e0.elapsed_time(e1) * 1e-3 / iters
-    return {"workload": f"encoder layer fwd+bwd 16x512 tokens, d=1024, 16 heads, d_ff=4096, {attention} attention operands", "ms_per_step": t * 1e3,
+    return {"workload": f"encoder layer fwd+bwd 16x512 tokens, d=1024, 16 heads, d_ff=4096, {attention} attention operands" + (", post-norm" if norm else ""), "ms_per_step": t * 1e3,
             "tflops": layer.flops() / t / 1e12, "tokens_per_s": T / t, "launches": layer.launches_per_step}
 
 
 if __name__ == "__main__":
     print(json.dumps({"elementwise": elementwise(), "encoder": encoder_step(),
-                      "encoder_fp8_attention": encoder_step(attention="fp8")}, indent=1))
+                      "encoder_fp8_attention": encoder_step(attention="fp8"),
+                      "encoder_fp8_attention_post_norm": encoder_step(attention="fp8", norm="post")}, indent=1))

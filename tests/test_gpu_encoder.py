@@ -107,3 +107,40 @@ def test_encoder_layer_fp8_attention(cfg):
     from oracle import formats as Fm
     d_p = U.code_distance(U.codes_of(layer.P), Fm.quantise_codes(r.P, Fm.E4M3), "e4m3")
     assert d_p.max() <= 2 and (d_p > 0).mean() < 0.08
+
+
+@pytest.mark.parametrize("attention", ["bf16", "fp8"])
+def test_encoder_layer_post_norm(attention):
+    """Post-norm arrangement: a scaled layer norm after each residual sum, forward and backward."""
+    from paper_2303_11257_b200 import encoder, synth
+    nseq, slen, d, nhead, f = 2, 128, 256, 4, 512
+    T = nseq * slen
+    host = (synth.normal(44, 0, (T, d)), synth.normal(44, 1, (d, 3 * d)), synth.normal(44, 2, (d, d)),
+            synth.normal(44, 3, (d, f)), synth.normal(44, 4, (f, d)), synth.normal(44, 5, (T, d)))
+    ln_host = [(1 + 0.2 * synth.normal(44, 6, (1, d)))[0], (0.1 * synth.normal(44, 7, (1, d)))[0],
+               (1 + 0.2 * synth.normal(44, 8, (1, d)))[0], (0.1 * synth.normal(44, 9, (1, d)))[0]]
+    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, f, attention=attention, norm="post")
+    layer.step(*[torch.from_numpy(t).cuda() for t in host], ln=[torch.from_numpy(v.astype(np.float32)).cuda() for v in ln_host])
+    layer.check()
+    r = E.encoder_layer(*host, nseq, slen, nhead, att=attention, norm="post", ln=[v.astype(np.float32) for v in ln_host])
+
+    def close(got, ref, name, mean_tol):
+        g = U.host_values(got)
+        scale = max(1.0, float(np.abs(ref).std()))
+        err = np.abs(g - ref) / scale
+        assert err.mean() <= mean_tol, f"{name}: mean err {err.mean():.3e}"
+        assert np.corrcoef(g.ravel(), ref.ravel())[0, 1] > 0.995, name
+
+    tol_f, tol_b = (2e-2, 8e-2) if attention == "fp8" else (1e-2, 5e-2)
+    for name, got, ref in (("U1", layer.U1, r.U1), ("R1", layer.R1, r.R1), ("U2", layer.ffn.R, r.ffn.R), ("R2", layer.R2, r.R2)):
+        close(got, ref, name, tol_f)
+    for name, got, ref in (("dU2", layer.dU2, r.dU2), ("dU1", layer.dU1, r.dU1), ("dX", layer.dX, r.dX), ("dWqkv", layer.dWqkv, r.dWqkv),
+                           ("dW1", layer.ffn.dW1, r.ffn.dW1), ("dln2_w", layer.dln[2], r.dln2[0].reshape(-1)),
+                           ("dln2_c", layer.dln[3], r.dln2[1].reshape(-1)), ("dln1_w", layer.dln[0], r.dln1[0].reshape(-1)),
+                           ("dln1_c", layer.dln[1], r.dln1[1].reshape(-1))):
+        close(got, ref, name, tol_b)
+    # the second norm's backward pass sees the same U2 up to chain noise and an exact G: strict-ish on its bias gradient
+    assert np.abs(layer.dln[3].cpu().numpy() - r.dln2[1].reshape(-1)).max() < 1e-4
+    # the layer output is normalised: per token, (R2 - c2) / w2 has zero mean and unit variance
+    z = (layer.R2.float().cpu().numpy() - ln_host[3]) / ln_host[2]
+    assert np.abs(z.mean(axis=1)).max() < 0.03 and np.abs(z.std(axis=1) - 1).max() < 0.03
