@@ -48,6 +48,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--operand", default="fp8", choices=["fp8", "bf16", "fp16"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--one-stream", action="store_true", help="issue the step's GEMMs on one stream (no overlap of independent launches)")
     return ap.parse_args()
 
 
@@ -281,6 +282,9 @@ def run_ours(args, rank: int, world: int, local: int):
     pinned = [[torch.from_numpy(t).pin_memory() for t in tensors] for tensors in host]
     sets = [[p.to(dev, non_blocking=True) for p in tensors] for tensors in pinned]
     blocks = [ffn.UnitScaledFFN(T, d, f, operand=args.operand, device=dev) for _ in sets]
+    if args.one_stream:
+        for b in blocks:
+            b.concurrent = False
     torch.cuda.synchronize()
     for blk, tensors in zip(blocks, sets):            # eager pass: first-call set-up happens here
         blk.step(*tensors)
