@@ -123,20 +123,38 @@ class UnitScaledEncoderLayer:
         else:
             f.backward(G, stream, cast_g=False)                     # f.dX = dL/dR1
             g1 = f.dX
-        L.us_cast_fp8(g1, 1.0, self.g1q, stream)
-        L.us_linear_bwd_x(self.g1q, self.Wo_q, sc["beta_o"], self.dC, ws, None, stream)
-        L.us_linear_bwd_w(self.Cq, self.g1q, sc["beta_w"], self.dWo, ws, None, stream)
+        # The weight-gradient GEMMs and one GEMM of each attention pair depend only on tensors that exist
+        # already; with no explicit stream they go to a side stream (parallel branches under graph capture).
+        par = stream is None and f.concurrent
+        cur = torch.cuda.current_stream() if par else stream
+        side = f._side_streams()[0] if par else stream
+
+        def beside(fn):
+            """Run fn on the side stream once everything issued so far on the main stream is done."""
+            if par:
+                ev = torch.cuda.Event()
+                ev.record(cur)
+                side.wait_event(ev)
+            fn(side)
+
+        L.us_cast_fp8(g1, 1.0, self.g1q, cur)
+        beside(lambda st: L.us_linear_bwd_w(self.Cq, self.g1q, sc["beta_w"], self.dWo, ws, None, st))
+        L.us_linear_bwd_x(self.g1q, self.Wo_q, sc["beta_o"], self.dC, ws, None, cur)
         dC_h = self.dC[:s, : self.hd]
-        L.us_linear_bwd_x_batched(dC_h, V, sc["beta_P"], self.dP[:s], self.bt["dP"], ws, stream)
-        L.us_linear_bwd_w_batched(self.P[:s], dC_h, sc["beta_V"], self._heads(self.dQKV, 2), self.bt["dV"], ws, stream)
-        L.us_softmax_bwd(self.P, self.dP, sc["sm"], sc["sm"], self.dS, stream)
-        L.us_linear_fwd_batched(self.dS[:s], K, sc["beta_Q"], self._heads(self.dQKV, 0), self.bt["dQ"], ws, stream)
-        L.us_linear_bwd_w_batched(self.dS[:s], Q, sc["beta_K"], self._heads(self.dQKV, 1), self.bt["dK"], ws, stream)
+        beside(lambda st: L.us_linear_bwd_w_batched(self.P[:s], dC_h, sc["beta_V"], self._heads(self.dQKV, 2), self.bt["dV"], ws, st))
+        L.us_linear_bwd_x_batched(dC_h, V, sc["beta_P"], self.dP[:s], self.bt["dP"], ws, cur)
+        L.us_softmax_bwd(self.P, self.dP, sc["sm"], sc["sm"], self.dS, cur)
+        beside(lambda st: L.us_linear_bwd_w_batched(self.dS[:s], Q, sc["beta_K"], self._heads(self.dQKV, 1), self.bt["dK"], ws, st))
+        L.us_linear_fwd_batched(self.dS[:s], K, sc["beta_Q"], self._heads(self.dQKV, 0), self.bt["dQ"], ws, cur)
+        if par:
+            cur.wait_stream(side)                                   # dQ, dK, dV all written
         if self.dQKV is not self.dQKVq:
-            L.us_cast_fp8(self.dQKV, 1.0, self.dQKVq, stream)
+            L.us_cast_fp8(self.dQKV, 1.0, self.dQKVq, cur)
+        beside(lambda st: L.us_linear_bwd_w(self.Xq, self.dQKVq, sc["beta_w"], self.dWqkv, ws, None, st))
         ep = L.epilogue(skip=g1, skip_coef=self.c_skip, out_coef=self.c_branch)
-        L.us_linear_bwd_x(self.dQKVq, self.Wqkv_q, sc["beta_qkv"], self.dX, ws, ep, stream)
-        L.us_linear_bwd_w(self.Xq, self.dQKVq, sc["beta_w"], self.dWqkv, ws, None, stream)
+        L.us_linear_bwd_x(self.dQKVq, self.Wqkv_q, sc["beta_qkv"], self.dX, ws, ep, cur)
+        if par:
+            cur.wait_stream(side)
         return self.dX
 
     def check(self) -> None:

@@ -132,11 +132,36 @@ class UnitScaledFFN:
             fn(stream)
         return self.R
 
+    def _side_streams(self):
+        if self._side is None:
+            self._side = (torch.cuda.Stream(), torch.cuda.Stream())
+        return self._side
+
     def backward(self, G, stream=None, cast_g: bool = True):
         """Backward pass from G = dL/dR.  cast_g=False: self.Gq already holds q(G) (a caller that
-        quantised G together with other tensors in one us_cast_fp8_multi launch)."""
-        for name, _, fn in self.stages(None, None, None, G, fused_casts=False)[5 if cast_g else 6:]:
-            fn(stream)
+        quantised G together with other tensors in one us_cast_fp8_multi launch).  With self.concurrent and
+        no explicit stream the two weight-gradient GEMMs run on side streams beside the input-gradient ones."""
+        st = self.stages(None, None, None, G, fused_casts=False)[5 if cast_g else 6:]
+        if not (self.concurrent and stream is None):
+            for name, _, fn in st:
+                fn(stream)
+            return self.dX, self.dW1, self.dW2
+        by = {name: fn for name, _, fn in st}
+        cur = torch.cuda.current_stream()
+        s_b, s_c = self._side_streams()
+        if cast_g:
+            by["cast_G"](cur)
+        s_b.wait_stream(cur)
+        s_c.wait_stream(cur)
+        by["bwd_w2"](s_c)
+        by["bwd_x2_gelu_grad"](cur)
+        have_dh = torch.cuda.Event()
+        have_dh.record(cur)
+        s_b.wait_event(have_dh)
+        by["bwd_w1"](s_b)
+        by["bwd_x1_residual"](cur)
+        cur.wait_stream(s_b)
+        cur.wait_stream(s_c)
         return self.dX, self.dW1, self.dW2
 
     def step(self, X, W1, W2, G, stream=None):
@@ -151,9 +176,7 @@ class UnitScaledFFN:
             return self.dX, self.dW1, self.dW2
         by = {name: fn for name, _, fn in st}
         cur = torch.cuda.current_stream()
-        if self._side is None:
-            self._side = (torch.cuda.Stream(), torch.cuda.Stream())
-        s_b, s_c = self._side
+        s_b, s_c = self._side_streams()
         by["cast_all"](cur)
         by["fwd1_gelu"](cur)
         s_b.wait_stream(cur)
