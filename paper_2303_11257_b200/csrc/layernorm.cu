@@ -299,7 +299,7 @@ __global__ void __launch_bounds__(kLnThreads, 2) ln_fwd16_kernel(const LnArgs a)
 }
 
 template <int NCH>
-__global__ void __launch_bounds__(kLnThreads) ln_bwd16_kernel(const LnArgs a) {
+__global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
   extern __shared__ __align__(16) float ln_smem[];                         // w[cols] as float32, then [warps][cols] for the combine
   float* w_s = ln_smem;
   float* comb = ln_smem + a.cols;
@@ -432,13 +432,15 @@ static us_status check_vector(const us_mat* v, int64_t cols, bool input) {
   return US_OK;
 }
 
-static int ln_bwd_grid(int64_t rows) {
+// CTAs of the backward kernel: `warps` rows in flight per CTA, at most `per_sm` CTAs per SM.
+static int ln_bwd_grid(int64_t rows, int warps = kLnWarps, int per_sm = 2) {
   const int sms = host::sm_count();
   if (sms <= 0) return 0;
-  const int64_t want = (rows + kLnWarps - 1) / kLnWarps;
-  const int64_t cap = (int64_t)sms * 2;
+  const int64_t want = (rows + warps - 1) / warps;
+  const int64_t cap = (int64_t)sms * per_sm;
   return (int)(want < cap ? want : cap);
 }
+constexpr int kLnFastWarps = 4, kLnFastPerSm = 3;   // the 16-bit backward kernel: three CTAs of four warps per SM
 
 }  // namespace us
 
@@ -484,7 +486,8 @@ extern "C" us_status us_layer_norm_fwd(const us_mat* X, const us_mat* w, const u
 
 extern "C" size_t us_layer_norm_bwd_workspace_bytes(int64_t rows, int64_t cols) {
   if (rows <= 0 || cols <= 0) return 0;
-  const int grid = ln_bwd_grid(rows);
+  const int g0 = ln_bwd_grid(rows), g1 = ln_bwd_grid(rows, kLnFastWarps, kLnFastPerSm);
+  const int grid = g0 > g1 ? g0 : g1;                // whichever kernel the call takes
   return (size_t)(grid > 0 ? grid : 1) * 2 * (size_t)cols * sizeof(float);
 }
 
@@ -503,7 +506,7 @@ extern "C" us_status us_layer_norm_bwd(const us_mat* X, const us_mat* w, const u
   if (X->cols == 0) return US_OK;
   const int grid = ln_bwd_grid(X->rows > 0 ? X->rows : 1);
   if (grid <= 0) return US_ERR_CUDA;
-  if (!ws || ws_bytes < (size_t)grid * 2 * (size_t)X->cols * sizeof(float)) return US_ERR_WORKSPACE;
+  if (!ws || ws_bytes < us_layer_norm_bwd_workspace_bytes(X->rows > 0 ? X->rows : 1, X->cols)) return US_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(ws) % 16) return US_ERR_ALIGNMENT;
   LnArgs a{};
   a.x = X->ptr; a.x_dt = X->dtype; a.x_ld = X->ld;
@@ -518,12 +521,11 @@ extern "C" us_status us_layer_norm_bwd(const us_mat* X, const us_mat* w, const u
   int nparts = grid;
   // With no rows the first kernel still runs (one CTA) and writes zero partials, so dw = dc = 0.
   if (a.vec_ok && nch <= 4 && (a.x_dt == US_BF16 || a.x_dt == US_F16) && a.g_dt == a.x_dt) {
-    const int sms = host::sm_count();
-    nparts = grid < sms ? grid : sms;                          // one resident CTA per SM
-    const size_t smem = (size_t)(1 + kLnWarps) * a.cols * sizeof(float);
-    if (nch <= 1) ln_bwd16_kernel<1><<<nparts, kLnThreads, smem, st>>>(a);
-    else if (nch <= 2) ln_bwd16_kernel<2><<<nparts, kLnThreads, smem, st>>>(a);
-    else ln_bwd16_kernel<4><<<nparts, kLnThreads, smem, st>>>(a);
+    nparts = ln_bwd_grid(X->rows > 0 ? X->rows : 1, kLnFastWarps, kLnFastPerSm);
+    const size_t smem = (size_t)(1 + kLnFastWarps) * a.cols * sizeof(float);
+    if (nch <= 1) ln_bwd16_kernel<1><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);
+    else if (nch <= 2) ln_bwd16_kernel<2><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);
+    else ln_bwd16_kernel<4><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);
   } else if (nch <= 4) {
     const size_t smem = (size_t)kLnWarps * a.cols * sizeof(float);
     if (nch <= 1) ln_bwd_kernel<1><<<grid, kLnThreads, smem, st>>>(a);
