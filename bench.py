@@ -432,7 +432,8 @@ def run_ours(args, rank: int, world: int, local: int):
         "config": {"workload": "ffn_bert_large fwd+bwd: T=8192 tokens (16x512), d_model=1024, d_ff=4096, tau=0.5",
                    "operand": args.operand, "replicas": world,
                    "l2": "two rotating input/buffer sets, ~0.45 GB touched per step (> 126 MB L2)",
-                   "launch": "one CUDA graph of 10 kernels per step"},
+                   "launch": f"one CUDA graph of {blocks[0].launches_per_step} kernels per step, "
+                             + ("GEMMs after the first on three streams" if blocks[0].concurrent else "one stream")},
         "tokens_per_s": T * world / (ms_per_step * 1e-3),
         "pct_of_nominal_fp8_peak": 100.0 * value / world / NOMINAL_FP8_TFLOPS,
         "pct_of_measured_tensor_peak": 100.0 * value / world / tensor_peak,
