@@ -130,3 +130,29 @@ def test_ffn_saturation_and_underflow_in_fused_cast(sigma):
     dA = U.code_deltas(blk.Aq, r.Aq_codes, "e4m3")
     tol = TOL * max(1.0, np.abs(r.dW2).max()) + blk.sc.beta_w * U.propagated(dA.T, r.Gq, "a")
     U.assert_close_stored(blk.dW2, r.dW2, "f32", tol, "dW2")
+
+
+def test_step_on_three_streams_equals_step_on_one_stream():
+    """The multi-stream issue order changes when kernels run, not what they compute: bit-identical outputs,
+    eagerly and from a captured graph."""
+    ffn, L, synth = _mods()
+    shape = synth.FFN_RAGGED
+    tensors = [torch.from_numpy(t).cuda() for t in synth.ffn_tensors(shape, seed=5)]
+    outs = []
+    for concurrent in (False, True):
+        blk = ffn.UnitScaledFFN(shape.tokens, shape.d_model, shape.d_ff)
+        blk.concurrent = concurrent
+        blk.step(*tensors)
+        blk.check()
+        eager = [t.clone() for t in (blk.R, blk.dX, blk.dW1, blk.dW2)]
+        g = blk.capture(*tensors)
+        for t in (blk.R, blk.dX, blk.dW1, blk.dW2):
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        blk.check()
+        for a, b in zip(eager, (blk.R, blk.dX, blk.dW1, blk.dW2)):
+            assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+        outs.append(eager)
+    for a, b in zip(*outs):
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
