@@ -136,6 +136,30 @@ def softmax_bwd(P, dP, alpha, beta):
     return _f32(beta) * p * (dP - np.sum(p * dP, axis=-1, keepdims=True))
 
 
+# --------------------------------------------------------------------------- softmax cross-entropy
+
+def softmax_xent_fwd(X, t):
+    """softmax_xent(x, t) = log softmax(x)_t per row (table row "softmax_xent", alpha = 1):
+    x_t - max(x) - log sum_j exp(x_j - max(x)).  t: integer class index per row."""
+    X = np.asarray(X, np.float64)
+    t = np.asarray(t, np.int64)
+    m = X.max(axis=-1, keepdims=True)
+    lse = np.log(np.exp(X - m).sum(axis=-1)) + m[..., 0]
+    return np.take_along_axis(X, t[..., None], axis=-1)[..., 0] - lse
+
+
+def softmax_xent_bwd(X, t, g, beta):
+    """beta * g_i * d softmax_xent(x, t)_i / dx = beta * g_i * (onehot(t_i) - softmax(x_i));
+    the table gives beta = s / sqrt(s - 1) for rows of s classes.  g: one incoming gradient per row."""
+    X = np.asarray(X, np.float64)
+    t = np.asarray(t, np.int64)
+    e = np.exp(X - X.max(axis=-1, keepdims=True))
+    p = e / e.sum(axis=-1, keepdims=True)
+    onehot = np.zeros_like(p)
+    np.put_along_axis(onehot, t[..., None], 1.0, axis=-1)
+    return _f32(beta) * np.asarray(g, np.float64)[..., None] * (onehot - p)
+
+
 # --------------------------------------------------------------------------- layer norm
 
 def layer_norm_fwd(X, w, c, eps=0.0):

@@ -108,3 +108,8 @@ def layer_norm_scales(b: int):
     """(alpha, beta_x, beta_w, beta_c) of layer_norm on a b x n input (table row "layer_norm"):
     alpha = 1, beta_x = 1, beta_w = beta_c = b^-1/2."""
     return 1.0, 1.0, b ** -0.5, b ** -0.5
+
+
+def softmax_xent_scales(s: int):
+    """(alpha, beta) of softmax_xent over s classes (table row "softmax_xent"): alpha = 1, beta = s / sqrt(s - 1)."""
+    return 1.0, s / math.sqrt(s - 1)
