@@ -238,6 +238,20 @@ us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, co
 us_status us_softmax_fwd(const us_mat* S, float alpha, const us_mat* P, void* stream);
 us_status us_softmax_bwd(const us_mat* P, const us_mat* dP, float alpha, float beta, const us_mat* dS, void* stream);
 
+/* Softmax cross-entropy (table row softmax_xent: softmax_xent(x, t) = log softmax(x)_t, alpha = 1,
+ * beta = s / sqrt(s - 1) for rows of s classes).
+ *
+ *   us_softmax_xent_fwd   out_i = x_{i,t_i} - log sum_j exp(x_ij)               (float32, one per row, <= 0)
+ *   us_softmax_xent_bwd   dX_ij = beta * g_i * ([j == t_i] - softmax(x_i)_j)    (g == NULL: g_i = 1)
+ *
+ * X [rows x s]: F32, BF16 or F16, any ld >= s; targets: device array of rows int32 class indices in
+ * [0, s) (an index outside gives NaN forward and no one-hot term backward); out, g: device float32
+ * arrays of rows elements; dX: any us_dtype, shape of X.
+ */
+us_status us_softmax_xent_fwd(const us_mat* X, const int32_t* targets, float* out, void* stream);
+us_status us_softmax_xent_bwd(const us_mat* X, const int32_t* targets, const float* g, float beta,
+                              const us_mat* dX, void* stream);
+
 /* ------------------------------------------------------------ scaled layer norm
  *
  * layer_norm(X, w, c)_ij = c_j + w_j (X_ij - mu_i) / sigma_i over the rows of X [b x n], mu_i the row

@@ -132,6 +132,76 @@ __global__ void __launch_bounds__(kSmThreads) softmax_bwd_kernel(const SmArgs a)
   }
 }
 
+// ---------------------------------------------------------------- softmax cross-entropy
+// softmax_xent(x, t) = log softmax(x)_t (table row "softmax_xent": alpha = 1, beta = s / sqrt(s - 1)).
+// One warp per row; the row is read twice (maximum, then sum of exponentials) from global memory /
+// cache, which keeps any class count in one code path; the backward pass reads it a third time to write
+// beta * g * (onehot(t) - softmax(x)).
+struct XentArgs {
+  const void* x; int x_dt; int64_t x_ld;
+  const int32_t* t;
+  const float* g;          // backward: one gradient per row, or null for ones
+  void* out; int out_dt; int64_t out_ld;   // forward: float32 [rows]; backward: dX
+  int64_t rows; int cols;
+  int vec_ok;
+  float beta;
+};
+
+template <bool BWD>
+__global__ void __launch_bounds__(kSmThreads) softmax_xent_kernel(const XentArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (kSmThreads / 32) + (threadIdx.x >> 5);
+  if (row >= a.rows) return;
+  const int64_t x_off = row * a.x_ld;
+  const bool vec = a.vec_ok != 0;
+  const int nch = (a.cols + 255) / 256;
+  float m = -INFINITY;
+  for (int c = 0; c < nch; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    if (col >= a.cols) continue;
+    float v[8];
+    load8(a.x, a.x_dt, x_off, col, a.cols, vec, -INFINITY, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m = fmaxf(m, v[i]);
+  }
+  m = warp_max(m);
+  const float mb = m * kLog2e;
+  float sum = 0.f;
+  for (int c = 0; c < nch; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    if (col >= a.cols) continue;
+    float v[8];
+    load8(a.x, a.x_dt, x_off, col, a.cols, vec, -INFINITY, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sum += ex2_approx(fmaf(v[i], kLog2e, -mb));
+  }
+  sum = warp_sum(sum);
+  const int t = a.t[row];
+  const bool valid = t >= 0 && t < a.cols;                   // a target outside the row: NaN forward, no one-hot term backward
+  if (!BWD) {
+    if (lane == 0) {
+      const float xt = valid ? load_one(a.x, a.x_dt, x_off + t) : __int_as_float(0x7fc00000);
+      static_cast<float*>(a.out)[row] = (xt - m) - 0.6931471805599453f * __log2f(sum);
+    }
+    return;
+  }
+  const float k = a.beta * (a.g ? a.g[row] : 1.0f);
+  const float inv = 1.0f / sum;
+  const int64_t out_off = row * a.out_ld;
+  for (int c = 0; c < nch; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    if (col >= a.cols) continue;
+    float v[8];
+    load8(a.x, a.x_dt, x_off, col, a.cols, vec, -INFINITY, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float p = ex2_approx(fmaf(v[i], kLog2e, -mb)) * inv;
+      v[i] = k * ((col + i == t ? 1.0f : 0.f) - p);
+    }
+    store8(a.out, a.out_dt, out_off, col, a.cols, vec, v);
+  }
+}
+
 static bool rows_aligned(const us_mat* m) {
   return reinterpret_cast<uintptr_t>(m->ptr) % 16 == 0 && (m->ld * dtype_size(m->dtype)) % 16 == 0;
 }
@@ -200,4 +270,46 @@ extern "C" us_status us_softmax_bwd(const us_mat* P, const us_mat* dP, float alp
   a.rows = P->rows; a.cols = (int)P->cols; a.alpha = alpha; a.beta = beta;
   a.vec_ok = rows_aligned(P) && rows_aligned(dP) && rows_aligned(dS) && P->cols % 8 == 0;
   return launch_softmax<true>(a, static_cast<cudaStream_t>(stream));
+}
+
+static us_status check_xent(const us_mat* X, const int32_t* targets) {
+  us_status s = check_mat(X, nullptr, true);
+  if (s != US_OK) return s;
+  if (X->rows > 0 && !targets) return US_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(targets) % 4) return US_ERR_ALIGNMENT;
+  if (X->rows > 0 && X->cols < 1) return US_ERR_INVALID_ARG;
+  return US_OK;
+}
+
+extern "C" us_status us_softmax_xent_fwd(const us_mat* X, const int32_t* targets, float* out, void* stream) {
+  us_status s = check_xent(X, targets);
+  if (s != US_OK) return s;
+  if (X->rows == 0) return US_OK;
+  if (!out || reinterpret_cast<uintptr_t>(out) % 4) return US_ERR_INVALID_ARG;
+  XentArgs a{};
+  a.x = X->ptr; a.x_dt = X->dtype; a.x_ld = X->ld; a.t = targets; a.out = out;
+  a.rows = X->rows; a.cols = (int)X->cols;
+  a.vec_ok = rows_aligned(X) && X->cols % 8 == 0;
+  const int64_t grid = (a.rows + kSmThreads / 32 - 1) / (kSmThreads / 32);
+  if (grid > 0x7fffffff) return US_ERR_INVALID_ARG;
+  softmax_xent_kernel<false><<<(int)grid, kSmThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
+}
+
+extern "C" us_status us_softmax_xent_bwd(const us_mat* X, const int32_t* targets, const float* g, float beta,
+                                         const us_mat* dX, void* stream) {
+  us_status s = check_xent(X, targets);
+  if (s == US_OK) s = check_mat(dX, X, false);
+  if (s != US_OK) return s;
+  if (g && reinterpret_cast<uintptr_t>(g) % 4) return US_ERR_ALIGNMENT;
+  if (X->rows == 0) return US_OK;
+  XentArgs a{};
+  a.x = X->ptr; a.x_dt = X->dtype; a.x_ld = X->ld; a.t = targets; a.g = g;
+  a.out = dX->ptr; a.out_dt = dX->dtype; a.out_ld = dX->ld;
+  a.rows = X->rows; a.cols = (int)X->cols; a.beta = beta;
+  a.vec_ok = rows_aligned(X) && rows_aligned(dX) && X->cols % 8 == 0;
+  const int64_t grid = (a.rows + kSmThreads / 32 - 1) / (kSmThreads / 32);
+  if (grid > 0x7fffffff) return US_ERR_INVALID_ARG;
+  softmax_xent_kernel<true><<<(int)grid, kSmThreads, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }

@@ -84,6 +84,9 @@ def _load() -> C.CDLL:
     lib.us_cast_fp8_multi.argtypes = [C.c_int, MP, C.POINTER(C.c_float), MP, V]
     lib.us_softmax_fwd.argtypes = [MP, F, MP, V]
     lib.us_softmax_bwd.argtypes = [MP, MP, F, F, MP, V]
+    lib.us_softmax_xent_fwd.argtypes = [MP, V, V, V]
+    lib.us_softmax_xent_bwd.argtypes = [MP, V, V, F, MP, V]
+    lib.us_softmax_xent_fwd.restype = lib.us_softmax_xent_bwd.restype = C.c_int
     lib.us_layer_norm_fwd.argtypes = [MP, MP, MP, F, MP, V]
     lib.us_layer_norm_bwd.argtypes = [MP, MP, MP, F, F, F, MP, MP, MP, V, SZ, V]
     lib.us_layer_norm_fwd.restype = lib.us_layer_norm_bwd.restype = C.c_int
@@ -278,6 +281,21 @@ def us_softmax_fwd(S, alpha, P, stream=None):
 def us_softmax_bwd(P, dP, alpha, beta, dS, stream=None):
     _check("us_softmax_bwd", _lib.us_softmax_bwd(C.byref(mat(P)), C.byref(mat(dP)), alpha, beta, C.byref(mat(dS)), _stream(stream)))
     return dS
+
+
+def us_softmax_xent_fwd(X, targets, out, stream=None):
+    """targets: int32 CUDA tensor [rows]; out: float32 CUDA tensor [rows]."""
+    assert targets.dtype == torch.int32 and out.dtype == torch.float32 and targets.is_contiguous() and out.is_contiguous()
+    _check("us_softmax_xent_fwd", _lib.us_softmax_xent_fwd(C.byref(mat(X)), targets.data_ptr(), out.data_ptr(), _stream(stream)))
+    return out
+
+
+def us_softmax_xent_bwd(X, targets, g, beta, dX, stream=None):
+    """g: float32 CUDA tensor [rows] or None (ones)."""
+    assert targets.dtype == torch.int32 and targets.is_contiguous() and (g is None or (g.dtype == torch.float32 and g.is_contiguous()))
+    _check("us_softmax_xent_bwd", _lib.us_softmax_xent_bwd(C.byref(mat(X)), targets.data_ptr(), g.data_ptr() if g is not None else None,
+                                                           beta, C.byref(mat(dX)), _stream(stream)))
+    return dX
 
 
 def _vec(t: torch.Tensor) -> us_mat:
