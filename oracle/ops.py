@@ -118,6 +118,19 @@ def residual_add(skip, branch, tau):
     return weighted_add(skip, branch, ca, cb)
 
 
+def weighted_add_n(xs, gammas, alpha=None):
+    """alpha * sum_i gamma_i x_i (table row "weighted_add": alpha = (sum_i gamma_i^2)^-1/2, which keeps
+    unit variance for independent unit-variance inputs; beta_i = 1 / gamma_i makes every input's
+    gradient the incoming gradient times alpha * gamma_i * beta_i = alpha)."""
+    gam = [_f32(g) for g in gammas]
+    if alpha is None:
+        alpha = sum(g * g for g in gam) ** -0.5
+    acc = np.zeros_like(np.asarray(xs[0], np.float64))
+    for g, x in zip(gam, xs):
+        acc = acc + g * np.asarray(x, np.float64)
+    return _f32(alpha) * acc
+
+
 # --------------------------------------------------------------------------- softmax
 
 def softmax_fwd(S, alpha):

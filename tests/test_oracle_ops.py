@@ -200,3 +200,17 @@ def test_ffn_chain_statistics_at_initialisation():
 
 def test_ffn_flops():
     assert O.ffn_flops(8192, 1024, 4096) == 6 * 2 * 8192 * 1024 * 4096
+
+
+def test_weighted_add_n_keeps_unit_variance_and_reduces_to_the_residual_add():
+    rng = np.random.default_rng(11)
+    xs = [rng.standard_normal((64, 512)) for _ in range(3)]
+    out = O.weighted_add_n(xs, [1.0, 0.5, 2.0])
+    assert abs(out.std() - 1) < 0.02                                   # alpha = (sum gamma^2)^-1/2
+    direct = (1.0 * xs[0] + 0.5 * xs[1] + 2.0 * xs[2]) / np.sqrt(1 + 0.25 + 4)
+    assert np.allclose(out, direct, rtol=1e-6, atol=1e-6)
+    tau = 0.3                                                          # n = 2 with gamma = (sqrt(1-tau), sqrt(tau)): alpha = 1
+    two = O.weighted_add_n(xs[:2], [np.sqrt(1 - tau), np.sqrt(tau)], alpha=1.0)
+    assert np.allclose(two, O.residual_add(xs[0], xs[1], tau), rtol=1e-12, atol=1e-12)
+    l = 5                                                              # running-mean residual: tau = 1 / (l + 1)
+    assert np.allclose(O.residual_add(xs[0], xs[1], 1 / (l + 1)), np.sqrt(l / (l + 1)) * xs[0] + np.sqrt(1 / (l + 1)) * xs[1], rtol=1e-6, atol=1e-6)
