@@ -191,6 +191,13 @@ typedef enum { US_FN_GELU = 0, US_FN_RELU = 1, US_FN_TANH = 2, US_FN_SIGMOID = 3
  *                  or gelu (table rows relu / gelu / tanh / sigmoid: alpha = 1 / std f(Z), Z ~ N(0,1));
  * us_activation_bwd  dH = beta * s_in * f'(s_in * H) * dA (beta = 1 / rms f'(Z)); relu'(0) = 0.
  *                  US_FN_GELU gives the same values as us_gelu_fwd / us_gelu_bwd.
+ * us_weighted_add  out = alpha * sum_i gamma_i * src_i over count (1..8) tensors of one shape (table row
+ *                  weighted_add: alpha = (sum_i gamma_i^2)^-1/2 keeps unit scale; each input's gradient
+ *                  is then the incoming gradient times alpha * gamma_i * beta_i with beta_i = 1 /
+ *                  gamma_i, i.e. no kernel of its own).  The coefficient alpha * gamma_i is formed in
+ *                  float32 and applied by one fused multiply-add per input, in the order given.
+ *                  The running-mean residual of section "Weighted addition" is us_residual_add
+ *                  with tau = 1 / (l + 1).  src, gamma: host arrays of count elements.
  * us_cast_fp8      dst = q(scale * src), q = nearest value of the FP8 format, ties to
  *                  even, saturating (section "Floating-point formats for deep learning",
  *                  paragraph "Quantisation error"); the product is one float32
@@ -216,6 +223,8 @@ us_status us_activation_fwd(us_fn fn, const us_mat* H, float s_in, float alpha, 
 us_status us_activation_bwd(us_fn fn, const us_mat* H, const us_mat* dA, float s_in, float beta,
                             const us_mat* dH, void* stream);
 us_status us_residual_add(const us_mat* skip, const us_mat* branch, float tau, const us_mat* out,
+                          void* stream);
+us_status us_weighted_add(int count, const us_mat* src, const float* gamma, float alpha, const us_mat* out,
                           void* stream);
 us_status us_cast_fp8(const us_mat* src, float scale, const us_mat* dst, void* stream);
 us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, const us_mat* dst,

@@ -151,6 +151,45 @@ __global__ void __launch_bounds__(kThreads) multi_cast_kernel(const MultiCastArg
   }
 }
 
+// alpha * sum_i gamma_i x_i over up to kMultiMax tensors of one shape (table row "weighted_add").
+struct WeightedAddArgs {
+  const void* src[kMultiMax];
+  int src_dt[kMultiMax];
+  int64_t src_ld[kMultiMax];
+  float coef[kMultiMax];          // alpha * gamma_i
+  void* out; int out_dt; int64_t out_ld;
+  int count;
+  int64_t rows, cols, chunks_per_row;
+  int vec_ok;
+};
+
+__global__ void __launch_bounds__(kThreads) weighted_add_kernel(const WeightedAddArgs p) {
+  const int64_t total = p.rows * p.chunks_per_row;
+  for (int64_t c = blockIdx.x * (int64_t)kThreads + threadIdx.x; c < total; c += (int64_t)gridDim.x * kThreads) {
+    const int64_t row = c / p.chunks_per_row;
+    const int64_t col = (c - row * p.chunks_per_row) * kVec;
+    if (p.vec_ok && col + kVec <= p.cols) {
+      float acc[kVec];
+#pragma unroll
+      for (int i = 0; i < kVec; ++i) acc[i] = 0.f;
+      for (int t = 0; t < p.count; ++t) {
+        float a[kVec];
+        load_vec<kVec>(static_cast<const char*>(p.src[t]) + (row * p.src_ld[t] + col) * dtype_size(p.src_dt[t]), p.src_dt[t], a);
+#pragma unroll
+        for (int i = 0; i < kVec; ++i) acc[i] = fmaf(p.coef[t], a[i], acc[i]);
+      }
+      store_vec<kVec>(static_cast<char*>(p.out) + (row * p.out_ld + col) * dtype_size(p.out_dt), p.out_dt, acc);
+    } else {
+      const int n = (int)min((int64_t)kVec, p.cols - col);
+      for (int i = 0; i < n; ++i) {
+        float acc = 0.f;
+        for (int t = 0; t < p.count; ++t) acc = fmaf(p.coef[t], load_one(p.src[t], p.src_dt[t], row * p.src_ld[t] + col + i), acc);
+        store_one(p.out, p.out_dt, row * p.out_ld + col + i, acc);
+      }
+    }
+  }
+}
+
 static bool row_starts_aligned(const us_mat* m, bool contiguous) {
   const int es = dtype_size(m->dtype);
   if (reinterpret_cast<uintptr_t>(m->ptr) % 16) return false;
@@ -239,6 +278,31 @@ extern "C" us_status us_cast_fp8_multi(int count, const us_mat* src, const float
   const int64_t want = (chunks + kThreads - 1) / kThreads;
   const int64_t cap = (int64_t)sms * 8;
   multi_cast_kernel<<<(int)(want < cap ? want : cap), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+  return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
+}
+
+extern "C" us_status us_weighted_add(int count, const us_mat* src, const float* gamma, float alpha, const us_mat* out,
+                                      void* stream) {
+  if (count < 1 || count > kMultiMax || !src || !gamma || !out) return US_ERR_INVALID_ARG;
+  WeightedAddArgs p{};
+  bool vec = row_starts_aligned(out, false);
+  for (int i = 0; i < count; ++i) {
+    us_status s = check_ew(&src[i], nullptr, out);
+    if (s != US_OK) return s;
+    p.src[i] = src[i].ptr; p.src_dt[i] = src[i].dtype; p.src_ld[i] = src[i].ld;
+    p.coef[i] = alpha * gamma[i];
+    vec = vec && row_starts_aligned(&src[i], false);
+  }
+  p.out = out->ptr; p.out_dt = out->dtype; p.out_ld = out->ld;
+  p.count = count; p.rows = out->rows; p.cols = out->cols;
+  p.chunks_per_row = (p.cols + kVec - 1) / kVec;
+  p.vec_ok = vec;
+  const int64_t total = p.rows * p.chunks_per_row;
+  if (total == 0) return US_OK;
+  const int sms = host::sm_count();
+  if (sms <= 0) return US_ERR_CUDA;
+  const int64_t want = (total + kThreads - 1) / kThreads, cap = (int64_t)sms * 8;
+  weighted_add_kernel<<<(int)(want < cap ? want : cap), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
   return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }
 

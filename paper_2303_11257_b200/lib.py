@@ -82,6 +82,8 @@ def _load() -> C.CDLL:
     lib.us_activation_bwd.argtypes = [C.c_int, MP, MP, F, F, MP, V]
     lib.us_activation_fwd.restype = lib.us_activation_bwd.restype = C.c_int
     lib.us_cast_fp8_multi.argtypes = [C.c_int, MP, C.POINTER(C.c_float), MP, V]
+    lib.us_weighted_add.argtypes = [C.c_int, MP, C.POINTER(C.c_float), F, MP, V]
+    lib.us_weighted_add.restype = C.c_int
     lib.us_softmax_fwd.argtypes = [MP, F, MP, V]
     lib.us_softmax_bwd.argtypes = [MP, MP, F, F, MP, V]
     lib.us_softmax_xent_fwd.argtypes = [MP, V, V, V]
@@ -261,6 +263,14 @@ def us_residual_add(skip, branch, tau, out, stream=None):
 def us_cast_fp8(src, scale, dst, stream=None):
     _check("us_cast_fp8", _lib.us_cast_fp8(C.byref(mat(src)), scale, C.byref(mat(dst)), _stream(stream)))
     return dst
+
+
+def us_weighted_add(srcs, gammas, alpha, out, stream=None):
+    n = len(srcs)
+    sm = (us_mat * n)(*[mat(t) for t in srcs])
+    gm = (C.c_float * n)(*[float(g) for g in gammas])
+    _check("us_weighted_add", _lib.us_weighted_add(n, sm, gm, alpha, C.byref(mat(out)), _stream(stream)))
+    return out
 
 
 def us_cast_fp8_multi(srcs, scales, dsts, stream=None):

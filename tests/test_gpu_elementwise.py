@@ -125,3 +125,25 @@ def test_activation_gelu_entry_equals_gelu_calls_and_unit_scale():
     with pytest.raises(L.UnitScaleError) as e:
         L.us_activation_fwd(9, z, 1.0, 1.0, a)
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("out_fmt", ["f32", "bf16", "e4m3"])
+@pytest.mark.parametrize("shape,ld", [((129, 515), None), ((64, 1024), 1040), ((3, 16), None)])
+def test_weighted_add_n(out_fmt, shape, ld):
+    L, synth = _lib()
+    fmts = ["f32", "bf16", "fp16"]
+    xs = [synth.normal(8, i, shape) for i in range(3)]
+    gammas = [1.0, 0.5, 2.0]
+    alpha = float(np.float32(sum(g * g for g in gammas) ** -0.5))
+    out = U.empty(shape[0], shape[1], out_fmt, ld)
+    L.us_weighted_add([U.to_device(x, f, ld) for x, f in zip(xs, fmts)], gammas, alpha, out)
+    # the device forms alpha * gamma_i in float32 first: mirror that rounding in the reference's coefficients
+    coefs = [float(np.float32(alpha) * np.float32(g)) for g in gammas]
+    ref = sum(c * U.values_of(x, f) for c, x, f in zip(coefs, xs, fmts))
+    U.assert_close_stored(out, ref, out_fmt, 1e-6, "weighted_add")
+    assert np.allclose(ref, O.weighted_add_n([U.values_of(x, f) for x, f in zip(xs, fmts)], gammas), rtol=1e-6, atol=1e-6)
+    if out_fmt == "f32":
+        assert abs(U.host_values(out).std() - 1) < 0.05 or shape[0] < 64
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_weighted_add([torch.zeros((4, 8), device="cuda")] * 9, [1.0] * 9, 1.0, torch.zeros((4, 8), device="cuda"))
+    assert e.value.status == 1
