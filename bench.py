@@ -48,6 +48,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--operand", default="fp8", choices=["fp8", "bf16", "fp16"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dp", action="store_true", help="token-sharded data parallelism: global beta_w and an all-reduce of the weight gradients every step (default: independent replicas)")
     ap.add_argument("--one-stream", action="store_true", help="issue the step's GEMMs on one stream (no overlap of independent launches)")
     return ap.parse_args()
 
@@ -266,7 +267,7 @@ def run_reference(args, rank: int, world: int):
 def run_ours(args, rank: int, world: int, local: int):
     import torch
 
-    from paper_2303_11257_b200 import ffn, synth
+    from paper_2303_11257_b200 import dp, ffn, synth
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
@@ -281,7 +282,9 @@ def run_ours(args, rank: int, world: int, local: int):
     host = [synth.ffn_tensors(shape, seed=1000 * rank + i) for i in range(2)]
     pinned = [[torch.from_numpy(t).pin_memory() for t in tensors] for tensors in host]
     sets = [[p.to(dev, non_blocking=True) for p in tensors] for tensors in pinned]
-    blocks = [ffn.UnitScaledFFN(T, d, f, operand=args.operand, device=dev) for _ in sets]
+    dp_on = args.dp and world > 1
+    scales = ffn.FFNScales.unit(T, d, f, dp_world=world) if dp_on else None
+    blocks = [ffn.UnitScaledFFN(T, d, f, scales=scales, operand=args.operand, device=dev) for _ in sets]
     if args.one_stream:
         for b in blocks:
             b.concurrent = False
@@ -307,6 +310,8 @@ def run_ours(args, rank: int, world: int, local: int):
     e0.record()
     for i in range(args.steps):
         graphs[i % 2].replay()
+        if dp_on:
+            dp.allreduce_weight_grads([blocks[i % 2].dW1, blocks[i % 2].dW2])
     e1.record()
     torch.cuda.synchronize()
     windows.append((w0, time.time()))
@@ -430,7 +435,7 @@ def run_ours(args, rank: int, world: int, local: int):
         "vs_baseline": None, "dtype": {"fp8": "fp8_e4m3/e5m2 (fp32 accumulate)", "bf16": "bf16", "fp16": "fp16"}[args.operand],
         "data": "synthetic",
         "config": {"workload": "ffn_bert_large fwd+bwd: T=8192 tokens (16x512), d_model=1024, d_ff=4096, tau=0.5",
-                   "operand": args.operand, "replicas": world,
+                   "operand": args.operand, "replicas": world, "weight_gradient_allreduce": dp_on,
                    "l2": "two rotating input/buffer sets, ~0.45 GB touched per step (> 126 MB L2)",
                    "launch": f"one CUDA graph of {blocks[0].launches_per_step} kernels per step, "
                              + ("GEMMs after the first on three streams" if blocks[0].concurrent else "one stream")},

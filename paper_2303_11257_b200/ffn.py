@@ -40,8 +40,12 @@ class FFNScales:
     tau: float = 0.5
 
     @staticmethod
-    def unit(T: int, d: int, f: int, tau: float = 0.5, constrained: bool = False) -> "FFNScales":
+    def unit(T: int, d: int, f: int, tau: float = 0.5, constrained: bool = False, dp_world: int = 1) -> "FFNScales":
+        """dp_world > 1: T tokens per rank of a token-sharded job; the weight-gradient factor then uses
+        the global batch T * dp_world, and the ranks' weight gradients are summed afterwards (dp.py)."""
         a1, bx1, bw = L.us_scales_linear(T, d, f, constrained)
+        if dp_world > 1:
+            bw = float(T * dp_world) ** -0.5
         a2, bx2, _ = L.us_scales_linear(T, f, d, constrained)
         ag, bg = L.us_scales_gelu(constrained)
         return FFNScales(a1, a2, bx1, bx2, bw, ag, bg, 1.0, tau)
