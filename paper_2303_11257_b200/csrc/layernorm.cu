@@ -298,7 +298,9 @@ __global__ void __launch_bounds__(kLnThreads, 2) ln_fwd16_kernel(const LnArgs a)
   }
 }
 
-template <int NCH>
+// G32: the gradient is float32 (the gradient of a layer's output often is): it is loaded at the top of the
+// iteration into float registers instead of being prefetched packed; X is still prefetched.
+template <int NCH, bool G32>
 __global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
   extern __shared__ __align__(16) float ln_smem[];                         // w[cols] as float32, then [warps][cols] for the combine
   float* w_s = ln_smem;
@@ -314,12 +316,23 @@ __global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) { sw[c][i] = 0.f; sc[c][i] = 0.f; }
   int64_t row = (int64_t)blockIdx.x * nw + warp;
-  uint4 cx[NCH], cg[NCH], nx[NCH], ng[NCH];
-  if (row < a.rows) { load_row16<NCH>(a.x, row * a.x_ld, lane, a.cols, cx); load_row16<NCH>(a.g, row * a.g_ld, lane, a.cols, cg); }
+  uint4 cx[NCH], cg[G32 ? 1 : NCH], nx[NCH], ng[G32 ? 1 : NCH];
+  if (row < a.rows) {
+    load_row16<NCH>(a.x, row * a.x_ld, lane, a.cols, cx);
+    if (!G32) load_row16<G32 ? 1 : NCH>(a.g, row * a.g_ld, lane, a.cols, cg);
+  }
   for (; row < a.rows; row += stride) {
     if (row + stride < a.rows) {
       load_row16<NCH>(a.x, (row + stride) * a.x_ld, lane, a.cols, nx);
-      load_row16<NCH>(a.g, (row + stride) * a.g_ld, lane, a.cols, ng);
+      if (!G32) load_row16<G32 ? 1 : NCH>(a.g, (row + stride) * a.g_ld, lane, a.cols, ng);
+    }
+    float gf[G32 ? NCH : 1][8];
+    if (G32) {
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        const int col = (c * 32 + lane) * 8;
+        if (col < a.cols) load_vec<8>(static_cast<const char*>(a.g) + (row * a.g_ld + col) * 4, US_F32, gf[G32 ? c : 0]);
+      }
     }
     float x[NCH][8];
 #pragma unroll
@@ -332,7 +345,12 @@ __global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
       const int col = (c * 32 + lane) * 8;
       if (col < a.cols) {
         float g[8];
-        unpack16x8(cg[c], a.g_dt, g);
+        if (G32) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) g[i] = gf[G32 ? c : 0][i];
+        } else {
+          unpack16x8(cg[G32 ? 0 : c], a.g_dt, g);
+        }
         const float4 w0 = *reinterpret_cast<const float4*>(w_s + col), w1 = *reinterpret_cast<const float4*>(w_s + col + 4);
         const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
@@ -354,7 +372,12 @@ __global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
       const int col = (c * 32 + lane) * 8;
       if (col < a.cols) {
         float g[8], d[8];
-        unpack16x8(cg[c], a.g_dt, g);
+        if (G32) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) g[i] = gf[G32 ? c : 0][i];
+        } else {
+          unpack16x8(cg[G32 ? 0 : c], a.g_dt, g);
+        }
         const float4 w0 = *reinterpret_cast<const float4*>(w_s + col), w1 = *reinterpret_cast<const float4*>(w_s + col + 4);
         const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
@@ -363,7 +386,7 @@ __global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
       }
     }
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) { cx[c] = nx[c]; cg[c] = ng[c]; }
+    for (int c = 0; c < NCH; ++c) { cx[c] = nx[c]; if (!G32) cg[G32 ? 0 : c] = ng[G32 ? 0 : c]; }
   }
   float* dst = a.partial + (size_t)blockIdx.x * 2 * a.cols;
 #pragma unroll
@@ -520,12 +543,19 @@ extern "C" us_status us_layer_norm_bwd(const us_mat* X, const us_mat* w, const u
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int nparts = grid;
   // With no rows the first kernel still runs (one CTA) and writes zero partials, so dw = dc = 0.
-  if (a.vec_ok && nch <= 4 && (a.x_dt == US_BF16 || a.x_dt == US_F16) && a.g_dt == a.x_dt) {
+  if (a.vec_ok && nch <= 4 && (a.x_dt == US_BF16 || a.x_dt == US_F16) && (a.g_dt == a.x_dt || a.g_dt == US_F32)) {
+    const bool g32 = a.g_dt == US_F32;
     nparts = ln_bwd_grid(X->rows > 0 ? X->rows : 1, kLnFastWarps, kLnFastPerSm);
     const size_t smem = (size_t)(1 + kLnFastWarps) * a.cols * sizeof(float);
-    if (nch <= 1) ln_bwd16_kernel<1><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);
-    else if (nch <= 2) ln_bwd16_kernel<2><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);
-    else ln_bwd16_kernel<4><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);
+#define US_LN_BWD16(N)                                                                             \
+  do {                                                                                            \
+    if (g32) ln_bwd16_kernel<N, true><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);                \
+    else ln_bwd16_kernel<N, false><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);                   \
+  } while (0)
+    if (nch <= 1) US_LN_BWD16(1);
+    else if (nch <= 2) US_LN_BWD16(2);
+    else US_LN_BWD16(4);
+#undef US_LN_BWD16
   } else if (nch <= 4) {
     const size_t smem = (size_t)kLnWarps * a.cols * sizeof(float);
     if (nch <= 1) ln_bwd_kernel<1><<<grid, kLnThreads, smem, st>>>(a);

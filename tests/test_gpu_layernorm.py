@@ -99,3 +99,22 @@ def test_layer_norm_errors_and_empty():
         L.us_layer_norm_bwd(big, vb, big, 0.0, 1.0, 0.5, torch.empty_like(big), torch.empty_like(vb), torch.empty_like(vb), wsb)
     assert e.value.status == 2
     L.us_layer_norm_fwd(torch.zeros((0, 16), device="cuda"), v, v, 0.0, torch.zeros((0, 16), device="cuda"))
+
+
+@pytest.mark.parametrize("rows,cols,ld", [(64, 256, None), (130, 768, 800), (257, 1024, None), (40, 512, None)])
+def test_layer_norm_backward_with_a_float32_gradient(rows, cols, ld):
+    """16-bit X with a float32 incoming gradient (the gradient of a layer's output)."""
+    L = _lib()
+    X, G, w, _ = _inputs(6, rows, cols, "bf16")
+    from paper_2303_11257_b200 import synth
+    G = synth.normal(6, 4, (rows, cols), 1.0)                      # not on the BF16 grid
+    eps, beta_wc = 1e-5, float(np.float32(rows ** -0.5))
+    dX, dw, dc = U.empty(rows, cols, "bf16", ld), torch.empty(cols, device="cuda"), torch.empty(cols, device="cuda")
+    ws = torch.empty(L.us_layer_norm_bwd_workspace_bytes(rows, cols), dtype=torch.uint8, device="cuda")
+    L.us_layer_norm_bwd(U.to_device(X, "bf16", ld), torch.from_numpy(w[0]).cuda(), U.to_device(G, "f32", ld), eps, 1.0, beta_wc,
+                        dX, dw, dc, ws)
+    rdX, rdw, rdc = O.layer_norm_bwd(X, w, G, np.float32(eps), 1.0, beta_wc)
+    scale = 1.0 / np.sqrt(X.var(axis=1).min() + eps)
+    U.assert_close_stored(dX, rdX, "bf16", 3e-5 * max(1.0, scale), "dX")
+    tol = 8 * (2e-6 * np.sqrt(rows) + 1e-6)
+    assert np.abs(dw.cpu().numpy() - rdw.reshape(-1)).max() <= tol and np.abs(dc.cpu().numpy() - rdc.reshape(-1)).max() <= tol
