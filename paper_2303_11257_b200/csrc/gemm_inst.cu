@@ -47,7 +47,7 @@ static bool make_tmap(CUtensorMap* tm, const us_mat* m, int es, int box_rows, in
     cuuint32_t box[2] = {(cuuint32_t)(box_bytes / es), (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     r = fn(tm, type, 2, m->ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
     // rank 4: (column, row, inner batch index, outer batch index); a box never spans problems
     cuuint64_t dims[4] = {(cuuint64_t)m->cols, (cuuint64_t)m->rows, (cuuint64_t)bd->nb1, (cuuint64_t)bd->nb0};
@@ -55,7 +55,7 @@ static bool make_tmap(CUtensorMap* tm, const us_mat* m, int es, int box_rows, in
     cuuint32_t box[4] = {(cuuint32_t)(box_bytes / es), (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     r = fn(tm, type, 4, m->ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   }
   return r == CUDA_SUCCESS;
 }
