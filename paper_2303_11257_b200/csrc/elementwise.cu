@@ -54,8 +54,16 @@ __device__ __forceinline__ float ew_apply(float a, float b, const EwArgs& p) {
   if (OP == kActBwd)                                                          // a = H, b = dA, c1 = beta
     return p.fn == US_FN_GELU ? gelu_grad_scaled(a, b, p.c0, p.c1) : (p.c1 * p.c0) * act_slope(p.fn, p.c0 * a) * b;
   if (OP == kCast) return p.c0 * a;                                   // scale * x, then the store rounds
-  if (OP == kGeluFwd) return gelu_scaled(a, p.c0, p.c1);              // c0 = s_in, c1 = alpha
-  if (OP == kGeluBwd) return gelu_grad_scaled(a, b, p.c0, p.c1);      // a = H, b = dA, c1 = beta
+  if (OP == kGeluFwd) {                                               // c0 = s_in, c1 = alpha; same arithmetic as the pair form
+    float y0, y1;
+    gelu_scaled2<false>(pack2(a, a), fabsf(p.c0) * (1.0f / kTailRange), p.c1 * p.c0, y0, y1);
+    return y0;
+  }
+  if (OP == kGeluBwd) {                                               // a = H, b = dA, c1 = beta
+    float y0, y1;
+    unpack2(gelu_grad_scaled2(pack2(a, a), pack2(b, b), splat2(p.c0), splat2(p.c1 * p.c0)), y0, y1);
+    return y0;
+  }
   return fmaf(p.c0, a, p.c1 * b);                                     // c0 = sqrt(1-tau), c1 = sqrt(tau)
 }
 
@@ -72,8 +80,19 @@ __global__ void __launch_bounds__(kThreads) ew_kernel(const EwArgs p) {
       float a[kVec], b[kVec], o[kVec];
       load_vec<kVec>(static_cast<const char*>(p.in0.ptr) + i0 * dtype_size(p.in0.dt), p.in0.dt, a);
       if (kTwoInputs) load_vec<kVec>(static_cast<const char*>(p.in1.ptr) + i1 * dtype_size(p.in1.dt), p.in1.dt, b);
+      if (OP == kGeluFwd) {                          // two values per instruction (packed float32 arithmetic)
+        const float k = fabsf(p.c0) * (1.0f / kTailRange), oi = p.c1 * p.c0;
 #pragma unroll
-      for (int i = 0; i < kVec; ++i) o[i] = ew_apply<OP>(a[i], kTwoInputs ? b[i] : 0.f, p);
+        for (int i = 0; i < kVec; i += 2) gelu_scaled2<false>(pack2(a[i], a[i + 1]), k, oi, o[i], o[i + 1]);
+      } else if (OP == kGeluBwd) {
+        const f32x2 in2 = splat2(p.c0), os2 = splat2(p.c1 * p.c0);
+#pragma unroll
+        for (int i = 0; i < kVec; i += 2)
+          unpack2(gelu_grad_scaled2(pack2(a[i], a[i + 1]), pack2(b[i], b[i + 1]), in2, os2), o[i], o[i + 1]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < kVec; ++i) o[i] = ew_apply<OP>(a[i], kTwoInputs ? b[i] : 0.f, p);
+      }
       store_vec<kVec>(static_cast<char*>(p.out.ptr) + io * dtype_size(p.out.dt), p.out.dt, o);
     } else {
       const int n = (int)min((int64_t)kVec, p.cols - col);
@@ -324,6 +343,7 @@ extern "C" us_status us_activation_fwd(us_fn fn, const us_mat* H, float s_in, fl
   if (fn < US_FN_GELU || fn > US_FN_SIGMOID) return US_ERR_INVALID_ARG;
   us_status s = check_ew(H, nullptr, A);
   if (s != US_OK) return s;
+  if (fn == US_FN_GELU) return ew_launch<kGeluFwd>(H, nullptr, A, s_in, alpha, stream);
   return ew_launch<kActFwd>(H, nullptr, A, s_in, alpha, stream, fn);
 }
 
@@ -332,6 +352,7 @@ extern "C" us_status us_activation_bwd(us_fn fn, const us_mat* H, const us_mat* 
   if (fn < US_FN_GELU || fn > US_FN_SIGMOID || !dA) return US_ERR_INVALID_ARG;
   us_status s = check_ew(H, dA, dH);
   if (s != US_OK) return s;
+  if (fn == US_FN_GELU) return ew_launch<kGeluBwd>(H, dA, dH, s_in, beta, stream);
   return ew_launch<kActBwd>(H, dA, dH, s_in, beta, stream, fn);
 }
 
