@@ -52,4 +52,22 @@ __device__ __forceinline__ void store8(void* base, int dt, int64_t row_off, int 
   }
 }
 
+// ---- rows of 16-bit elements kept packed in registers (one 128-bit load per lane and chunk of 8)
+__device__ __forceinline__ void unpack16x8(const uint4& r, int dt, float (&v)[8]) {
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 f = dt == US_BF16 ? unpack_bf16x2(w[j]) : unpack_f16x2(w[j]);
+    v[2 * j] = f.x; v[2 * j + 1] = f.y;
+  }
+}
+template <int NCH>
+__device__ __forceinline__ void load_row16(const void* base, int64_t row_off, int lane, int cols, uint4 (&d)[NCH]) {
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    d[c] = col < cols ? __ldg(reinterpret_cast<const uint4*>(static_cast<const char*>(base) + (row_off + col) * 2))
+                      : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
 }  // namespace us

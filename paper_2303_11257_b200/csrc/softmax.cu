@@ -132,6 +132,97 @@ __global__ void __launch_bounds__(kSmThreads) softmax_bwd_kernel(const SmArgs a)
   }
 }
 
+// ---------------------------------------------------------------- 16-bit inputs, rows of at most 1024 elements
+// Persistent warps: each walks rows grid-stride and fetches its next row, still packed, before working on
+// the current one, so that a warp always has a row in flight.  Padding chunks (beyond the row) read as zero
+// and are masked out of the maximum and the sums.
+template <int NCH>
+__global__ void __launch_bounds__(kSmThreads, 2) softmax_fwd16_kernel(const SmArgs a) {
+  const int lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const int64_t stride = (int64_t)gridDim.x * nw;
+  int64_t row = (int64_t)blockIdx.x * nw + (threadIdx.x >> 5);
+  uint4 cur[NCH], nxt[NCH];
+  if (row < a.rows) load_row16<NCH>(a.in0, row * a.in0_ld, lane, a.cols, cur);
+  for (; row < a.rows; row += stride) {
+    if (row + stride < a.rows) load_row16<NCH>(a.in0, (row + stride) * a.in0_ld, lane, a.cols, nxt);
+    float x[NCH][8];
+    float m = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      unpack16x8(cur[c], a.in0_dt, x[c]);
+      if ((c * 32 + lane) * 8 < a.cols) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) m = fmaxf(m, x[c][i]);
+      }
+    }
+    m = warp_max(m);
+    const float mb = m * kLog2e;
+    float sum = 0.f;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      if ((c * 32 + lane) * 8 < a.cols) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { x[c][i] = ex2_approx(fmaf(x[c][i], kLog2e, -mb)); sum += x[c][i]; }
+      }
+    }
+    sum = warp_sum(sum);
+    const float inv = a.alpha / sum;
+    const int64_t out_off = row * a.out_ld;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const int col = (c * 32 + lane) * 8;
+      if (col < a.cols) {
+        float t[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t[i] = x[c][i] * inv;
+        store8(a.out, a.out_dt, out_off, col, a.cols, true, t);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) cur[c] = nxt[c];
+  }
+}
+
+// P and dP both 16-bit and of one format.
+template <int NCH>
+__global__ void __launch_bounds__(kSmThreads, 2) softmax_bwd16_kernel(const SmArgs a) {
+  const int lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const int64_t stride = (int64_t)gridDim.x * nw;
+  const float inv_alpha = 1.0f / a.alpha;
+  int64_t row = (int64_t)blockIdx.x * nw + (threadIdx.x >> 5);
+  uint4 cp[NCH], cg[NCH], np_[NCH], ng[NCH];
+  if (row < a.rows) { load_row16<NCH>(a.in0, row * a.in0_ld, lane, a.cols, cp); load_row16<NCH>(a.in1, row * a.in1_ld, lane, a.cols, cg); }
+  for (; row < a.rows; row += stride) {
+    if (row + stride < a.rows) {
+      load_row16<NCH>(a.in0, (row + stride) * a.in0_ld, lane, a.cols, np_);
+      load_row16<NCH>(a.in1, (row + stride) * a.in1_ld, lane, a.cols, ng);
+    }
+    float pt[NCH][8], g[NCH][8];
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      unpack16x8(cp[c], a.in0_dt, pt[c]);
+      unpack16x8(cg[c], a.in1_dt, g[c]);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { pt[c][i] *= inv_alpha; dot = fmaf(pt[c][i], g[c][i], dot); }   // padding: 0 * 0
+    }
+    dot = warp_sum(dot);
+    const int64_t out_off = row * a.out_ld;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const int col = (c * 32 + lane) * 8;
+      if (col < a.cols) {
+        float t[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t[i] = a.beta * pt[c][i] * (g[c][i] - dot);
+        store8(a.out, a.out_dt, out_off, col, a.cols, true, t);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) { cp[c] = np_[c]; cg[c] = ng[c]; }
+  }
+}
+
 // ---------------------------------------------------------------- softmax cross-entropy
 // softmax_xent(x, t) = log softmax(x)_t (table row "softmax_xent": alpha = 1, beta = s / sqrt(s - 1)).
 // One warp per row; the row is read twice (maximum, then sum of exponentials) from global memory /
@@ -213,6 +304,22 @@ static us_status launch_softmax(const SmArgs& a, cudaStream_t st) {
   if (grid64 > 0x7fffffff) return US_ERR_INVALID_ARG;
   const int grid = (int)grid64;
   const int nch = (a.cols + 255) / 256;
+  const bool in16 = a.in0_dt == US_BF16 || a.in0_dt == US_F16;
+  if (a.vec_ok && nch <= 4 && in16 && (!BWD || a.in1_dt == a.in0_dt)) {
+    const int sms = host::sm_count();
+    if (sms <= 0) return US_ERR_CUDA;
+    const int pgrid = grid < 2 * sms ? grid : 2 * sms;        // two resident CTAs per SM, warps walk the rows
+#define US_SM16(N)                                                                   \
+  do {                                                                               \
+    if (BWD) softmax_bwd16_kernel<N><<<pgrid, kSmThreads, 0, st>>>(a);               \
+    else softmax_fwd16_kernel<N><<<pgrid, kSmThreads, 0, st>>>(a);                   \
+  } while (0)
+    if (nch <= 1) US_SM16(1);
+    else if (nch <= 2) US_SM16(2);
+    else US_SM16(4);
+#undef US_SM16
+    return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
+  }
 #define US_SM_LAUNCH(N)                                                          \
   do {                                                                           \
     if (BWD) softmax_bwd_kernel<N><<<grid, kSmThreads, 0, st>>>(a);              \
