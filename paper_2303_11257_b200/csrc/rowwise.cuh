@@ -70,4 +70,21 @@ __device__ __forceinline__ void load_row16(const void* base, int64_t row_off, in
                       : make_uint4(0u, 0u, 0u, 0u);
   }
 }
+// The same for rows of FP8 codes: one 64-bit load per lane and chunk of 8.
+__device__ __forceinline__ void unpack8x8(const uint2& r, int dt, float (&v)[8]) {
+  const uint32_t w[2] = {r.x, r.y};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 f = unpack_fp8x2((uint16_t)(w[j >> 1] >> (16 * (j & 1))), dt == US_E5M2);
+    v[2 * j] = f.x; v[2 * j + 1] = f.y;
+  }
+}
+template <int NCH>
+__device__ __forceinline__ void load_row8(const void* base, int64_t row_off, int lane, int cols, uint2 (&d)[NCH]) {
+#pragma unroll
+  for (int c = 0; c < NCH; ++c) {
+    const int col = (c * 32 + lane) * 8;
+    d[c] = col < cols ? __ldg(reinterpret_cast<const uint2*>(static_cast<const char*>(base) + row_off + col)) : make_uint2(0u, 0u);
+  }
+}
 }  // namespace us

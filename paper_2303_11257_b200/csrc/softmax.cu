@@ -183,25 +183,32 @@ __global__ void __launch_bounds__(kSmThreads, 2) softmax_fwd16_kernel(const SmAr
   }
 }
 
-// P and dP both 16-bit and of one format.
-template <int NCH>
+// dP 16-bit; P 16-bit of the same format, or (P8) FP8 codes as stored for an FP8 matmul.
+template <int NCH, bool P8>
 __global__ void __launch_bounds__(kSmThreads, 2) softmax_bwd16_kernel(const SmArgs a) {
   const int lane = threadIdx.x & 31, nw = blockDim.x >> 5;
   const int64_t stride = (int64_t)gridDim.x * nw;
   const float inv_alpha = 1.0f / a.alpha;
   int64_t row = (int64_t)blockIdx.x * nw + (threadIdx.x >> 5);
-  uint4 cp[NCH], cg[NCH], np_[NCH], ng[NCH];
-  if (row < a.rows) { load_row16<NCH>(a.in0, row * a.in0_ld, lane, a.cols, cp); load_row16<NCH>(a.in1, row * a.in1_ld, lane, a.cols, cg); }
+  uint4 cp[P8 ? 1 : NCH], cg[NCH], np_[P8 ? 1 : NCH], ng[NCH];
+  uint2 cp8[P8 ? NCH : 1], np8[P8 ? NCH : 1];
+  if (row < a.rows) {
+    if (P8) load_row8<P8 ? NCH : 1>(a.in0, row * a.in0_ld, lane, a.cols, cp8);
+    else load_row16<P8 ? 1 : NCH>(a.in0, row * a.in0_ld, lane, a.cols, cp);
+    load_row16<NCH>(a.in1, row * a.in1_ld, lane, a.cols, cg);
+  }
   for (; row < a.rows; row += stride) {
     if (row + stride < a.rows) {
-      load_row16<NCH>(a.in0, (row + stride) * a.in0_ld, lane, a.cols, np_);
+      if (P8) load_row8<P8 ? NCH : 1>(a.in0, (row + stride) * a.in0_ld, lane, a.cols, np8);
+      else load_row16<P8 ? 1 : NCH>(a.in0, (row + stride) * a.in0_ld, lane, a.cols, np_);
       load_row16<NCH>(a.in1, (row + stride) * a.in1_ld, lane, a.cols, ng);
     }
     float pt[NCH][8], g[NCH][8];
     float dot = 0.f;
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
-      unpack16x8(cp[c], a.in0_dt, pt[c]);
+      if (P8) unpack8x8(cp8[P8 ? c : 0], a.in0_dt, pt[c]);
+      else unpack16x8(cp[P8 ? 0 : c], a.in0_dt, pt[c]);
       unpack16x8(cg[c], a.in1_dt, g[c]);
 #pragma unroll
       for (int i = 0; i < 8; ++i) { pt[c][i] *= inv_alpha; dot = fmaf(pt[c][i], g[c][i], dot); }   // padding: 0 * 0
@@ -219,7 +226,11 @@ __global__ void __launch_bounds__(kSmThreads, 2) softmax_bwd16_kernel(const SmAr
       }
     }
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) { cp[c] = np_[c]; cg[c] = ng[c]; }
+    for (int c = 0; c < NCH; ++c) {
+      if (P8) cp8[P8 ? c : 0] = np8[P8 ? c : 0];
+      else cp[P8 ? 0 : c] = np_[P8 ? 0 : c];
+      cg[c] = ng[c];
+    }
   }
 }
 
@@ -305,13 +316,15 @@ static us_status launch_softmax(const SmArgs& a, cudaStream_t st) {
   const int grid = (int)grid64;
   const int nch = (a.cols + 255) / 256;
   const bool in16 = a.in0_dt == US_BF16 || a.in0_dt == US_F16;
-  if (a.vec_ok && nch <= 4 && in16 && (!BWD || a.in1_dt == a.in0_dt)) {
+  const bool p8 = BWD && (a.in0_dt == US_E4M3 || a.in0_dt == US_E5M2) && (a.in1_dt == US_BF16 || a.in1_dt == US_F16);
+  if (a.vec_ok && nch <= 4 && ((in16 && (!BWD || a.in1_dt == a.in0_dt)) || p8)) {
     const int sms = host::sm_count();
     if (sms <= 0) return US_ERR_CUDA;
     const int pgrid = grid < 2 * sms ? grid : 2 * sms;        // two resident CTAs per SM, warps walk the rows
 #define US_SM16(N)                                                                   \
   do {                                                                               \
-    if (BWD) softmax_bwd16_kernel<N><<<pgrid, kSmThreads, 0, st>>>(a);               \
+    if (BWD && p8) softmax_bwd16_kernel<N, true><<<pgrid, kSmThreads, 0, st>>>(a);   \
+    else if (BWD) softmax_bwd16_kernel<N, false><<<pgrid, kSmThreads, 0, st>>>(a);   \
     else softmax_fwd16_kernel<N><<<pgrid, kSmThreads, 0, st>>>(a);                   \
   } while (0)
     if (nch <= 1) US_SM16(1);
