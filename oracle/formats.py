@@ -176,3 +176,24 @@ def snr(x, fmt: Format) -> float:
     x = np.asarray(x, dtype=np.float64)
     err = quantise(x, fmt) - x
     return float(np.mean(x * x) / np.mean(err * err))
+
+
+def exponent_histogram(x, exp_lo: int, nbins: int) -> np.ndarray:
+    """Counts of floor(log2 |x|) over the samples (appendix "Histograms of tensor-scaling within BERT":
+    the figures plot exactly this for activations, weights and gradients).
+
+    Returns nbins + 2 counts: [0] everything below 2^exp_lo (zeros included), [1 + k] the values with
+    2^(exp_lo + k) <= |x| < 2^(exp_lo + k + 1), [nbins + 1] everything at or above 2^(exp_lo + nbins),
+    infinities and NaNs."""
+    a = np.abs(np.asarray(x, dtype=np.float64)).ravel()
+    out = np.zeros(nbins + 2, dtype=np.int64)
+    finite = np.isfinite(a)
+    out[nbins + 1] += int((~finite).sum())
+    a = a[finite]
+    lo, hi = 2.0 ** exp_lo, 2.0 ** (exp_lo + nbins)
+    out[0] += int((a < lo).sum())
+    out[nbins + 1] += int((a >= hi).sum())
+    mid = a[(a >= lo) & (a < hi)]
+    _, e = np.frexp(mid)                       # mid = m * 2^e with 0.5 <= m < 1, so floor(log2 mid) = e - 1
+    np.add.at(out, 1 + (e - 1 - exp_lo), 1)
+    return out

@@ -187,3 +187,22 @@ def test_folded_normal_mass_pin():
     from scipy import special
     mass = special.erf(2 / np.sqrt(2)) - special.erf(2.0 ** -4 / np.sqrt(2))
     assert abs(mass - GOLD["folded_normal_mass"]) < 0.01
+
+
+def test_exponent_histogram_bins_by_floor_log2():
+    x = np.array([0.0, -0.0, 1.0, -1.0, 1.5, 2.0, 3.999, 4.0, 0.5, 0.49, 2.0 ** -10, 2.0 ** 10, np.inf, np.nan, -7.0])
+    h = F.exponent_histogram(x, -2, 5)          # bins for exponents -2 .. 2
+    assert h.sum() == x.size
+    #        below(<2^-2)  e=-2  e=-1  e=0  e=1  e=2  above
+    assert h.tolist() == [3, 1, 1, 3, 2, 2, 3]      # 0.49 is in [2^-2, 2^-1), 0.5 in [2^-1, 1)
+    # brute force with math.log2 on a random sample
+    rng = np.random.default_rng(0)
+    y = rng.standard_normal(5000) * 3
+    ref = np.zeros(12, dtype=np.int64)
+    import math
+    for v in y:
+        e = math.floor(math.log2(abs(v)))
+        ref[0 if e < -6 else 11 if e >= 4 else 1 + e + 6] += 1
+    assert np.array_equal(F.exponent_histogram(y, -6, 10), ref)
+    # a unit-normal tensor has most of its mass in the exponents -3 .. 1 (figure of the appendix: narrow histogram)
+    assert F.exponent_histogram(rng.standard_normal(100000), -3, 5)[1:6].sum() > 0.9 * 100000
