@@ -289,6 +289,25 @@ us_status us_layer_norm_bwd(const us_mat* X, const us_mat* w, const us_mat* G, f
                             float beta_wc, const us_mat* dX, const us_mat* dw, const us_mat* dc, void* ws,
                             size_t ws_bytes, void* stream);
 
+/* ------------------------------------------------------------ quantisation diagnostics
+ *
+ * us_quant_stats: for v = scale * src (one float32 multiply per element) and a storage format fmt
+ * (E4M3 / E5M2 saturating, BF16 / F16 IEEE), in one pass:
+ *   sums[0] = sum v^2,  sums[1] = sum (q_fmt(v) - v)^2        (double; their ratio is the signal-to-noise
+ *             ratio of section "Floating-point formats for deep learning", paragraph "Quantisation error")
+ *   hist[0]         count of |v| < 2^exp_lo (zeros included)
+ *   hist[1 + k]     count of 2^(exp_lo + k) <= |v| < 2^(exp_lo + k + 1),  k = 0 .. nbins - 1
+ *   hist[nbins + 1] count of |v| >= 2^(exp_lo + nbins), infinities and NaNs
+ *             (the histograms of floor(log2 |x|) of appendix "Histograms of tensor-scaling within BERT")
+ * src: F32 / BF16 / F16, any ld >= cols.  1 <= nbins <= 64, -126 <= exp_lo, exp_lo + nbins <= 128.
+ * sums (2 doubles) and hist (nbins + 2 64-bit counts) are device arrays; ws is a device workspace of
+ * us_quant_stats_workspace_bytes() bytes owned by the caller (US_ERR_WORKSPACE if smaller).  Sums are
+ * formed in a fixed order without atomics on global memory: repeated calls give identical results.
+ */
+size_t us_quant_stats_workspace_bytes(void);
+us_status us_quant_stats(const us_mat* src, float scale, us_dtype fmt, int exp_lo, int nbins, double* sums,
+                         unsigned long long* hist, void* ws, size_t ws_bytes, void* stream);
+
 /* ---------------------------------------------------------------- host helpers
  *
  * us_scales_linear: unit-scaling factors of matmul(X[b x m], W[m x n]).

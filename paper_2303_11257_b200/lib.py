@@ -94,6 +94,10 @@ def _load() -> C.CDLL:
     lib.us_layer_norm_fwd.restype = lib.us_layer_norm_bwd.restype = C.c_int
     lib.us_layer_norm_bwd_workspace_bytes.argtypes = [C.c_int64, C.c_int64]
     lib.us_layer_norm_bwd_workspace_bytes.restype = SZ
+    lib.us_quant_stats_workspace_bytes.argtypes = []
+    lib.us_quant_stats_workspace_bytes.restype = SZ
+    lib.us_quant_stats.argtypes = [MP, F, C.c_int, C.c_int, C.c_int, V, V, V, SZ, V]
+    lib.us_quant_stats.restype = C.c_int
     for name in ("us_gelu_fwd", "us_gelu_bwd", "us_residual_add", "us_cast_fp8", "us_cast_fp8_multi", "us_softmax_fwd", "us_softmax_bwd"):
         getattr(lib, name).restype = C.c_int
     FP = C.POINTER(C.c_float)
@@ -306,6 +310,18 @@ def us_softmax_xent_bwd(X, targets, g, beta, dX, stream=None):
     _check("us_softmax_xent_bwd", _lib.us_softmax_xent_bwd(C.byref(mat(X)), targets.data_ptr(), g.data_ptr() if g is not None else None,
                                                            beta, C.byref(mat(dX)), _stream(stream)))
     return dX
+
+
+def us_quant_stats(src, scale, fmt, exp_lo, nbins, stream=None):
+    """Returns (snr, sum v^2, sum err^2, hist) with hist a list of nbins + 2 counts; fmt: a torch dtype.
+    Allocates its small outputs and the workspace with torch and synchronises to read them back."""
+    sums = torch.empty(2, dtype=torch.float64, device=src.device)
+    hist = torch.empty(nbins + 2, dtype=torch.int64, device=src.device)
+    ws = torch.empty(int(_lib.us_quant_stats_workspace_bytes()), dtype=torch.uint8, device=src.device)
+    _check("us_quant_stats", _lib.us_quant_stats(C.byref(mat(src)), scale, _TORCH_DTYPES[fmt], exp_lo, nbins, sums.data_ptr(),
+                                                 hist.data_ptr(), ws.data_ptr(), ws.numel(), _stream(stream)))
+    s = sums.cpu().tolist()
+    return (s[0] / s[1] if s[1] > 0 else float("inf")), s[0], s[1], hist.cpu().tolist()
 
 
 def _vec(t: torch.Tensor) -> us_mat:
