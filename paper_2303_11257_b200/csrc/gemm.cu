@@ -41,6 +41,7 @@ static us_status linear(Op op, const us_mat* A, const us_mat* B, float scale, co
   p.scale = scale;
   p.out = out->ptr; p.out_dt = out->dtype; p.out_ld = out->ld;
   p.out_coef = 1.f;
+  p.wait_limit = kWaitLimit;
   if (ep) {
     if (ep->act < US_ACT_NONE || ep->act > US_ACT_GELU_GRAD) return US_ERR_INVALID_ARG;
     p.act = ep->act; p.act_in = ep->act_in_scale; p.act_out = ep->act_out_scale;

@@ -71,7 +71,8 @@ static us_status launch(const us_mat* A, const us_mat* B, const GemmParams& p, c
   // epilogue boxes: 32 rows x 128 bytes; unused maps alias the output's so that every parameter is valid
   if (!make_tmap(&t_out, em.out, dtype_size(em.out->dtype), 32, EW == 16 ? 64 : 128, b4, b4 ? bd->out : nullptr)) return US_ERR_CUDA;
   t_aux = t_out; t_skip = t_out;
-  if (EPI != kEpiLegacy && em.aux && !make_tmap(&t_aux, em.aux, dtype_size(em.aux->dtype), 32)) return US_ERR_CUDA;
+  // the 16-warp GELU-gradient epilogue reads the stored pre-activation as 32-row x 64-byte boxes (one per 32-column slice)
+  if (EPI != kEpiLegacy && em.aux && !make_tmap(&t_aux, em.aux, dtype_size(em.aux->dtype), 32, (EW == 16 && EPI == kEpiGeluGrad) ? 64 : 128)) return US_ERR_CUDA;
   if (EPI != kEpiLegacy && em.skip && !make_tmap(&t_skip, em.skip, dtype_size(em.skip->dtype), 32)) return US_ERR_CUDA;
   auto kern = gemm_kernel<ES, A_MN, B_MN, BN, CG, EPI, EW, BATCHED>;
   constexpr int smem = GemmSmem<BN, CG, EW>::kTotal;

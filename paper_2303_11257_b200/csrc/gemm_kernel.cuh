@@ -60,6 +60,8 @@ struct GemmParams {
   void* aux; int aux_dt; int64_t aux_ld;
   const void* skip; int skip_dt; int64_t skip_ld; float skip_coef, out_coef;
   unsigned int* status;
+  uint32_t wait_limit;                      // polls a bounded wait makes before it gives up (kWaitLimit unless a test shortens it)
+  int no_loads;                             // test hook: the producer issues no operand loads, so that the waits run out
 };
 
 constexpr int kBM = 128;                 // tile rows = TMEM lanes
@@ -126,8 +128,8 @@ __device__ __forceinline__ void tile_batch(const GemmParams& p, int tile, int& b
 // (Each attempt already suspends the thread in hardware for a while, so polling costs few issue
 // slots: pausing between attempts made no measurable difference.)
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                             unsigned int* status) {
-  for (uint32_t it = 0; it < kWaitLimit; ++it) {
+                                             unsigned int* status, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 63u && *abort_flag) return false;
   }
@@ -278,11 +280,13 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
     while (tile < c.num_tiles && tile_cols(tile) >= p.N) tile += c.num_groups;
     return tile;
   };
+  bool in_pending = false;                                   // an input box load has been issued and not yet waited for
   auto issue_in = [&](int col, int row0) {
     if (lane == 0) {
       ptx::mbar_expect_tx(c.in_bar, 4096);
       ptx::tma_load_2d(buf_in, tm_in, c.in_bar, col, row0);      // fused inputs exist for single problems only
     }
+    in_pending = true;
   };
   // This warp is done reading accumulator a: its values are in registers, so the buffer is handed
   // back to the MMA warp before the arithmetic and the stores of the last slice, not after them.
@@ -304,7 +308,7 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
   for (int tile = c.group; ok && tile < c.num_tiles; tile += c.num_groups, ++local) {
     const uint32_t acc = local & 1u, acc_phase = (local >> 1) & 1u;
     const int row0 = tile_rows(tile), n_w = tile_cols(tile);
-    ok = wait_bounded(c.acc_full0 + 8u * acc, acc_phase, c.abort_flag, p.status);
+    ok = wait_bounded(c.acc_full0 + 8u * acc, acc_phase, c.abort_flag, p.status, p.wait_limit);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) break;
     ptx::tc_fence_after_sync();
@@ -322,10 +326,11 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
         if (in_kind) {
           const int off = (32 * sl) & (in_box_cols - 1);       // box widths are powers of two
           if (off == 0) {
-            ok = wait_bounded(c.in_bar, in_phase, c.abort_flag, p.status);
+            ok = wait_bounded(c.in_bar, in_phase, c.abort_flag, p.status, p.wait_limit);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             in_phase ^= 1u;
+            in_pending = false;
           }
           const uint32_t cb = (uint32_t)(off * in_es) >> 4;
           const int nchunk = 2 * in_es;                      // 32 values
@@ -456,6 +461,185 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
     if (!ok) break;
     if (!released) release_acc(acc);                           // tile without columns for this warp
   }
+  // Leaving early (a wait ran out somewhere in the CTA): an input box may still be in flight; let it
+  // land before the CTA may give up its shared memory.
+  if (in_kind && in_pending && lane == 0)
+    for (uint32_t it = 0; it < p.wait_limit && !ptx::mbar_try_wait(c.in_bar, in_phase); ++it) {}
+  if (lane == 0) ptx::bulk_wait_group_read<0>();             // stores have left shared memory before the CTA may exit
+  __syncwarp();
+}
+
+// Epilogue of the two GELU kinds with an FP8 output, run by sixteen warps: warp (quarter q, part)
+// owns the 32 rows of TMEM lane quarter q and 64 columns of the tile, as two 32-column slices.
+// The per-tile chain of one warp is kept short, because with K = d_model the main loop of a tile
+// lasts only a few thousand cycles:
+//   * the second slice is loaded from tensor memory while the first is being worked on, and the
+//     accumulator is handed back to the MMA warp as soon as both slices are in registers;
+//   * the coordinates of the next tile are computed while the first load is in flight;
+//   * GELU gradient: the stored pre-activation arrives as two 32-row x 64-byte boxes (one per
+//     slice), each refilled for the next tile right after its slice has been read, so that a
+//     load has a slice's worth of arithmetic and the tile change-over to land;
+//   * one proxy fence and one bulk group per tile for all stores of the warp.
+// Staging per warp (6 KB): GELU: [0, 4096) kept pre-activation, 32 rows x 128 bytes (128-byte
+// swizzle), [4096, 6144) output; GELU gradient: [0, 2048) and [2048, 4096) the input boxes,
+// [4096, 6144) output; 64-byte rows use the 64-byte swizzle: 16-byte chunk c of row r sits at
+// chunk c ^ ((r >> 1) & 3).
+template <int BN, int CG, int EPI, bool OUT_E5, bool AUX_BF16>
+__device__ __forceinline__ void epilogue_act16(const GemmParams& p, const CUtensorMap* tm_out, const CUtensorMap* tm_aux,
+                                               const EpiCtx& c, uint32_t in_bar1) {
+  static_assert(EPI == kEpiGelu || EPI == kEpiGeluGrad, "GELU kinds only");
+  constexpr bool kIn = EPI == kEpiGeluGrad;
+  const int q = c.warp & 3, part = (c.warp - 2) >> 2;
+  if (part >= BN / 64) return;
+  const int lane = c.lane;
+  const bool aux_out = EPI == kEpiGelu && p.aux != nullptr;
+  const uint32_t buf_aux = c.buf0, buf_out = c.buf0 + 4096u;
+  const uint32_t row128 = (uint32_t)lane * 128u, sw128 = (uint32_t)(lane & 7);
+  const uint32_t row64 = (uint32_t)lane * 64u, sw64 = (uint32_t)((lane >> 1) & 3);
+  const f32x2 scale2 = splat2(p.scale), in2 = splat2(p.act_in), os2 = splat2(p.act_out * p.act_in);
+  const float tail_k = fabsf(p.act_in) * (1.0f / kTailRange), act_oi = p.act_out * p.act_in;
+
+  auto coords = [&](int tile, int& row0, int& n_w) {
+    int tm, tn;
+    tile_mn(p, tile, tm, tn);
+    row0 = tm * (kBM * CG) + c.rank * kBM + q * 32;
+    n_w = tn * BN + part * 64;
+  };
+  auto issue_in = [&](int half, int n_w, int row0) {          // lane 0 only; a box wholly outside the matrix reads zeros
+    const uint32_t bar = half ? in_bar1 : c.in_bar;
+    ptx::mbar_expect_tx(bar, 2048);
+    ptx::tma_load_2d(buf_aux + 2048u * half, tm_aux, bar, n_w + 32 * half, row0);
+  };
+  auto release_acc = [&](uint32_t a) {
+    ptx::tc_fence_before_sync();
+    __syncwarp();
+    if (lane == 0) {
+      if (CG == 2) ptx::mbar_arrive_cluster(ptx::in_even_cta(c.acc_empty0 + 8u * a));
+      else ptx::mbar_arrive(c.acc_empty0 + 8u * a);
+    }
+  };
+  // One 32-column slice: scale, (kept pre-activation,) activation, rounding, staging stores.
+  auto slice = [&](const uint32_t (&r)[32], int s) {
+    uint32_t held[2];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      f32x2 x[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        x[k] = mul2(pack2(__uint_as_float(r[8 * g + 2 * k]), __uint_as_float(r[8 * g + 2 * k + 1])), scale2);
+      float y[8];
+      if (EPI == kEpiGelu) {
+        if (aux_out) {
+          uint32_t w[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            float a, b;
+            unpack2(x[k], a, b);
+            w[k] = AUX_BF16 ? pack_bf16x2(a, b) : pack_f16x2(a, b);
+          }
+          ptx::sts128(buf_aux + row128 + ((((uint32_t)(4 * s + g)) ^ sw128) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) gelu_scaled2<true>(x[k], tail_k, act_oi, y[2 * k], y[2 * k + 1]);
+      } else {
+        const uint4 raw = ptx::lds128(buf_aux + 2048u * s + row64 + ((((uint32_t)g) ^ sw64) << 4));
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float2 h = AUX_BF16 ? unpack_bf16x2(w[k]) : unpack_f16x2(w[k]);
+          unpack2(gelu_grad_scaled2(pack2(h.x, h.y), x[k], in2, os2), y[2 * k], y[2 * k + 1]);
+        }
+      }
+      const uint32_t lo = cvt_fp8x4<OUT_E5>(y[0], y[1], y[2], y[3]);
+      const uint32_t hi = cvt_fp8x4<OUT_E5>(y[4], y[5], y[6], y[7]);
+      if ((g & 1) == 0) {
+        held[0] = lo; held[1] = hi;
+      } else {
+        ptx::sts128(buf_out + row64 + ((((uint32_t)(2 * s + (g >> 1))) ^ sw64) << 4), make_uint4(held[0], held[1], lo, hi));
+      }
+    }
+  };
+
+  int tile = c.group, row0 = 0, n_w = 0;
+  bool pending[2] = {false, false};                          // an input box load is in flight
+  if (tile < c.num_tiles) {
+    coords(tile, row0, n_w);
+    if (kIn) {
+      if (lane == 0) { issue_in(0, n_w, row0); issue_in(1, n_w, row0); }
+      pending[0] = pending[1] = true;
+    }
+  }
+  uint32_t local = 0, ph0 = 0, ph1 = 0;                      // parities of the two input barriers
+  bool ok = true;
+  for (; tile < c.num_tiles; ++local) {
+    const uint32_t acc = local & 1u, acc_phase = (local >> 1) & 1u;
+    ok = wait_bounded(c.acc_full0 + 8u * acc, acc_phase, c.abort_flag, p.status, p.wait_limit);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) break;
+    ptx::tc_fence_after_sync();
+    const uint32_t t_row = c.tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN + part * 64;
+    const bool active = n_w < p.N;                            // warp-uniform
+    uint32_t r0[32], r1[32];
+    if (active) ptx::tmem_ld_32x32_issue(t_row, r0);
+    const int next = tile + c.num_groups;
+    int next_row0 = 0, next_n_w = 0;
+    if (next < c.num_tiles) coords(next, next_row0, next_n_w);
+    if (active) {
+      if (lane == 0) ptx::bulk_wait_group_read<0>();          // the previous tile's stores have read the staging boxes
+      __syncwarp();
+      ptx::tmem_ld_fence(r0);
+      ptx::tmem_ld_32x32_issue(t_row + 32, r1);
+    }
+    if (kIn) {
+      ok = wait_bounded(c.in_bar, ph0, c.abort_flag, p.status, p.wait_limit);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      pending[0] = false;
+      ph0 ^= 1u;
+    }
+    if (active) slice(r0, 0);
+    if (kIn) {
+      __syncwarp();                                           // every lane has read the first input box
+      if (next < c.num_tiles) {
+        if (lane == 0) issue_in(0, next_n_w, next_row0);
+        pending[0] = true;
+      }
+    }
+    if (active) ptx::tmem_ld_fence(r1);
+    release_acc(acc);
+    if (kIn) {
+      ok = wait_bounded(in_bar1, ph1, c.abort_flag, p.status, p.wait_limit);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      pending[1] = false;
+      ph1 ^= 1u;
+    }
+    if (active) slice(r1, 1);
+    if (kIn) {
+      __syncwarp();
+      if (next < c.num_tiles) {
+        if (lane == 0) issue_in(1, next_n_w, next_row0);
+        pending[1] = true;
+      }
+    }
+    if (active) {
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        if (aux_out) ptx::tma_store_2d(tm_aux, buf_aux, n_w, row0);
+        ptx::tma_store_2d(tm_out, buf_out, n_w, row0);
+        ptx::bulk_commit_group();
+      }
+    }
+    tile = next; row0 = next_row0; n_w = next_n_w;
+  }
+  // Leaving early (a wait ran out somewhere in the CTA): let tensor-memory loads and input boxes
+  // that are still in flight land before the CTA may give up its resources.
+  ptx::tmem_ld_wait_all();
+  if (kIn && lane == 0) {
+    if (pending[0]) for (uint32_t it = 0; it < p.wait_limit && !ptx::mbar_try_wait(c.in_bar, ph0); ++it) {}
+    if (pending[1]) for (uint32_t it = 0; it < p.wait_limit && !ptx::mbar_try_wait(in_bar1, ph1); ++it) {}
+  }
   if (lane == 0) ptx::bulk_wait_group_read<0>();             // stores have left shared memory before the CTA may exit
   __syncwarp();
 }
@@ -485,14 +669,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_addr(smem_raw));
   const uint32_t epi_base = smem_base + S::kStages * S::kStageBytes;      // 1024-byte aligned staging boxes
   const uint32_t bars = epi_base + S::kEpiBytes;
-  // barrier layout (8 bytes each): full[kStages], empty[kStages], acc_full[2], acc_empty[2], drained, epi_in[8]
+  // barrier layout (8 bytes each): full[kStages], empty[kStages], acc_full[2], acc_empty[2], drained, epi_in[2 * EW]
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (S::kStages + s); };
   auto acc_full_bar = [&](int a) { return bars + 8u * (2 * S::kStages + a); };
   auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * S::kStages + 2 + a); };
   const uint32_t drained_bar = bars + 8u * (2 * S::kStages + 4);
-  auto epi_in_bar = [&](int w) { return bars + 8u * (2 * S::kStages + 5 + w); };
-  uint8_t* tail = smem_gen + S::kStages * S::kStageBytes + S::kEpiBytes + 8 * (2 * S::kStages + 5 + EW);
+  auto epi_in_bar = [&](int w) { return bars + 8u * (2 * S::kStages + 5 + w); };   // epilogue warp w owns 2 w and 2 w + 1
+  static_assert(8 * (2 * S::kStages + 5 + 2 * EW) + 8 <= S::kBarrierBytes, "barrier area too small");
+  uint8_t* tail = smem_gen + S::kStages * S::kStageBytes + S::kEpiBytes + 8 * (2 * S::kStages + 5 + 2 * EW);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
 
@@ -508,7 +693,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int epi_arrivals = EPI != kEpiLegacy ? CG * 4 * (BN / (EW == 16 ? 64 : 128)) : CG * kEpilogueWarps;
     for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full_bar(a), 1); ptx::mbar_init(acc_empty_bar(a), epi_arrivals); }
     ptx::mbar_init(drained_bar, 1);
-    for (int w = 0; w < EW; ++w) ptx::mbar_init(epi_in_bar(w), 1);
+    for (int w = 0; w < 2 * EW; ++w) ptx::mbar_init(epi_in_bar(w), 1);
     *abort_flag = 0;
     ptx::mbar_init_fence();
     ptx::prefetch_tensormap(&tmap_a);
@@ -530,13 +715,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       uint32_t issued = 0;
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
-      for (int tile = group; ok && tile < num_tiles; tile += num_groups) {
+      for (int tile = group; ok && !p.no_loads && tile < num_tiles; tile += num_groups) {
         const int m0 = tile_m(p, tile) * (kBM * CG) + rank * kBM;
         const int n0 = tile_n(p, tile) * BN + rank * kBRows;
         int b0 = 0, b1 = 0;
         if (BATCHED) tile_batch(p, tile, b0, b1);
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status);
+          ok = wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status, p.wait_limit);
           if (!ok) break;
           const uint32_t a_dst = smem_base + stage * S::kStageBytes;
           const uint32_t b_dst = a_dst + S::kABytes;
@@ -573,7 +758,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
         for (uint32_t i = 0; i < n; ++i) {
           if (stage == 0) { stage = S::kStages; phase ^= 1u; }
           --stage;
-          for (uint32_t it = 0; it < kWaitLimit && !ptx::mbar_try_wait(full_bar(stage), phase); ++it) {}
+          for (uint32_t it = 0; it < p.wait_limit && !ptx::mbar_try_wait(full_bar(stage), phase); ++it) {}
         }
       }
     }
@@ -598,14 +783,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       const uint32_t idesc = p.idesc;
       for (int tile = group; ok && tile < num_tiles; tile += num_groups, ++local) {
         const uint32_t acc = local & 1u, acc_phase = (local >> 1) & 1u;
-        ok = wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status);
+        ok = wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, p.wait_limit);
         if (!ok) break;
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         uint32_t accumulate = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!ptx::mbar_try_wait(full_bar(stage), phase)) {
-            ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status);
+            ok = wait_bounded(full_bar(stage), phase, abort_flag, p.status, p.wait_limit);
             if (!ok) break;
           }
           ptx::tc_fence_after_sync();
@@ -628,17 +813,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       }
       if (*abort_flag) {
         if (CG == 2) ptx::mma_commit_pair(drained_bar, 1); else ptx::mma_commit(drained_bar);
-        for (uint32_t it = 0; it < kWaitLimit && !ptx::mbar_try_wait(drained_bar, 0); ++it) {}
+        for (uint32_t it = 0; it < p.wait_limit && !ptx::mbar_try_wait(drained_bar, 0); ++it) {}
       }
     }
   } else if (EPI != kEpiLegacy) {
     // ------------------------------------------------------------ epilogue warps, through shared memory + TMA
     EpiCtx c;
     c.tmem_base = tmem_base; c.acc_full0 = acc_full_bar(0); c.acc_empty0 = acc_empty_bar(0);
-    c.in_bar = epi_in_bar(warp - 2); c.buf0 = epi_base + (warp - 2) * epi_warp_bytes(EW);
+    c.in_bar = epi_in_bar(2 * (warp - 2)); c.buf0 = epi_base + (warp - 2) * epi_warp_bytes(EW);
     c.abort_flag = abort_flag; c.warp = warp; c.lane = lane; c.rank = rank;
     c.group = group; c.num_groups = num_groups; c.num_tiles = num_tiles;
-    epilogue_staged<BN, CG, EPI, EW, BATCHED>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
+    if constexpr (EW == 16) {
+      const uint32_t in_bar1 = epi_in_bar(2 * (warp - 2) + 1);
+      const bool e5 = p.out_dt == US_E5M2, bf = p.aux_dt == US_BF16;
+      if (e5 && bf) epilogue_act16<BN, CG, EPI, true, true>(p, &tmap_out, &tmap_aux, c, in_bar1);
+      else if (e5) epilogue_act16<BN, CG, EPI, true, false>(p, &tmap_out, &tmap_aux, c, in_bar1);
+      else if (bf) epilogue_act16<BN, CG, EPI, false, true>(p, &tmap_out, &tmap_aux, c, in_bar1);
+      else epilogue_act16<BN, CG, EPI, false, false>(p, &tmap_out, &tmap_aux, c, in_bar1);
+    } else {
+      epilogue_staged<BN, CG, EPI, EW, BATCHED>(p, &tmap_out, &tmap_aux, &tmap_skip, c);
+    }
   } else {
     // ------------------------------------------------------------ epilogue warps, direct global accesses
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
@@ -654,7 +848,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       EpiloguePrefetch pf;
       const int c_first = 32 * half;
       if (row_ok && n0 + c_first + 32 <= p.N) prefetch_full(p, row, n0 + c_first, pf);
-      ok = wait_bounded(acc_full_bar(acc), acc_phase, abort_flag, p.status);
+      ok = wait_bounded(acc_full_bar(acc), acc_phase, abort_flag, p.status, p.wait_limit);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       ptx::tc_fence_after_sync();
