@@ -142,6 +142,12 @@ us_status us_linear_bwd_w_batched(const us_mat* X, const us_mat* G, float beta_w
 /* Bytes of device workspace the linear ops need. */
 size_t us_workspace_bytes(void);
 
+/* us_linear_fwd_check: the host-side checks of us_linear_fwd (arguments, dtypes, shapes, alignment,
+ * workspace) without a launch: returns what us_linear_fwd would return before it reaches the device,
+ * US_OK if it would launch.  Touches neither the device nor `ws` (only its address and size are looked at). */
+us_status us_linear_fwd_check(const us_mat* X, const us_mat* W, const us_epilogue* ep, const us_mat* Y,
+                              const void* ws, size_t ws_bytes);
+
 /* Waits for `stream`, copies the workspace status word to the host and returns
  * US_OK, US_ERR_TIMEOUT (a device-side wait gave up: the outputs of that call are
  * not valid) or US_ERR_CUDA.  This is the only call that synchronises. */
@@ -161,8 +167,9 @@ us_status us_workspace_status(const void* ws, void* stream);
  *
  *  - The first call on a device looks up the array's device address (a one-time set-up with
  *    that device current).  Make that first call before starting any stream capture.
- *  - All calls share the one array and it keeps the previous call's contents, so every call
- *    first clears the status word on `stream`.  Two calls that overlap on the GPU (different
+ *  - All calls share the one array and it keeps the previous call's contents, so every call that
+ *    passes the host-side checks first clears the status word on `stream` (a call that returns an
+ *    argument, dtype, alignment or workspace error enqueues nothing and leaves the word as it was).  Two calls that overlap on the GPU (different
  *    streams) race on that word: keep calls to this entry point on one stream, or order them.
  *  - If the kernel's scratch requirement ever exceeds the built-in 1024 bytes the call returns
  *    US_ERR_WORKSPACE and launches nothing; the requirement does not depend on the matrix sizes.
@@ -172,6 +179,20 @@ us_status us_workspace_status(const void* ws, void* stream);
  */
 us_status us_linear_fwd_static_ws(const us_mat* X, const us_mat* W, float alpha, const us_epilogue* ep,
                                   const us_mat* Y, void** ws_out, void* stream);
+
+/*
+ * us_test_linear_fwd_starved: exercises the failure path of the linear kernels (the paper has no counterpart;
+ * this exists so that the bounded waits and their clean-up can be tested without faulting a GPU).
+ * It launches the kernel of us_linear_fwd (no epilogue) with two changes: the warp that loads the
+ * operands issues no loads, and every device-side wait gives up after `wait_limit` polls
+ * (1 .. 65536) instead of the library's normal limit.  Nothing is in flight, so the waits of all roles run
+ * out, the kernel raises the status word in `ws`, releases its tensor memory and returns by itself;
+ * us_workspace_status(ws) then reports US_ERR_TIMEOUT and Y is not valid.  The device and the
+ * context stay usable: clear the word (cudaMemsetAsync) and carry on.  Arguments and host-side
+ * errors as for us_linear_fwd.
+ */
+us_status us_test_linear_fwd_starved(const us_mat* X, const us_mat* W, float alpha, const us_mat* Y, void* ws,
+                                     size_t ws_bytes, unsigned int wait_limit, void* stream);
 
 /* Activations of the table "Table of unit scaling factors", section Activations. */
 typedef enum { US_FN_GELU = 0, US_FN_RELU = 1, US_FN_TANH = 2, US_FN_SIGMOID = 3 } us_fn;

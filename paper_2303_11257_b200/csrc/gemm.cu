@@ -19,9 +19,16 @@ static bool is_fp8(int dt) { return dt == US_E4M3 || dt == US_E5M2; }
 
 enum Op { kFwd, kBwdX, kBwdW };
 
+// Failure-path test settings of one call: a short wait limit, and a producer that issues no loads.
+struct WaitTest {
+  uint32_t wait_limit;
+  int no_loads;
+};
+
 // A, B: the two operands in call order; out [M x N].
 static us_status linear(Op op, const us_mat* A, const us_mat* B, float scale, const us_epilogue* ep, const us_mat* out,
-                        void* ws, size_t ws_bytes, void* stream, const us_batch* batch = nullptr) {
+                        void* ws, size_t ws_bytes, void* stream, const us_batch* batch = nullptr,
+                        const WaitTest* wt = nullptr, bool validate_only = false) {
   if (!valid_mat(A) || !valid_mat(B) || !valid_mat(out)) return US_ERR_INVALID_ARG;
   int64_t M, N, K;
   bool shapes_ok;
@@ -41,7 +48,8 @@ static us_status linear(Op op, const us_mat* A, const us_mat* B, float scale, co
   p.scale = scale;
   p.out = out->ptr; p.out_dt = out->dtype; p.out_ld = out->ld;
   p.out_coef = 1.f;
-  p.wait_limit = kWaitLimit;
+  p.wait_limit = wt ? wt->wait_limit : kWaitLimit;
+  p.no_loads = wt ? wt->no_loads : 0;
   if (ep) {
     if (ep->act < US_ACT_NONE || ep->act > US_ACT_GELU_GRAD) return US_ERR_INVALID_ARG;
     p.act = ep->act; p.act_in = ep->act_in_scale; p.act_out = ep->act_out_scale;
@@ -92,6 +100,7 @@ static us_status linear(Op op, const us_mat* A, const us_mat* B, float scale, co
     }
     if ((long long)((M + 127) / 128) * ((N + 127) / 128) * bd.nb0 * bd.nb1 > 0x7fffffffll) return US_ERR_INVALID_ARG;
   }
+  if (validate_only) return US_OK;                     // every host check has passed; nothing has been launched
   const bool a_mn = (op == kBwdW), b_mn = (op != kBwdX);
   const int a_fmt = f8 ? (A->dtype == US_E5M2) : (A->dtype == US_BF16);
   const int b_fmt = f8 ? (B->dtype == US_E5M2) : (B->dtype == US_BF16);
@@ -140,6 +149,18 @@ extern "C" us_status us_linear_bwd_w_batched(const us_mat* X, const us_mat* G, f
                                              const us_batch* batch, void* ws, size_t ws_bytes, void* stream) {
   if (!batch) return US_ERR_INVALID_ARG;
   return us::linear(us::kBwdW, X, G, beta_w, nullptr, dW, ws, ws_bytes, stream, batch);
+}
+
+extern "C" us_status us_linear_fwd_check(const us_mat* X, const us_mat* W, const us_epilogue* ep, const us_mat* Y,
+                                         const void* ws, size_t ws_bytes) {
+  return us::linear(us::kFwd, X, W, 1.f, ep, Y, const_cast<void*>(ws), ws_bytes, nullptr, nullptr, nullptr, true);
+}
+
+extern "C" us_status us_test_linear_fwd_starved(const us_mat* X, const us_mat* W, float alpha, const us_mat* Y, void* ws,
+                                                size_t ws_bytes, unsigned int wait_limit, void* stream) {
+  if (wait_limit < 1 || wait_limit > (1u << 16)) return US_ERR_INVALID_ARG;
+  const us::WaitTest wt = {wait_limit, 1};
+  return us::linear(us::kFwd, X, W, alpha, nullptr, Y, ws, ws_bytes, stream, nullptr, &wt);
 }
 
 extern "C" size_t us_workspace_bytes(void) { return 256; }

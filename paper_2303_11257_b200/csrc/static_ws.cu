@@ -20,7 +20,9 @@ constexpr size_t kStaticWsBytes = 1024;
 __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_ws_addr[kMaxDevices];      // device address of g_static_ws on each device, 0 = not set up
+// Device address of g_static_ws on each device, 0 = not set up.  Written without a lock: threads that race
+// on the first call of a device all store the same value.
+void* g_ws_addr[kMaxDevices];
 
 // In host code `g_static_ws` names a host-side shadow of the symbol, not device memory, so it
 // must never be handed to a kernel.  Ask the runtime for the real address, once per device,
@@ -46,6 +48,10 @@ extern "C" us_status us_linear_fwd_static_ws(const us_mat* X, const us_mat* W, f
   if (us_workspace_bytes() > kStaticWsBytes) return US_ERR_WORKSPACE;
   void* ws = nullptr;
   us_status s = static_ws_address(&ws);
+  if (s != US_OK) return s;
+  // Every host-side check of us_linear_fwd first, so that a call with bad arguments enqueues nothing
+  // (no clearing of the status word either) and leaves the previous call's status readable.
+  s = us_linear_fwd_check(X, W, ep, Y, ws, kStaticWsBytes);
   if (s != US_OK) return s;
   // The array keeps whatever the previous call left in it: the status word has to start at zero.
   if (cudaMemsetAsync(ws, 0, us_workspace_bytes(), static_cast<cudaStream_t>(stream)) != cudaSuccess)

@@ -70,6 +70,10 @@ def _load() -> C.CDLL:
         fn.restype = C.c_int
     lib.us_linear_fwd_static_ws.argtypes = [MP, MP, F, EP, MP, C.POINTER(C.c_void_p), V]
     lib.us_linear_fwd_static_ws.restype = C.c_int
+    lib.us_linear_fwd_check.argtypes = [MP, MP, EP, MP, V, SZ]
+    lib.us_linear_fwd_check.restype = C.c_int
+    lib.us_test_linear_fwd_starved.argtypes = [MP, MP, F, MP, V, SZ, C.c_uint, V]
+    lib.us_test_linear_fwd_starved.restype = C.c_int
     lib.us_workspace_bytes.argtypes = []
     lib.us_workspace_bytes.restype = SZ
     lib.us_workspace_status.argtypes = [V, V]
@@ -225,6 +229,21 @@ def us_linear_fwd_static_ws(X, W, alpha, Y, ep=None, stream=None) -> int:
            _lib.us_linear_fwd_static_ws(C.byref(mat(X)), C.byref(mat(W)), alpha, epp, C.byref(mat(Y)),
                                         C.byref(ws), _stream(stream)))
     return ws.value
+
+
+def us_linear_fwd_check(X, W, Y, ws, ep=None) -> int:
+    """Status us_linear_fwd would return from its host-side checks (0 = it would launch); launches nothing."""
+    epp = C.byref(ep) if ep is not None else None
+    return int(_lib.us_linear_fwd_check(C.byref(mat(X)), C.byref(mat(W)), epp, C.byref(mat(Y)),
+                                        ws.data_ptr(), ws.numel() * ws.element_size()))
+
+
+def us_test_linear_fwd_starved(X, W, alpha, Y, ws, wait_limit: int, stream=None):
+    """The failure-path exercise of the header: a forward linear launch whose loads are withheld and
+    whose waits give up after wait_limit polls; the status word in ws is raised and the kernel returns."""
+    _check("us_test_linear_fwd_starved",
+           _lib.us_test_linear_fwd_starved(C.byref(mat(X)), C.byref(mat(W)), alpha, C.byref(mat(Y)), ws.data_ptr(),
+                                           ws.numel() * ws.element_size(), wait_limit, _stream(stream)))
 
 
 def us_workspace_status_ptr(ws_ptr: int, stream=None) -> int:
