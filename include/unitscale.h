@@ -139,6 +139,37 @@ us_status us_linear_bwd_x_batched(const us_mat* G, const us_mat* W, float beta_x
 us_status us_linear_bwd_w_batched(const us_mat* X, const us_mat* G, float beta_w, const us_mat* dW, const us_batch* batch,
                                   void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * us_linear_group: count (1..4) independent linear ops as ONE kernel launch.
+ *
+ * Each call is one of the three GEMMs of section "Example" with the same arithmetic, rounding and
+ * scale handling as the single entry points (bit-identical results: a tile is always accumulated by
+ * one accumulator over its whole K range).  The ops must not depend on one another (no output of one
+ * is an operand, skip tensor or output of another).  Meant for the tail of a training step, where
+ * several GEMMs of different shapes are ready at once -- for the FFN block the second forward GEMM,
+ * both weight-gradient GEMMs and the first layer's input-gradient GEMM -- and separate launches
+ * would each leave a partly filled last wave: the tiles of all calls are dealt to the SMs together,
+ * longest contraction first.
+ *
+ * a, b: the two operands in the order of the single entry point for `op` (X, W / G, W / X, G);
+ * scale: alpha, beta_x or beta_w; ep: act must be US_ACT_NONE, the skip path (fixed(tau) residual) is
+ * available; out as for the single entry points.
+ *
+ * Covered by this form: FP8 operands, outputs with more than 128 rows and more than 128 columns.
+ * Any other valid call (16-bit operands, a fused activation, a small output, more tiles than the
+ * work list holds) returns US_ERR_UNSUPPORTED and launches nothing: issue those calls one by one.
+ * Other errors and the workspace as for us_linear_fwd.
+ */
+typedef enum { US_OP_FWD = 0, US_OP_BWD_X = 1, US_OP_BWD_W = 2 } us_linear_op;
+typedef struct {
+  int32_t op; /* us_linear_op */
+  us_mat a, b;
+  float scale;
+  us_epilogue ep;
+  us_mat out;
+} us_linear_call;
+us_status us_linear_group(int count, const us_linear_call* calls, void* ws, size_t ws_bytes, void* stream);
+
 /* Bytes of device workspace the linear ops need. */
 size_t us_workspace_bytes(void);
 

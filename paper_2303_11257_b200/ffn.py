@@ -88,6 +88,11 @@ class UnitScaledFFN:
         # 128 tiles on 74 CTA pairs); measured 6 % faster than one stream once the power cap holds the clock.
         self.concurrent = self.fused_casts
         self._side = None
+        # FP8 operands: the four GEMMs that remain after the GELU-gradient GEMM are independent of one another and
+        # go out as one us_linear_group launch (4 launches per step instead of 7).
+        self.grouped = operand == "fp8"
+        if self.grouped:
+            self.launches_per_step = 4
 
     def _cast(self, src, dst, stream):
         if dst.dtype in (torch.float8_e4m3fn, torch.float8_e5m2):
@@ -126,6 +131,17 @@ class UnitScaledFFN:
             ("bwd_x1_residual", "gemm", lambda st=None: L.us_linear_bwd_x(self.dHq, self.W1q, sc.beta_x1, self.dX, ws, ep5, st)),
             ("bwd_w1", "gemm", lambda st=None: L.us_linear_bwd_w(self.Xq, self.dHq, sc.beta_w, self.dW1, ws, None, st)),
         ]
+
+    def group_calls(self, X, G):
+        """The four GEMMs that follow the GELU-gradient GEMM, as the entries of one us_linear_group launch
+        (same operands, scales and epilogues as the stages fwd2_residual, bwd_w2, bwd_x1_residual, bwd_w1)."""
+        sc, (c_skip, c_branch) = self.sc, self._c
+        ep2 = L.epilogue(skip=X, skip_coef=c_skip, out_coef=c_branch)
+        ep5 = L.epilogue(skip=G, skip_coef=c_skip, out_coef=c_branch)
+        return [L.linear_call(L.US_OP_BWD_W, self.Aq, self.Gq, sc.beta_w, self.dW2),
+                L.linear_call(L.US_OP_BWD_W, self.Xq, self.dHq, sc.beta_w, self.dW1),
+                L.linear_call(L.US_OP_FWD, self.Aq, self.W2q, sc.alpha2, self.R, ep2),
+                L.linear_call(L.US_OP_BWD_X, self.dHq, self.W1q, sc.beta_x1, self.dX, ep5)]
 
     def cast_weights(self, W1, W2, stream=None):
         self._cast(W1, self.W1q, stream)
@@ -174,6 +190,22 @@ class UnitScaledFFN:
         With self.concurrent and no explicit stream, independent GEMMs go to two side streams that fork from
         and join back into the current stream (this also records as parallel branches under graph capture)."""
         st = self.stages(X, W1, W2, G)
+        if self.grouped and self.fused_casts:
+            by = {name: fn for name, _, fn in st}
+            for name in ("cast_all", "fwd1_gelu", "bwd_x2_gelu_grad"):
+                by[name](stream)
+            try:
+                L.us_linear_group(self.group_calls(X, G), self.ws, stream)
+                return self.dX, self.dW1, self.dW2
+            except L.UnitScaleError as e:
+                if e.status != L.US_ERR_UNSUPPORTED:
+                    raise
+                # a shape the grouped form does not cover (an output of at most 128 rows or columns): nothing was
+                # launched; the four GEMMs go out one by one, now and in later steps
+                self.grouped, self.launches_per_step = False, 7
+                for name in ("fwd2_residual", "bwd_w2", "bwd_x1_residual", "bwd_w1"):
+                    by[name](stream)
+                return self.dX, self.dW1, self.dW2
         if not (self.concurrent and self.fused_casts and stream is None):
             for name, _, fn in st:
                 fn(stream)

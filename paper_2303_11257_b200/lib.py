@@ -11,7 +11,7 @@ import os
 
 import torch
 
-US_OK = 0
+US_OK, US_ERR_INVALID_ARG, US_ERR_UNSUPPORTED, US_ERR_ALIGNMENT, US_ERR_WORKSPACE, US_ERR_CUDA, US_ERR_TIMEOUT = range(7)
 STATUS_NAMES = {
     0: "US_OK", 1: "US_ERR_INVALID_ARG", 2: "US_ERR_UNSUPPORTED", 3: "US_ERR_ALIGNMENT",
     4: "US_ERR_WORKSPACE", 5: "US_ERR_CUDA", 6: "US_ERR_TIMEOUT",
@@ -40,6 +40,13 @@ class us_epilogue(C.Structure):
 
 class us_batch(C.Structure):
     _fields_ = [("count", C.c_int64 * 2), ("a_stride", C.c_int64 * 2), ("b_stride", C.c_int64 * 2), ("out_stride", C.c_int64 * 2)]
+
+
+class us_linear_call(C.Structure):
+    _fields_ = [("op", C.c_int32), ("a", us_mat), ("b", us_mat), ("scale", C.c_float), ("ep", us_epilogue), ("out", us_mat)]
+
+
+US_OP_FWD, US_OP_BWD_X, US_OP_BWD_W = 0, 1, 2
 
 
 class UnitScaleError(RuntimeError):
@@ -74,6 +81,8 @@ def _load() -> C.CDLL:
     lib.us_linear_fwd_check.restype = C.c_int
     lib.us_test_linear_fwd_starved.argtypes = [MP, MP, F, MP, V, SZ, C.c_uint, V]
     lib.us_test_linear_fwd_starved.restype = C.c_int
+    lib.us_linear_group.argtypes = [C.c_int, C.POINTER(us_linear_call), V, SZ, V]
+    lib.us_linear_group.restype = C.c_int
     lib.us_workspace_bytes.argtypes = []
     lib.us_workspace_bytes.restype = SZ
     lib.us_workspace_status.argtypes = [V, V]
@@ -190,6 +199,24 @@ def us_linear_bwd_x(G, W, beta_x, dX, ws, ep=None, stream=None):
 
 def us_linear_bwd_w(X, G, beta_w, dW, ws, ep=None, stream=None):
     return _linear("us_linear_bwd_w", X, G, beta_w, ep, dW, ws, stream)
+
+
+def linear_call(op: int, a, b, scale: float, out, ep=None) -> us_linear_call:
+    """One entry of a us_linear_group launch: op in (US_OP_FWD, US_OP_BWD_X, US_OP_BWD_W), operands in that op's order."""
+    c = us_linear_call()
+    c.op, c.a, c.b, c.scale, c.out = op, mat(a), mat(b), scale, mat(out)
+    if ep is not None:
+        c.ep = ep
+    else:
+        c.ep.out_coef = 1.0
+    c._keep_alive = (a, b, out, ep)
+    return c
+
+
+def us_linear_group(calls, ws, stream=None):
+    """Several independent linear ops in one launch (see the header for what this form covers)."""
+    arr = (us_linear_call * len(calls))(*calls)
+    _check("us_linear_group", _lib.us_linear_group(len(calls), arr, ws.data_ptr(), ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def batch(count, a_stride, b_stride, out_stride) -> us_batch:
