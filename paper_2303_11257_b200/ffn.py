@@ -132,6 +132,17 @@ class UnitScaledFFN:
             ("bwd_w1", "gemm", lambda st=None: L.us_linear_bwd_w(self.Xq, self.dHq, sc.beta_w, self.dW1, ws, None, st)),
         ]
 
+    def step_launches(self, X, W1, W2, G):
+        """The launches step() makes, in order, as (name, kind, GEMMs in the launch, callable(stream)): with the
+        grouped form the four GEMMs after the GELU-gradient GEMM are one entry of kind "group"."""
+        st = self.stages(X, W1, W2, G)
+        if not (self.grouped and self.fused_casts):
+            return [(n, k, 1 if k == "gemm" else 0, fn) for n, k, fn in st]
+        by = {n: (k, fn) for n, k, fn in st}
+        head = [(n, by[n][0], 1 if by[n][0] == "gemm" else 0, by[n][1]) for n in ("cast_all", "fwd1_gelu", "bwd_x2_gelu_grad")]
+        return head + [("group_fwd2_bwd_w2_bwd_x1_bwd_w1", "group", 4,
+                        lambda stream=None: L.us_linear_group(self.group_calls(X, G), self.ws, stream))]
+
     def group_calls(self, X, G):
         """The four GEMMs that follow the GELU-gradient GEMM, as the entries of one us_linear_group launch
         (same operands, scales and epilogues as the stages fwd2_residual, bwd_w2, bwd_x1_residual, bwd_w1)."""
