@@ -49,7 +49,13 @@ typedef struct {
   int64_t rows, cols, ld;
 } us_mat;
 
-typedef enum { US_ACT_NONE = 0, US_ACT_GELU = 1, US_ACT_GELU_GRAD = 2 } us_act;
+typedef enum {
+  US_ACT_NONE = 0,
+  US_ACT_GELU = 1, US_ACT_GELU_GRAD = 2,
+  US_ACT_RELU = 3, US_ACT_RELU_GRAD = 4,
+  US_ACT_TANH = 5, US_ACT_TANH_GRAD = 6,
+  US_ACT_SIGMOID = 7, US_ACT_SIGMOID_GRAD = 8
+} us_act;
 
 /*
  * Work fused after the scaled accumulator of a linear op, applied per element in
@@ -64,6 +70,9 @@ typedef enum { US_ACT_NONE = 0, US_ACT_GELU = 1, US_ACT_GELU_GRAD = 2 } us_act;
  *   skip.ptr != NULL:  v = skip_coef * skip + out_coef * v
  *   out = round_to(out dtype, v)
  *
+ * The RELU / TANH / SIGMOID pairs do the same with f = max(x, 0), tanh, (1 + e^-x)^-1 (table section
+ * "Activations"; us_scales_activation gives their factors): forward v = act_out_scale * f(act_in_scale * v),
+ * gradient v = act_out_scale * act_in_scale * f'(act_in_scale * h) * v, relu'(0) = 0.
  * gelu(x) = x * Phi(x) with the exact normal CDF (table "Table of unit scaling
  * factors"); act_in_scale is the alignment pre-scale of appendix "Aligning a unit
  * scaled model with an existing model" (1 when unused).  The skip path is the
@@ -369,12 +378,24 @@ us_status us_quant_stats(const us_mat* src, float scale, us_dtype fmt, int exp_l
  *   them as 1.701 / 1.481); constrained: both equal their geometric mean.
  * us_scales_activation: the same pair for any us_fn (relu: sqrt(2 / (1 - 1/pi)), sqrt 2; tanh
  *   1.593 / 1.467; sigmoid 4.802 / 4.722 as printed, carried here to float precision).
+ * us_scales_residual: the coefficients of the fixed(tau) residual of section "Weighted addition",
+ *   sqrt(1 - tau) for the skip connection and sqrt(tau) for the branch, 0 <= tau <= 1 (tau = 1 / (l + 1)
+ *   gives the running-mean scheme for layer l).
+ * us_scales_attention: factors of scaled dot-product attention for sequences of s tokens and heads of
+ *   d_head features (appendix "Unit scaling and attention"; table row "softmax"; paragraph "Softmax
+ *   (followed by matmul)"): scores S = alpha_scores Q K^T with alpha_scores = beta_scores = d_head^-1/2 (beta for both
+ *   dQ and dK); softmax_scale = s (alpha and beta of the scaled softmax); context C = alpha_context P V, an
+ *   ordinary matmul with fan_in = s, fan_out = d_head, batch = s: alpha_context = s^-1/2, beta_p = d_head^-1/2
+ *   (gradient of P), beta_v = s^-1/2 (gradient of V); constrained: alpha_context = beta_p = (s d_head)^-1/4.
  * Pure host arithmetic; output pointers must be non-NULL.
  */
 us_status us_scales_linear(int64_t b, int64_t m, int64_t n, int constrained, float* alpha,
                            float* beta_x, float* beta_w);
 us_status us_scales_gelu(int constrained, float* alpha, float* beta);
 us_status us_scales_activation(us_fn fn, int constrained, float* alpha, float* beta);
+us_status us_scales_residual(float tau, float* skip_coef, float* branch_coef);
+us_status us_scales_attention(int64_t s, int64_t d_head, int constrained, float* alpha_scores, float* beta_scores,
+                              float* softmax_scale, float* alpha_context, float* beta_p, float* beta_v);
 
 const char* us_status_string(us_status s);
 int us_version(void);

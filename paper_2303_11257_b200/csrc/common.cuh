@@ -189,6 +189,34 @@ __device__ __forceinline__ float gelu_grad_scaled(float h, float g, float in_sca
   return (out_scale * in_scale) * d * g;
 }
 
+// relu, tanh and sigmoid of the table "Activations" and their derivatives.  exp through ex2.approx and a
+// correctly rounded division: absolute error about 2e-7 for the bounded functions.
+__device__ __forceinline__ float sigmoid_f(float z) {
+  const float e = ex2_approx(-1.4426950408889634f * fabsf(z));     // e^-|z| in (0, 1]
+  const float r = __fdiv_rn(1.0f, 1.0f + e);
+  return z >= 0.f ? r : e * r;
+}
+__device__ __forceinline__ float act_value(int fn, float z) {
+  if (fn == US_FN_RELU) return fmaxf(z, 0.f);
+  if (fn == US_FN_TANH) return 2.0f * sigmoid_f(2.0f * z) - 1.0f;
+  if (fn == US_FN_SIGMOID) return sigmoid_f(z);
+  return 0.f;   // gelu is dispatched before this point
+}
+__device__ __forceinline__ float act_slope(int fn, float z) {
+  if (fn == US_FN_RELU) return z > 0.f ? 1.0f : 0.f;
+  if (fn == US_FN_TANH) { const float s = sigmoid_f(2.0f * z), m = sigmoid_f(-2.0f * z); return 4.0f * s * m; }   // 1 - tanh^2
+  if (fn == US_FN_SIGMOID) return sigmoid_f(z) * sigmoid_f(-z);
+  return 0.f;
+}
+
+// out_scale * f(in_scale * h) and out_scale * in_scale * f'(in_scale * h) * g for any us_fn.
+__device__ __forceinline__ float act_scaled(int fn, float h, float in_scale, float out_scale) {
+  return fn == US_FN_GELU ? gelu_scaled(h, in_scale, out_scale) : out_scale * act_value(fn, in_scale * h);
+}
+__device__ __forceinline__ float act_grad_scaled(int fn, float h, float g, float in_scale, float out_scale) {
+  return fn == US_FN_GELU ? gelu_grad_scaled(h, g, in_scale, out_scale) : (out_scale * in_scale) * act_slope(fn, in_scale * h) * g;
+}
+
 // ---------------------------------------------------------------- two floats per instruction
 // sm_100 executes add / mul / fma on pairs of float32 held in a 64-bit register (same IEEE
 // rounding per lane as the scalar forms); the GEMM epilogues use it to halve the number of

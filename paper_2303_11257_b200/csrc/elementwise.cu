@@ -27,26 +27,6 @@ struct EwArgs {
 
 enum EwOp { kCast = 0, kGeluFwd = 1, kGeluBwd = 2, kResidual = 3, kActFwd = 4, kActBwd = 5 };
 
-// relu, tanh and sigmoid of the table "Activations" and their derivatives.  exp through ex2.approx and a
-// correctly rounded division: absolute error about 2e-7 for the bounded functions.
-__device__ __forceinline__ float sigmoid_f(float z) {
-  const float e = ex2_approx(-1.4426950408889634f * fabsf(z));     // e^-|z| in (0, 1]
-  const float r = __fdiv_rn(1.0f, 1.0f + e);
-  return z >= 0.f ? r : e * r;
-}
-__device__ __forceinline__ float act_value(int fn, float z) {
-  if (fn == US_FN_RELU) return fmaxf(z, 0.f);
-  if (fn == US_FN_TANH) return 2.0f * sigmoid_f(2.0f * z) - 1.0f;
-  if (fn == US_FN_SIGMOID) return sigmoid_f(z);
-  return 0.f;   // gelu is dispatched before this point
-}
-__device__ __forceinline__ float act_slope(int fn, float z) {
-  if (fn == US_FN_RELU) return z > 0.f ? 1.0f : 0.f;
-  if (fn == US_FN_TANH) { const float s = sigmoid_f(2.0f * z), m = sigmoid_f(-2.0f * z); return 4.0f * s * m; }   // 1 - tanh^2
-  if (fn == US_FN_SIGMOID) return sigmoid_f(z) * sigmoid_f(-z);
-  return 0.f;
-}
-
 template <int OP>
 __device__ __forceinline__ float ew_apply(float a, float b, const EwArgs& p) {
   if (OP == kActFwd)                                                          // c0 = s_in, c1 = alpha

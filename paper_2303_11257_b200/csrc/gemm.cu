@@ -51,9 +51,15 @@ static us_status linear(Op op, const us_mat* A, const us_mat* B, float scale, co
   p.wait_limit = wt ? wt->wait_limit : kWaitLimit;
   p.no_loads = wt ? wt->no_loads : 0;
   if (ep) {
-    if (ep->act < US_ACT_NONE || ep->act > US_ACT_GELU_GRAD) return US_ERR_INVALID_ARG;
-    p.act = ep->act; p.act_in = ep->act_in_scale; p.act_out = ep->act_out_scale;
-    if (ep->act == US_ACT_GELU_GRAD && !ep->aux.ptr) return US_ERR_INVALID_ARG;
+    if (ep->act < US_ACT_NONE || ep->act > US_ACT_SIGMOID_GRAD) return US_ERR_INVALID_ARG;
+    // the activation's class (forward: value from the accumulator; gradient: slope from the stored pre-activation)
+    // and which function of the table it is
+    const bool grad = ep->act != US_ACT_NONE && (ep->act % 2) == 0;
+    p.act = ep->act == US_ACT_NONE ? US_ACT_NONE : grad ? US_ACT_GELU_GRAD : US_ACT_GELU;
+    p.fn = ep->act <= US_ACT_GELU_GRAD ? US_FN_GELU : ep->act <= US_ACT_RELU_GRAD ? US_FN_RELU
+         : ep->act <= US_ACT_TANH_GRAD ? US_FN_TANH : US_FN_SIGMOID;
+    p.act_in = ep->act_in_scale; p.act_out = ep->act_out_scale;
+    if (grad && !ep->aux.ptr) return US_ERR_INVALID_ARG;
     if (ep->act != US_ACT_NONE && ep->aux.ptr) {
       if (ep->aux.rows != M || ep->aux.cols != N || ep->aux.ld < N) return US_ERR_INVALID_ARG;
       if (ep->aux.dtype != US_BF16 && ep->aux.dtype != US_F16) return US_ERR_UNSUPPORTED;

@@ -69,7 +69,7 @@ us_status check_call(const us_linear_call* c, Shape* sh) {
     const bool h16 = (c->a.dtype == US_BF16 || c->a.dtype == US_F16) && c->a.dtype == c->b.dtype;
     return h16 ? US_ERR_UNSUPPORTED : US_ERR_UNSUPPORTED;
   }
-  if (c->ep.act != US_ACT_NONE) return c->ep.act < US_ACT_NONE || c->ep.act > US_ACT_GELU_GRAD ? US_ERR_INVALID_ARG : US_ERR_UNSUPPORTED;
+  if (c->ep.act != US_ACT_NONE) return c->ep.act < US_ACT_NONE || c->ep.act > US_ACT_SIGMOID_GRAD ? US_ERR_INVALID_ARG : US_ERR_UNSUPPORTED;
   if (c->ep.skip.ptr) {
     const us_mat* s = &c->ep.skip;
     if (s->rows != M || s->cols != N || s->ld < N) return US_ERR_INVALID_ARG;

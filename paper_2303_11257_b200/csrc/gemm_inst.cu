@@ -103,7 +103,7 @@ static us_status pick_epilogue(const us_mat* A, const us_mat* B, const GemmParam
   }
   // The GELU epilogues with an FP8 output (the FFN's forward and backward hidden layer) are ALU
   // bound with eight epilogue warps; they run with sixteen.
-  const bool fp8_out = em.out->dtype == US_E4M3 || em.out->dtype == US_E5M2;
+  const bool fp8_out = (em.out->dtype == US_E4M3 || em.out->dtype == US_E5M2) && p.fn == US_FN_GELU;   // the 16-warp epilogue is the GELU pair's
   switch (epi) {
     case kEpiPlain:    return launch<ES, A_MN, B_MN, BN, CG, kEpiPlain, 8>(A, B, p, em, stream);
     case kEpiGelu:     return fp8_out ? launch<ES, A_MN, B_MN, BN, CG, kEpiGelu, 16>(A, B, p, em, stream)

@@ -56,7 +56,8 @@ struct GemmParams {
   float scale;
   uint32_t idesc;
   void* out; int out_dt; int64_t out_ld;
-  int act; float act_in, act_out;
+  int act; float act_in, act_out;          // act: US_ACT_NONE, or the forward / gradient class as US_ACT_GELU / US_ACT_GELU_GRAD
+  int fn;                                   // us_fn of the activation (US_FN_GELU for the GELU pair)
   void* aux; int aux_dt; int64_t aux_ld;
   const void* skip; int skip_dt; int64_t skip_ld; float skip_coef, out_coef;
   unsigned int* status;
@@ -182,12 +183,12 @@ __device__ __forceinline__ void epilogue_chunk_full(const GemmParams& p, float (
   if (p.act == US_ACT_GELU) {
     if (p.aux) store_vec<32>(static_cast<char*>(p.aux) + (row * p.aux_ld + col) * 2, p.aux_dt, v);
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = gelu_scaled(v[i], p.act_in, p.act_out);
+    for (int i = 0; i < 32; ++i) v[i] = act_scaled(p.fn, v[i], p.act_in, p.act_out);
   } else if (p.act == US_ACT_GELU_GRAD) {
     float h[32];
     unpack16<32>(f.aux, p.aux_dt, h);
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = gelu_grad_scaled(h[i], v[i], p.act_in, p.act_out);
+    for (int i = 0; i < 32; ++i) v[i] = act_grad_scaled(p.fn, h[i], v[i], p.act_in, p.act_out);
   }
   if (p.skip) {
     float sk[32];
@@ -215,12 +216,12 @@ __device__ __forceinline__ void epilogue_chunk_ragged(const GemmParams& p, float
         if (i < ncols) store_one(p.aux, p.aux_dt, row * p.aux_ld + col + i, v[i]);
     }
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = gelu_scaled(v[i], p.act_in, p.act_out);
+    for (int i = 0; i < 32; ++i) v[i] = act_scaled(p.fn, v[i], p.act_in, p.act_out);
   } else if (p.act == US_ACT_GELU_GRAD) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
       const float h = (i < ncols) ? load_one(p.aux, p.aux_dt, row * p.aux_ld + col + i) : 0.f;
-      v[i] = gelu_grad_scaled(h, v[i], p.act_in, p.act_out);
+      v[i] = act_grad_scaled(p.fn, h, v[i], p.act_in, p.act_out);
     }
   }
   if (p.skip) {
@@ -388,13 +389,27 @@ __device__ __forceinline__ void epilogue_staged(const GemmParams& p, const CUten
               ptx::sts128(buf_aux + row_off + (((aux_cb + g) ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
             }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) gelu_scaled2<kNarrowOut>(x[k], tail_k, act_oi, y[2 * k], y[2 * k + 1]);
+            for (int k = 0; k < 4; ++k) {
+              if (p.fn == US_FN_GELU) {
+                gelu_scaled2<kNarrowOut>(x[k], tail_k, act_oi, y[2 * k], y[2 * k + 1]);
+              } else {                                          // relu, tanh, sigmoid (table section "Activations")
+                float a, b;
+                unpack2(x[k], a, b);
+                y[2 * k] = act_scaled(p.fn, a, p.act_in, p.act_out); y[2 * k + 1] = act_scaled(p.fn, b, p.act_in, p.act_out);
+              }
+            }
           } else if (EPI == kEpiGeluGrad) {
             const uint32_t w[4] = {raw[g].x, raw[g].y, raw[g].z, raw[g].w};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               const float2 h = in_dt == US_BF16 ? unpack_bf16x2(w[k]) : unpack_f16x2(w[k]);
-              unpack2(gelu_grad_scaled2(pack2(h.x, h.y), x[k], in2, os2), y[2 * k], y[2 * k + 1]);
+              if (p.fn == US_FN_GELU) {
+                unpack2(gelu_grad_scaled2(pack2(h.x, h.y), x[k], in2, os2), y[2 * k], y[2 * k + 1]);
+              } else {
+                float a, b;
+                unpack2(x[k], a, b);
+                y[2 * k] = act_grad_scaled(p.fn, h.x, a, p.act_in, p.act_out); y[2 * k + 1] = act_grad_scaled(p.fn, h.y, b, p.act_in, p.act_out);
+              }
             }
           } else if (EPI == kEpiSkip) {
             float sk[8];

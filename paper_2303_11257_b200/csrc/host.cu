@@ -62,6 +62,30 @@ extern "C" us_status us_scales_activation(us_fn fn, int constrained, float* alph
   return US_OK;
 }
 
+extern "C" us_status us_scales_residual(float tau, float* skip_coef, float* branch_coef) {
+  if (!skip_coef || !branch_coef || !(tau >= 0.f && tau <= 1.f)) return US_ERR_INVALID_ARG;
+  *skip_coef = (float)sqrt(1.0 - (double)tau);
+  *branch_coef = (float)sqrt((double)tau);
+  return US_OK;
+}
+
+extern "C" us_status us_scales_attention(int64_t s, int64_t d_head, int constrained, float* alpha_scores, float* beta_scores,
+                                         float* softmax_scale, float* alpha_context, float* beta_p, float* beta_v) {
+  if (s < 1 || d_head < 1 || !alpha_scores || !beta_scores || !softmax_scale || !alpha_context || !beta_p || !beta_v)
+    return US_ERR_INVALID_ARG;
+  // scores Q K^T: 1 / sqrt(d_head) in both passes; context P V is an ordinary matmul with fan_in = batch = s, fan_out = d_head
+  const double a_s = 1.0 / sqrt((double)d_head);
+  double a_c = 1.0 / sqrt((double)s), b_p = 1.0 / sqrt((double)d_head);
+  if (constrained) a_c = b_p = sqrt(a_c * b_p);
+  *alpha_scores = (float)a_s;
+  *beta_scores = (float)a_s;
+  *softmax_scale = (float)s;
+  *alpha_context = (float)a_c;
+  *beta_p = (float)b_p;
+  *beta_v = (float)(1.0 / sqrt((double)s));
+  return US_OK;
+}
+
 extern "C" const char* us_status_string(us_status s) {
   switch (s) {
     case US_OK: return "ok";

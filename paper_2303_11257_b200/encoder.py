@@ -26,7 +26,6 @@ cast launch fewer); S and dP, which feed no matmul, stay in BF16.
 """
 from __future__ import annotations
 
-import math
 
 import torch
 
@@ -70,14 +69,12 @@ class UnitScaledEncoderLayer:
             self.dU1, self.dU2 = e(T, d, torch.bfloat16), e(T, d, torch.bfloat16)
             self.dln = [torch.empty(d, dtype=torch.float32, device=device) for _ in range(4)]      # dw1, dc1, dw2, dc2
             self.ln_ws = torch.empty(max(16, L.us_layer_norm_bwd_workspace_bytes(T, d)), dtype=torch.uint8, device=device)
-            self.beta_ln = T ** -0.5
-        self.c_skip, self.c_branch = math.sqrt(1.0 - tau), math.sqrt(tau)
+            self.beta_ln = L.us_scales_linear(T, 1, 1)[2]          # b^-1/2 with b = all tokens
+        self.c_skip, self.c_branch = L.us_scales_residual(tau)
         s, hd = slen, self.hd
-        self.sc = dict(
-            alpha_qkv=d ** -0.5, beta_qkv=(3 * d) ** -0.5, alpha_o=d ** -0.5, beta_o=d ** -0.5, beta_w=T ** -0.5,
-            alpha_s=hd ** -0.5, beta_Q=hd ** -0.5, beta_K=hd ** -0.5,          # attention scores: 1 / sqrt(d_head)
-            alpha_c=s ** -0.5, beta_P=hd ** -0.5, beta_V=s ** -0.5,            # context matmul: fan_in = s, fan_out = d_head, batch = s
-            sm=float(s))
+        a_qkv, b_qkv, b_w = L.us_scales_linear(T, d, 3 * d)
+        a_o, b_o, _ = L.us_scales_linear(T, d, d)
+        self.sc = dict(alpha_qkv=a_qkv, beta_qkv=b_qkv, alpha_o=a_o, beta_o=b_o, beta_w=b_w, **L.us_scales_attention(s, hd))
         qkv = (slen * 3 * d, hd)          # (outer, inner) strides of a head slice of a [T x 3d] matrix
         sq = (nhead * slen * slen, slen * slen)
         td = (slen * d, hd)               # head slice of a [T x d] matrix

@@ -19,7 +19,6 @@ mode the matmul inputs are rounded to that format instead (no loss scale, same f
 """
 from __future__ import annotations
 
-import math
 from dataclasses import dataclass
 
 import torch
@@ -45,7 +44,7 @@ class FFNScales:
         the global batch T * dp_world, and the ranks' weight gradients are summed afterwards (dp.py)."""
         a1, bx1, bw = L.us_scales_linear(T, d, f, constrained)
         if dp_world > 1:
-            bw = float(T * dp_world) ** -0.5
+            _, _, bw = L.us_scales_linear(T * dp_world, d, f, constrained)      # the batch of the weight gradient is global
         a2, bx2, _ = L.us_scales_linear(T, f, d, constrained)
         ag, bg = L.us_scales_gelu(constrained)
         return FFNScales(a1, a2, bx1, bx2, bw, ag, bg, 1.0, tau)
@@ -76,7 +75,7 @@ class UnitScaledFFN:
         self.dW1 = e(d, f, torch.float32)
         self.dW2 = e(f, d, torch.float32)
         self.ws = L.new_workspace(device)
-        c_skip, c_branch = math.sqrt(1.0 - self.sc.tau), math.sqrt(self.sc.tau)
+        c_skip, c_branch = L.us_scales_residual(self.sc.tau)
         self._c = (c_skip, c_branch)
         # step() has all four tensors to quantise at hand when it starts, so in FP8 mode it casts them
         # with one launch; forward() / backward() on their own cast what they are given.

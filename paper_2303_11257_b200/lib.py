@@ -17,7 +17,7 @@ STATUS_NAMES = {
     4: "US_ERR_WORKSPACE", 5: "US_ERR_CUDA", 6: "US_ERR_TIMEOUT",
 }
 US_F32, US_BF16, US_F16, US_E4M3, US_E5M2 = range(5)
-US_ACT_NONE, US_ACT_GELU, US_ACT_GELU_GRAD = range(3)
+US_ACT_NONE, US_ACT_GELU, US_ACT_GELU_GRAD, US_ACT_RELU, US_ACT_RELU_GRAD, US_ACT_TANH, US_ACT_TANH_GRAD, US_ACT_SIGMOID, US_ACT_SIGMOID_GRAD = range(9)
 US_FN_GELU, US_FN_RELU, US_FN_TANH, US_FN_SIGMOID = range(4)
 FN_BY_NAME = {"gelu": US_FN_GELU, "relu": US_FN_RELU, "tanh": US_FN_TANH, "sigmoid": US_FN_SIGMOID}
 
@@ -120,6 +120,10 @@ def _load() -> C.CDLL:
     lib.us_scales_activation.argtypes = [C.c_int, C.c_int, FP, FP]
     lib.us_scales_activation.restype = C.c_int
     lib.us_scales_gelu.restype = C.c_int
+    lib.us_scales_residual.argtypes = [C.c_float, FP, FP]
+    lib.us_scales_residual.restype = C.c_int
+    lib.us_scales_attention.argtypes = [C.c_int64, C.c_int64, C.c_int, FP, FP, FP, FP, FP, FP]
+    lib.us_scales_attention.restype = C.c_int
     lib.us_status_string.argtypes = [C.c_int]
     lib.us_status_string.restype = C.c_char_p
     lib.us_version.argtypes = []
@@ -403,6 +407,21 @@ def us_scales_gelu(constrained: bool = False):
     a, b = C.c_float(), C.c_float()
     _check("us_scales_gelu", _lib.us_scales_gelu(int(constrained), C.byref(a), C.byref(b)))
     return a.value, b.value
+
+
+def us_scales_residual(tau: float):
+    """(sqrt(1 - tau), sqrt(tau)) as the float32 values the library uses."""
+    a, b = C.c_float(), C.c_float()
+    _check("us_scales_residual", _lib.us_scales_residual(tau, C.byref(a), C.byref(b)))
+    return a.value, b.value
+
+
+def us_scales_attention(s: int, d_head: int, constrained: bool = False) -> dict:
+    """Factors of scaled dot-product attention (see the header), keyed as the encoder driver uses them."""
+    v = [C.c_float() for _ in range(6)]
+    _check("us_scales_attention", _lib.us_scales_attention(s, d_head, int(constrained), *[C.byref(x) for x in v]))
+    a_s, b_s, sm, a_c, b_p, b_v = (x.value for x in v)
+    return dict(alpha_s=a_s, beta_Q=b_s, beta_K=b_s, sm=sm, alpha_c=a_c, beta_P=b_p, beta_V=b_v)
 
 
 def us_status_string(status: int) -> str:

@@ -88,3 +88,27 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(L, "library_path", lambda: str(tmp_path / "nope.so"))
     with pytest.raises(ImportError):
         L._load()
+
+
+def test_residual_and_attention_scale_helpers(lib):
+    from oracle import scales as S
+    for tau in (0.0, 0.3, 0.5, 1.0 / 7, 1.0):
+        cs, cb = lib.us_scales_residual(tau)
+        ws, wb = S.residual_coefficients(float(C.c_float(tau).value))
+        assert cs == C.c_float(ws).value and cb == C.c_float(wb).value
+        assert abs(cs * cs + cb * cb - 1) < 2e-7                   # unit variance of the sum of independent unit inputs
+    with pytest.raises(lib.UnitScaleError):
+        lib.us_scales_residual(1.5)
+    for s, hd in ((512, 64), (128, 64), (80, 64), (272, 128)):
+        a = lib.us_scales_attention(s, hd)
+        f32 = lambda v: C.c_float(v).value
+        assert a["alpha_s"] == a["beta_Q"] == a["beta_K"] == f32(hd ** -0.5)      # appendix: 1 / sqrt(d) in both passes
+        assert a["sm"] == float(s)
+        # the context matmul P[s x s] V[s x d_head] takes the ordinary matmul factors with batch = fan_in = s
+        al, bx, bw = S.linear_scales(s, s, hd)
+        assert (a["alpha_c"], a["beta_P"], a["beta_V"]) == (f32(al), f32(bx), f32(bw))
+        c = lib.us_scales_attention(s, hd, True)
+        alc, bxc, _ = S.linear_scales(s, s, hd, True)
+        assert c["alpha_c"] == c["beta_P"] == f32(alc) and f32(bxc) == f32(alc)
+    with pytest.raises(lib.UnitScaleError):
+        lib.us_scales_attention(0, 64)

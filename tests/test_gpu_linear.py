@@ -187,3 +187,37 @@ def test_linear_argument_errors():
     ep = L.epilogue(act=L.US_ACT_GELU, aux=U.empty(32, 48, "f32"))
     assert status(L.us_linear_fwd, X, W, 1.0, Y, ws, ep) == 2                              # aux must be 16 bit
     assert L.us_workspace_status(ws) == 0
+
+
+@pytest.mark.parametrize("fn", ["relu", "tanh", "sigmoid"])
+@pytest.mark.parametrize("shape", [(256, 128, 512), (200, 144, 336)])
+def test_other_activations_as_epilogues(fn, shape):
+    """relu / tanh / sigmoid fused like GELU: forward with the kept pre-activation, gradient from the stored one
+    (table section "Activations"), against the oracle's activation_fwd / activation_bwd on the fp64 GEMM result."""
+    L, synth = _lib()
+    b, m, n = shape
+    X, W, G = synth.linear_tensors(b, m, n, 8)
+    a, bx, _ = S.linear_scales(b, m, n)
+    alpha_f, beta_f = {"relu": S.relu_scales, "tanh": S.tanh_scales, "sigmoid": S.sigmoid_scales}[fn]()
+    fwd_code = {"relu": L.US_ACT_RELU, "tanh": L.US_ACT_TANH, "sigmoid": L.US_ACT_SIGMOID}[fn]
+    ws = L.new_workspace()
+    val = O.linear_fwd(U.values_of(X, "e4m3"), U.values_of(W, "e4m3"), a)
+    for out_fmt in ("e4m3", "bf16", "f32"):
+        H = U.empty(b, n, "bf16")
+        A = U.empty(b, n, out_fmt)
+        ep = L.epilogue(act=fwd_code, act_in_scale=0.8, act_out_scale=float(alpha_f), aux=H)
+        L.us_linear_fwd(U.to_device(X, "e4m3"), U.to_device(W, "e4m3"), float(a), A, ws, ep)
+        U.assert_close_stored(H, val, "bf16", TOL, f"{fn}: stored pre-activation")
+        U.assert_close_stored(A, O.activation_fwd(fn, val, 0.8, alpha_f), out_fmt, TOL * float(alpha_f), f"{fn} -> {out_fmt}")
+    # gradient: dH = beta f'(s H) * (beta_x G W^T), H read back from its stored 16-bit form
+    Hh = synth.normal(8, 7, (b, m))
+    Hh[np.abs(Hh) < 1e-2] = 0.25                                # keep relu's kink away from rounding noise
+    Ht = U.to_device(Hh, "bf16")
+    gval = O.linear_bwd_x(U.values_of(G, "e5m2"), U.values_of(W, "e4m3"), bx)
+    ref = O.activation_bwd(fn, U.values_of(Hh, "bf16"), gval, 1.0, beta_f)
+    for out_fmt in ("e5m2", "bf16"):
+        dH = U.empty(b, m, out_fmt)
+        ep = L.epilogue(act=fwd_code + 1, act_in_scale=1.0, act_out_scale=float(beta_f), aux=Ht)
+        L.us_linear_bwd_x(U.to_device(G, "e5m2"), U.to_device(W, "e4m3"), float(bx), dH, ws, ep)
+        U.assert_close_stored(dH, ref, out_fmt, TOL * float(beta_f), f"{fn} gradient -> {out_fmt}")
+    assert L.us_workspace_status(ws) == 0
