@@ -113,8 +113,12 @@ typedef struct {
  *
  * ws: device workspace of at least us_workspace_bytes() bytes, 16-byte aligned,
  * zeroed once by the caller before its first use (cudaMemsetAsync).  It holds a
- * status word that a kernel sets if one of its bounded waits runs out; calls on
- * the same stream may share it.  Read it with us_workspace_status.
+ * status word that a kernel sets if one of its bounded waits runs out.  The word
+ * is sticky and only ever set, atomically, to one constant, so linear calls may
+ * share a workspace, also calls that run concurrently on different streams; it
+ * then tells that some call since the last clearing timed out, not which one.
+ * Read it with us_workspace_status (after the streams in question have been
+ * joined or synchronised) and clear it with cudaMemsetAsync.
  */
 us_status us_linear_fwd(const us_mat* X, const us_mat* W, float alpha, const us_epilogue* ep,
                         const us_mat* Y, void* ws, size_t ws_bytes, void* stream);

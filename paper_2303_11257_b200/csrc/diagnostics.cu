@@ -2,7 +2,8 @@
 // formats for deep learning", paragraph "Quantisation error": SNR = E[X^2] / E[(q(X) - X)^2]) and the
 // histogram of floor(log2 |x|) (appendix "Histograms of tensor-scaling within BERT").
 //
-// One pass over the tensor, HBM bound.  Every CTA accumulates its sums in double precision and its bin
+// One pass over the tensor (an analysis tool, not on the training path: element-wise loads and a per-element
+// shared-memory histogram update; no bandwidth figure is claimed for it).  Every CTA accumulates its sums in double precision and its bin
 // counts in shared-memory integers, and writes one partial record to the caller's workspace; a second,
 // single-CTA kernel adds the records in order.  No global atomics and nothing to zero beforehand: the
 // result is the same from run to run.

@@ -184,9 +184,15 @@ def test_scaled_cast_multiplies_in_float32():
 
 
 def test_folded_normal_mass_pin():
+    """The paper prints that about 90 % of a unit normal's mass lies in [2^-4, 2^1]: the oracle's exponent histogram of a
+    large unit-normal sample must put that share into the bins of exponents -4 .. 0, and the closed form agrees."""
+    rng = np.random.default_rng(1)
+    n = 400000
+    h = F.exponent_histogram(rng.standard_normal(n), -4, 5)
+    assert abs(h[1:6].sum() / n - GOLD["folded_normal_mass"]) < 0.01
     from scipy import special
     mass = special.erf(2 / np.sqrt(2)) - special.erf(2.0 ** -4 / np.sqrt(2))
-    assert abs(mass - GOLD["folded_normal_mass"]) < 0.01
+    assert abs(h[1:6].sum() / n - mass) < 3e-3
 
 
 def test_exponent_histogram_bins_by_floor_log2():
