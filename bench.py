@@ -61,6 +61,7 @@ def parse_args():
     ap.add_argument("--sustain-seconds", type=float, default=2.0, help="length of the sustained leg (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dp", action="store_true", help="token-sharded data parallelism: global beta_w and an all-reduce of the weight gradients every step (default: independent replicas)")
+    ap.add_argument("--dp-transport", default="f32", choices=["f32", "bf16", "e5m2"], help="with --dp: format the partial weight gradients travel in (f32 = all-reduce; bf16 / e5m2 = all-gather of unit-scaled partials, summed locally in float32 in rank order)")
     ap.add_argument("--one-stream", action="store_true", help="issue the step's GEMMs on one stream (no overlap of independent launches)")
     return ap.parse_args()
 
@@ -411,7 +412,11 @@ def run_ours(args, rank: int, world: int, local: int):
     for i in range(args.steps):
         graphs[i % 2].replay()
         if dp_on:
-            dp.allreduce_weight_grads([blocks[i % 2].dW1, blocks[i % 2].dW2])
+            grads = [blocks[i % 2].dW1, blocks[i % 2].dW2]
+            if args.dp_transport == "f32":
+                dp.allreduce_weight_grads(grads)
+            else:
+                dp.exchange_weight_grads(grads, grads, transport=args.dp_transport)
     e1.record()
     torch.cuda.synchronize()
     main_window = (w0, time.time())
@@ -562,7 +567,7 @@ def run_ours(args, rank: int, world: int, local: int):
         "vs_baseline": None, "dtype": {"fp8": "fp8_e4m3/e5m2 (fp32 accumulate)", "bf16": "bf16", "fp16": "fp16"}[args.operand],
         "data": "synthetic",
         "config": {"workload": "ffn_bert_large fwd+bwd: T=8192 tokens (16x512), d_model=1024, d_ff=4096, tau=0.5",
-                   "operand": args.operand, "replicas": world, "weight_gradient_allreduce": dp_on,
+                   "operand": args.operand, "replicas": world, "weight_gradient_allreduce": dp_on, "weight_gradient_transport": args.dp_transport if dp_on else None,
                    "l2": "two rotating input/buffer sets, ~0.45 GB touched per step (> 126 MB L2)",
                    "launch": f"one CUDA graph of {blocks[0].launches_per_step} kernels per step, "
                              + ("the last four GEMMs as one grouped launch" if blocks[0].grouped else

@@ -278,8 +278,8 @@ typedef enum { US_FN_GELU = 0, US_FN_RELU = 1, US_FN_TANH = 2, US_FN_SIGMOID = 3
  *                  on a 16-byte boundary: US_ERR_UNSUPPORTED / US_ERR_ALIGNMENT otherwise, and
  *                  nothing is launched.  Tensors must not overlap.
  *
- * Inputs may be F32, BF16 or F16; outputs any us_dtype (us_cast_fp8, us_cast_fp8_multi: E4M3
- * or E5M2 only).  0 <= tau <= 1.
+ * Inputs may be F32, BF16 or F16 (us_weighted_add also takes E4M3 / E5M2 inputs: partial results that travelled
+ * in 8 bits); outputs any us_dtype (us_cast_fp8, us_cast_fp8_multi: E4M3 or E5M2 only).  0 <= tau <= 1.
  */
 us_status us_gelu_fwd(const us_mat* H, float s_in, float alpha, const us_mat* A, void* stream);
 us_status us_gelu_bwd(const us_mat* H, const us_mat* dA, float s_in, float beta, const us_mat* dH,

@@ -72,7 +72,7 @@ __device__ __forceinline__ void load_vec(const void* p, int dt, float (&v)[N]) {
       float4 t = __ldg(q + i);
       v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
     }
-  } else {
+  } else if (dt == US_BF16 || dt == US_F16) {
     const uint4* q = reinterpret_cast<const uint4*>(p);
 #pragma unroll
     for (int i = 0; i < N / 8; ++i) {
@@ -82,6 +82,18 @@ __device__ __forceinline__ void load_vec(const void* p, int dt, float (&v)[N]) {
       for (int j = 0; j < 4; ++j) {
         float2 f = (dt == US_BF16) ? unpack_bf16x2(w[j]) : unpack_f16x2(w[j]);
         v[8 * i + 2 * j] = f.x; v[8 * i + 2 * j + 1] = f.y;
+      }
+    }
+  } else {                                             // FP8 codes, 16 per 16-byte vector (N a multiple of 16)
+    const uint4* q = reinterpret_cast<const uint4*>(p);
+#pragma unroll
+    for (int i = 0; i < N / 16; ++i) {
+      uint4 t = __ldg(q + i);
+      uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 lo = unpack_fp8x2((uint16_t)(w[j] & 0xffffu), dt == US_E5M2), hi = unpack_fp8x2((uint16_t)(w[j] >> 16), dt == US_E5M2);
+        v[16 * i + 4 * j] = lo.x; v[16 * i + 4 * j + 1] = lo.y; v[16 * i + 4 * j + 2] = hi.x; v[16 * i + 4 * j + 3] = hi.y;
       }
     }
   }

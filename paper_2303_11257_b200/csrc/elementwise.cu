@@ -283,11 +283,18 @@ extern "C" us_status us_cast_fp8_multi(int count, const us_mat* src, const float
 extern "C" us_status us_weighted_add(int count, const us_mat* src, const float* gamma, float alpha, const us_mat* out,
                                       void* stream) {
   if (count < 1 || count > kMultiMax || !src || !gamma || !out) return US_ERR_INVALID_ARG;
+  if (out->rows < 0 || out->cols < 0 || out->ld < out->cols || (out->rows * out->cols > 0 && !out->ptr)) return US_ERR_INVALID_ARG;
+  if (!is_dtype(out->dtype)) return US_ERR_UNSUPPORTED;
+  if (out->ptr && reinterpret_cast<uintptr_t>(out->ptr) % dtype_size(out->dtype)) return US_ERR_ALIGNMENT;
   WeightedAddArgs p{};
   bool vec = row_starts_aligned(out, false);
   for (int i = 0; i < count; ++i) {
-    us_status s = check_ew(&src[i], nullptr, out);
-    if (s != US_OK) return s;
+    // inputs may also be FP8 tensors (partial results that travelled in 8 bits): checked like an output dtype
+    const us_mat* m = &src[i];
+    if (m->rows < 0 || m->cols < 0 || m->ld < m->cols || m->rows != out->rows || m->cols != out->cols) return US_ERR_INVALID_ARG;
+    if (m->rows * m->cols > 0 && !m->ptr) return US_ERR_INVALID_ARG;
+    if (!is_dtype(m->dtype)) return US_ERR_UNSUPPORTED;
+    if (m->ptr && reinterpret_cast<uintptr_t>(m->ptr) % dtype_size(m->dtype)) return US_ERR_ALIGNMENT;
     p.src[i] = src[i].ptr; p.src_dt[i] = src[i].dtype; p.src_ld[i] = src[i].ld;
     p.coef[i] = alpha * gamma[i];
     vec = vec && row_starts_aligned(&src[i], false);

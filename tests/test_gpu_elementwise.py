@@ -147,3 +147,30 @@ def test_weighted_add_n(out_fmt, shape, ld):
     with pytest.raises(L.UnitScaleError) as e:
         L.us_weighted_add([torch.zeros((4, 8), device="cuda")] * 9, [1.0] * 9, 1.0, torch.zeros((4, 8), device="cuda"))
     assert e.value.status == 1
+
+
+@pytest.mark.parametrize("transport", ["e5m2", "e4m3", "bf16"])
+@pytest.mark.parametrize("world", [3, 10])
+def test_low_precision_gradient_exchange_arithmetic_on_device(transport, world):
+    """The pack and sum steps of the token-sharded weight-gradient exchange (dp.exchange_weight_grads), run on one GPU over
+    the partials of `world` stand-in ranks: packed codes bit-exact against the oracle's cast of scale * partial, the
+    float32 sum in rank order against the oracle's sum of the decoded codes (more than eight ranks continue from the
+    running sum)."""
+    from oracle import formats as F
+    from paper_2303_11257_b200 import dp, synth
+    fmt = F.FORMATS[transport]
+    rows, cols = 272, 304
+    scale = dp.transport_scale(world)
+    parts = [(synth.normal(71, r, (rows, cols)) * np.float32(world ** -0.5)).astype(np.float32) for r in range(world)]
+    packed = [dp._pack_device(torch.from_numpy(p).cuda(), scale, dp._TRANSPORT[transport][0]) for p in parts]
+    want_codes = [F.quantise_codes((p * np.float32(scale)).astype(np.float64), fmt) for p in parts]
+    for got, want in zip(packed, want_codes):
+        assert np.array_equal(U.codes_of(got), want)
+    out = torch.empty(rows, cols, device="cuda")
+    dp._sum_device(packed, 1.0 / scale, out)
+    ref = sum(F.decode(c, fmt) for c in want_codes) / scale
+    assert np.abs(out.cpu().numpy() - ref).max() <= 4e-7 * max(1.0, np.abs(ref).max()) * world
+    # single-process form of the public call: no collective, same arithmetic
+    res = torch.empty(rows, cols, device="cuda")
+    dp.exchange_weight_grads([torch.from_numpy(parts[0]).cuda()], [res], transport=transport)
+    assert np.abs(res.cpu().numpy() - F.decode(F.quantise_codes(parts[0].astype(np.float64), fmt), fmt)).max() <= 1e-6
