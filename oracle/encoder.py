@@ -9,7 +9,8 @@ weights, E5 gradients); the attention matmuls take 16-bit operands (att = "bf16"
 att = "fp8", FP8 operands like every other matmul (section "Experiments": all matmul inputs are
 quantised): Q, K, V and the softmax output P as E4, the gradients dC, dS and dQ, dK, dV as E5, while
 the softmax input S and the gradient dP of its output, which feed no matmul, stay in BF16.  Every
-stored intermediate is rounded to the format it is stored in.
+stored intermediate is rounded to the format it is stored in; with fused_scores the scores are not
+stored between the first matmul and the softmax and therefore not rounded.
 
 norm = "post" adds the post-norm arrangement of the appendix "Model architectures"
 (res^PostNorm(f, z) = layernorm(interp(z, f(z)))): each of the two residual sums goes through a scaled
@@ -61,9 +62,11 @@ def _unheads(H, nseq, slen, nhead, hd):
 
 
 def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16", norm=None, ln=None,
-                  eps=1e-5) -> EncoderResult:
+                  eps=1e-5, fused_scores=False) -> EncoderResult:
     """norm = None: R2 = res(ffn, res(attention, X)), G = dL/dR2 (the FFN block's output r.ffn.R).
-    norm = "post": ln = (w1, c1, w2, c2), each [d]; R1 = LN1(U1), R2 = LN2(U2) with U the residual sums."""
+    norm = "post": ln = (w1, c1, w2, c2), each [d]; R1 = LN1(U1), R2 = LN2(U2) with U the residual sums.
+    fused_scores: the scores S feed the softmax directly and are never stored, hence never rounded
+    (ops.attention_fwd); r.S then holds the unrounded scores."""
     T, d = X.shape
     hd = d // nhead
     f32 = lambda v: float(np.float32(v))
@@ -83,9 +86,13 @@ def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16"
     # ---- forward
     r.QKV, _ = O.store(O.linear_fwd(Xq, Wqkv_q, a_qkv), f_act)
     Q, K, V = (_heads(r.QKV, nseq, slen, nhead, hd, i, d) for i in range(3))
-    S4, _ = O.store(f32(a_s) * (Q @ K.transpose(0, 1, 3, 2)), f_wide)              # alpha Q K^T per (sequence, head)
-    P4, _ = O.store(O.softmax_fwd(S4, sm), f_act)
-    C4 = f32(a_c) * (P4 @ V)
+    if fused_scores:
+        S4 = f32(a_s) * (Q @ K.transpose(0, 1, 3, 2))
+        P4, C4 = O.attention_fwd(Q, K, V, a_s, sm, a_c, f_act)
+    else:
+        S4, _ = O.store(f32(a_s) * (Q @ K.transpose(0, 1, 3, 2)), f_wide)          # alpha Q K^T per (sequence, head)
+        P4, _ = O.store(O.softmax_fwd(S4, sm), f_act)
+        C4 = f32(a_c) * (P4 @ V)
     r.Cq, _ = O.store(_unheads(C4, nseq, slen, nhead, hd), "e4m3")
     r.S, r.P = S4.reshape(-1, slen), P4.reshape(-1, slen)
     ep = O.Epilogue(skip=np.asarray(X, np.float64), skip_coef=c_skip, out_coef=c_branch)

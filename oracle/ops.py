@@ -149,6 +149,25 @@ def softmax_bwd(P, dP, alpha, beta):
     return _f32(beta) * p * (dP - np.sum(p * dP, axis=-1, keepdims=True))
 
 
+# --------------------------------------------------------------------------- scaled dot-product attention
+
+def attention_fwd(Q, K, V, alpha_scores, softmax_scale, alpha_context, p_dtype: str):
+    """Scaled dot-product attention of one (sequence, head) problem with the scores kept unrounded
+    (appendix "Unit scaling and attention", paragraph "Softmax (followed by matmul)"):
+
+        S = alpha_scores * Q K^T            Q [s_q x d], K [s_k x d]          (never stored)
+        P = store(softmax_scale * softmax(S) over each row, p_dtype)          [s_q x s_k]
+        C = alpha_context * P V             V [s_k x d]                       [s_q x d]
+
+    P is a matmul input and is therefore rounded to its operand format before the second matmul; S
+    feeds no matmul and no memory, so it is not rounded at all.  Returns (P as stored, C unrounded).
+    Leading batch axes are allowed on all three operands."""
+    Q, K, V = (np.asarray(t, np.float64) for t in (Q, K, V))
+    S = _f32(alpha_scores) * (Q @ np.swapaxes(K, -1, -2))
+    P, _ = store(softmax_fwd(S, softmax_scale), p_dtype)
+    return P, _f32(alpha_context) * (P @ V)
+
+
 # --------------------------------------------------------------------------- softmax cross-entropy
 
 def softmax_xent_fwd(X, t):
