@@ -295,6 +295,40 @@ us_status us_cast_fp8(const us_mat* src, float scale, const us_mat* dst, void* s
 us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, const us_mat* dst,
                             void* stream);
 
+/* ------------------------------------------------------------ fused scaled dot-product attention (forward)
+ *
+ * Appendix "Unit scaling and attention" and paragraph "Softmax (followed by matmul)", for count[0] x
+ * count[1] independent (sequence, head) problems in one launch:
+ *
+ *   S = alpha_scores * Q K^T                       Q [s_q x 64], K [s_k x 64]; S is never stored and never rounded
+ *   P = softmax_scale * softmax(S), row by row     rounded to the operands' 16-bit format (it is a matmul input)
+ *   C = alpha_context * P V                        V [s_k x 64]; C [s_q x 64] rounded to C's dtype
+ *
+ * with alpha_scores = 1 / sqrt(64), softmax_scale = s_k and alpha_context = s_k^-1/2 for the
+ * unconstrained unit-scaled layer (us_scales_attention).  The us_mat arguments describe problem (0, 0);
+ * problem (i, j) of a tensor starts stride[0] * i + stride[1] * j elements further (heads are 64-column
+ * slices of a [tokens x 3 d] QKV matrix, C a 64-column slice of a [tokens x d] matrix).  P may be NULL;
+ * otherwise the rounded weights are also written to P [s_q x s_k] (the backward pass needs them).
+ * Q, K, V (and P): all BF16 or all F16, device memory; C: any us_dtype.  Head width must be 64 and
+ * s_k at most 512, else US_ERR_UNSUPPORTED; s_k = 0 with s_q > 0 is US_ERR_INVALID_ARG, s_q = 0 is
+ * a no-op.  Base addresses, row pitches and the strides of dimensions with count > 1 must be multiples
+ * of 16 bytes (US_ERR_ALIGNMENT); those strides must be positive and counts lie in 1..65535
+ * (US_ERR_INVALID_ARG).  Nothing is allocated and nothing owned; ws as for the linear ops (a wait that
+ * runs out inside the kernel raises US_ERR_TIMEOUT there).
+ */
+typedef struct {
+  int64_t count[2];      /* number of problems in the outer / inner batch dimension (>= 1 each) */
+  int64_t q_stride[2];   /* elements between consecutive problems, outer / inner */
+  int64_t k_stride[2];
+  int64_t v_stride[2];
+  int64_t c_stride[2];
+  int64_t p_stride[2];   /* ignored when P is NULL */
+} us_attention_batch;
+
+us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us_mat* V, float alpha_scores, float softmax_scale,
+                           float alpha_context, const us_mat* C, const us_mat* P, const us_attention_batch* batch,
+                           void* ws, size_t ws_bytes, void* stream);
+
 /* ------------------------------------------------------------ scaled softmax
  *
  * Row-wise scaled softmax and its gradient (table "Table of unit scaling factors", row softmax:

@@ -1,0 +1,319 @@
+// Fused scaled dot-product attention, forward (appendix "Unit scaling and attention"; paragraph
+// "Softmax (followed by matmul)"): per (sequence, head) problem
+//     S = alpha_scores * Q K^T,   P = softmax_scale * softmax(S) per row,   C = alpha_context * P V
+// in ONE kernel.  A CTA owns 128 query rows of one problem and all of its (at most 512) keys:
+//   * Q [128 x 64] and K [<=512 x 64] arrive by TMA (128-byte swizzle), V [<=512 x 64] behind them;
+//   * tcgen05.mma (kind::f16, M = 128, N = 256, twice) leaves the whole score block, 128 x 512
+//     float32, in tensor memory (all 512 columns): the scores never reach shared or global memory
+//     and are never rounded;
+//   * four warps (one TMEM lane = one query row per thread) make three passes over their row in
+//     tensor memory: maximum; sum of exponentials; weights, scaled, rounded to the operand format and
+//     written to shared memory in the K-major swizzled layout of an MMA A operand, over the bytes Q
+//     and K occupied (both are dead by then);
+//   * a second chain of MMAs (M = 128, N = 64, K = keys) multiplies the weights by V into tensor
+//     memory columns 0..63 (the scores are dead by then); the same shared-memory tiles leave by TMA
+//     store as the stored P the backward pass needs;
+//   * the four warps scale the context and store it in the output format.
+// Every wait on an mbarrier is bounded; a wait that runs out raises the status word (as in the GEMM
+// kernels) and the CTA leaves after its own copies have landed and its tensor memory is freed.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "../../include/unitscale.h"
+#include "common.cuh"
+#include "gemm_kernel.cuh"
+#include "host.h"
+#include "sm100.cuh"
+
+namespace us {
+namespace {
+
+constexpr int kAttnD = 64;                 // head width
+constexpr int kAttnMaxKeys = 512;          // 128 x 512 float32 scores fill the 512 TMEM columns
+constexpr int kAttnThreads = 192;          // warp 0: TMA + MMA issue; warp 1: TMEM owner; warps 2-5: softmax
+constexpr uint32_t kQBytes = 128 * 128;    // 128 rows x 64 x 2 bytes
+constexpr uint32_t kKeyBlockBytes = 128 * 128;   // P tile of one 64-key block: 128 rows x 128 bytes
+constexpr uint32_t kPBytes = 8 * kKeyBlockBytes; // 128 KB; Q and K (16 + 64 KB) live in its first 80 KB until the scores exist
+constexpr uint32_t kVBytes = 512 * 128;
+constexpr uint32_t kAttnSmem = kPBytes + kVBytes + 1024 /* alignment */ + 128 /* barriers, slots */;
+
+struct AttnParams {
+  int s_q, s_k;
+  float exp_scale;          // alpha_scores * log2(e)
+  float softmax_scale;
+  float alpha_context;
+  void* c; int c_dt; int64_t c_ld, c_stride0, c_stride1;
+  int op_bf16;              // operands (and stored P) are BF16 (1) or F16 (0)
+  int store_p;
+  uint32_t idesc_s, idesc_c;
+  unsigned int* status;
+  uint32_t wait_limit;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_constant__ CUtensorMap tk,
+                     const __grid_constant__ CUtensorMap tv, const __grid_constant__ CUtensorMap tp, const AttnParams a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - ptx::smem_addr(smem_raw));
+  const uint32_t q_s = base, k_s = base + kQBytes, p_s = base, v_s = base + kPBytes;
+  const uint32_t bars = v_s + kVBytes;
+  const uint32_t bar_qk = bars, bar_v = bars + 8, bar_s = bars + 16, bar_p = bars + 24, bar_o = bars + 32;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kPBytes + kVBytes + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kPBytes + kVBytes + 68);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q0 = blockIdx.x * 128, b1 = blockIdx.y, b0 = blockIdx.z;
+  const int nkb = (a.s_k + 63) >> 6;                 // 64-key blocks with at least one key
+  const bool two_halves = a.s_k > 256;
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar_qk, 1); ptx::mbar_init(bar_v, 1); ptx::mbar_init(bar_s, 1);
+    ptx::mbar_init(bar_p, 4); ptx::mbar_init(bar_o, 1);
+    *abort_flag = 0;
+    ptx::mbar_init_fence();
+  }
+  if (warp == 1) { ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), 512); ptx::tmem_relinquish(); }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- loads
+      ptx::mbar_expect_tx(bar_qk, kQBytes + (two_halves ? 2u : 1u) * 256u * 128u);
+      ptx::tma_load_4d(q_s, &tq, bar_qk, 0, q0, b1, b0);
+      ptx::tma_load_4d(k_s, &tk, bar_qk, 0, 0, b1, b0);
+      if (two_halves) ptx::tma_load_4d(k_s + 256u * 128u, &tk, bar_qk, 0, 256, b1, b0);
+      ptx::mbar_expect_tx(bar_v, (two_halves ? 2u : 1u) * 256u * 128u);
+      ptx::tma_load_4d(v_s, &tv, bar_v, 0, 0, b1, b0);
+      if (two_halves) ptx::tma_load_4d(v_s + 256u * 128u, &tv, bar_v, 0, 256, b1, b0);
+      // ---------------------------------------------------------------- S = Q K^T
+      bool ok = wait_bounded(bar_qk, 0, abort_flag, a.status, a.wait_limit);
+      if (ok) {
+        ptx::tc_fence_after_sync();
+        const uint64_t qd = ptx::smem_desc_sw128(q_s, 16, 1024);
+        for (int h = 0; h < (two_halves ? 2 : 1); ++h) {
+          const uint64_t kd = ptx::smem_desc_sw128(k_s + (uint32_t)h * 256u * 128u, 16, 1024);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)                     // 16 of the 64 head columns (32 bytes) per MMA
+            ptx::mma_ss<false>(tmem + 256u * h, qd + 2u * k, kd + 2u * k, a.idesc_s, k > 0);
+        }
+        ptx::mma_commit(bar_s);
+        // -------------------------------------------------------------- C = P V once the weights are in shared memory
+        ok = wait_bounded(bar_p, 0, abort_flag, a.status, a.wait_limit) &&
+             wait_bounded(bar_v, 0, abort_flag, a.status, a.wait_limit);
+      }
+      if (ok) {
+        ptx::tc_fence_after_sync();
+        for (int kb = 0; kb < nkb; ++kb) {
+          const uint64_t pd = ptx::smem_desc_sw128(p_s + (uint32_t)kb * kKeyBlockBytes, 16, 1024);
+          const uint64_t vd = ptx::smem_desc_sw128(v_s + (uint32_t)kb * 8192u, 8192, 1024);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)                     // 16 keys per MMA: 32 bytes along a P row, 16 rows of V
+            ptx::mma_ss<false>(tmem, pd + 2u * k, vd + 128u * k, a.idesc_c, (kb | k) != 0);
+        }
+        ptx::mma_commit(bar_o);
+        if (a.store_p) {
+          for (int kb = 0; kb < nkb; ++kb)
+            ptx::tma_store_4d(&tp, p_s + (uint32_t)kb * kKeyBlockBytes, kb * 64, q0, b1, b0);
+          ptx::bulk_commit_group();
+        }
+      }
+      if (*abort_flag) {
+        // loads that were issued land before the CTA gives up its shared memory
+        for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_qk, 0); ++it) {}
+        for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_v, 0); ++it) {}
+      }
+      ptx::bulk_wait_group_read<0>();                      // the stored P has left shared memory
+    }
+  } else if (warp >= 2) {
+    // ------------------------------------------------------------------ softmax and output, one query row per thread
+    const int q = warp & 3, r = q * 32 + lane;              // TMEM lane quarter of this warp; row within the tile
+    const uint32_t t_row = tmem + ((uint32_t)(q * 32) << 16);
+    bool ok = wait_bounded(bar_s, 0, abort_flag, a.status, a.wait_limit);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      ptx::tc_fence_after_sync();
+      const int nchunk = 2 * nkb;                           // 32-column chunks, whole key blocks
+      float v[32];
+      float m = -3.0e38f;
+      // columns at and beyond s_k hold products with zero-filled key rows: they are kept out of the maximum and
+      // the sum by replacing them with a very negative score, whose weight is exactly zero
+      auto load_chunk = [&](int c) {
+        ptx::tmem_ld_32x32(t_row + 32u * c, v);
+        if (32 * c + 32 > a.s_k) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) if (32 * c + i >= a.s_k) v[i] = -3.0e38f;
+        }
+      };
+      for (int c = 0; c < nchunk; ++c) {
+        load_chunk(c);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) m = fmaxf(m, v[i]);
+      }
+      const float mk = m * a.exp_scale;
+      float sum = 0.f;
+      for (int c = 0; c < nchunk; ++c) {
+        load_chunk(c);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) sum += ex2(fmaf(v[i], a.exp_scale, -mk));
+      }
+      const float inv = a.softmax_scale / sum;
+      const uint32_t row_off = (uint32_t)r * 128u, sw = (uint32_t)(r & 7);
+      for (int c = 0; c < nchunk; ++c) {
+        load_chunk(c);
+        const uint32_t blk = p_s + (uint32_t)(c >> 1) * kKeyBlockBytes + row_off;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint32_t w[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float p0 = ex2(fmaf(v[8 * g + 2 * j], a.exp_scale, -mk)) * inv;       // masked columns: ex2(-huge) = 0
+            const float p1 = ex2(fmaf(v[8 * g + 2 * j + 1], a.exp_scale, -mk)) * inv;
+            w[j] = a.op_bf16 ? pack_bf16x2(p0, p1) : pack_f16x2(p0, p1);
+          }
+          const uint32_t chunk16 = (uint32_t)((c & 1) * 4 + g);
+          ptx::sts128(blk + ((chunk16 ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+        }
+      }
+      ptx::fence_proxy_async_smem();                         // the MMA and the TMA store read these bytes
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_p);
+      // ---------------------------------------------------------------- context
+      ok = wait_bounded(bar_o, 0, abort_flag, a.status, a.wait_limit);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        ptx::tc_fence_after_sync();
+        const int row = q0 + r;
+        char* dst = static_cast<char*>(a.c) + ((int64_t)b0 * a.c_stride0 + (int64_t)b1 * a.c_stride1 + (int64_t)row * a.c_ld) *
+                                                  dtype_size(a.c_dt);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          ptx::tmem_ld_32x32(t_row + 32u * h, v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] *= a.alpha_context;
+          if (row < a.s_q) store_vec<32>(dst + 32 * h * dtype_size(a.c_dt), a.c_dt, v);
+        }
+      }
+    }
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) { ptx::tc_fence_after_sync(); ptx::tmem_dealloc(tmem, 512); }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn attn_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+// 4-d map (column, row, inner problem index, outer problem index) over 16-bit elements; box of 64 columns
+// (128 bytes, 128-byte swizzle) x box_rows rows of one problem.
+static bool attn_tmap(CUtensorMap* tm, const us_mat* m, const int64_t* stride, const int64_t* count, int box_rows) {
+  EncodeTiledFn fn = attn_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)m->cols, (cuuint64_t)m->rows, (cuuint64_t)count[1], (cuuint64_t)count[0]};
+  // a dimension of extent 1 still needs a valid (multiple of 16 bytes) stride
+  const cuuint64_t s1 = count[1] > 1 ? (cuuint64_t)stride[1] * 2 : 16, s0 = count[0] > 1 ? (cuuint64_t)stride[0] * 2 : 16;
+  cuuint64_t strides[3] = {(cuuint64_t)m->ld * 2, s1, s0};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, m->ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static bool ok16(const us_mat* m, const int64_t* stride, const int64_t* count, int es) {
+  if (reinterpret_cast<uintptr_t>(m->ptr) % 16 || (m->ld * es) % 16) return false;
+  for (int i = 0; i < 2; ++i)
+    if (count[i] > 1 && (stride[i] * es) % 16) return false;
+  return true;
+}
+
+}  // namespace
+}  // namespace us
+
+extern "C" us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us_mat* V, float alpha_scores,
+                                      float softmax_scale, float alpha_context, const us_mat* C, const us_mat* P,
+                                      const us_attention_batch* batch, void* ws, size_t ws_bytes, void* stream) {
+  using namespace us;
+  if (!Q || !K || !V || !C || !batch) return US_ERR_INVALID_ARG;
+  const int64_t* cnt = batch->count;
+  if (cnt[0] < 1 || cnt[1] < 1 || cnt[0] > 65535 || cnt[1] > 65535) return US_ERR_INVALID_ARG;
+  const us_mat* all[5] = {Q, K, V, C, P};
+  for (int i = 0; i < 5; ++i) {
+    const us_mat* m = all[i];
+    if (!m) continue;
+    if (m->rows < 0 || m->cols < 0 || m->ld < m->cols) return US_ERR_INVALID_ARG;
+    if (m->rows * m->cols > 0 && !m->ptr) return US_ERR_INVALID_ARG;
+  }
+  const int64_t s_q = Q->rows, s_k = K->rows;
+  if (K->cols != Q->cols || V->cols != Q->cols || V->rows != s_k || C->rows != s_q || C->cols != Q->cols)
+    return US_ERR_INVALID_ARG;
+  if (P && (P->rows != s_q || P->cols != s_k)) return US_ERR_INVALID_ARG;
+  if (!(alpha_scores > 0.f) || !(softmax_scale > 0.f)) return US_ERR_INVALID_ARG;
+  const int64_t* strides[5] = {batch->q_stride, batch->k_stride, batch->v_stride, batch->c_stride, batch->p_stride};
+  for (int i = 0; i < 5; ++i)
+    for (int j = 0; j < 2; ++j)
+      if (all[i] && cnt[j] > 1 && strides[i][j] <= 0) return US_ERR_INVALID_ARG;
+  const bool h16 = (Q->dtype == US_BF16 || Q->dtype == US_F16) && K->dtype == Q->dtype && V->dtype == Q->dtype;
+  if (!h16 || (P && P->dtype != Q->dtype)) return US_ERR_UNSUPPORTED;
+  if (C->dtype < US_F32 || C->dtype > US_E5M2) return US_ERR_UNSUPPORTED;
+  if (Q->cols != kAttnD || s_k > kAttnMaxKeys) return US_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < us_workspace_bytes()) return US_ERR_WORKSPACE;
+  if (s_q == 0 || s_k == 0) return s_k == 0 && s_q > 0 ? US_ERR_INVALID_ARG : US_OK;   // a softmax over no keys is undefined
+  const int c_es = (int)dtype_size(C->dtype);
+  if (!ok16(Q, batch->q_stride, cnt, 2) || !ok16(K, batch->k_stride, cnt, 2) || !ok16(V, batch->v_stride, cnt, 2) ||
+      !ok16(C, batch->c_stride, cnt, c_es) || (P && !ok16(P, batch->p_stride, cnt, 2)))
+    return US_ERR_ALIGNMENT;
+
+  CUtensorMap tq, tk, tv, tp;
+  if (!attn_tmap(&tq, Q, batch->q_stride, cnt, 128) || !attn_tmap(&tk, K, batch->k_stride, cnt, 256) ||
+      !attn_tmap(&tv, V, batch->v_stride, cnt, 256))
+    return US_ERR_CUDA;
+  tp = tq;
+  if (P && !attn_tmap(&tp, P, batch->p_stride, cnt, 128)) return US_ERR_CUDA;
+
+  AttnParams a{};
+  a.s_q = (int)s_q; a.s_k = (int)s_k;
+  a.exp_scale = alpha_scores * 1.4426950408889634f;
+  a.softmax_scale = softmax_scale;
+  a.alpha_context = alpha_context;
+  a.c = C->ptr; a.c_dt = C->dtype; a.c_ld = C->ld;
+  a.c_stride0 = cnt[0] > 1 ? batch->c_stride[0] : 0; a.c_stride1 = cnt[1] > 1 ? batch->c_stride[1] : 0;
+  a.op_bf16 = Q->dtype == US_BF16;
+  a.store_p = P != nullptr;
+  const int fmt = a.op_bf16 ? 1 : 0;
+  a.idesc_s = make_idesc(fmt, fmt, false, false, 128, 256);
+  a.idesc_c = make_idesc(fmt, fmt, false, true, 128, 64);
+  a.status = static_cast<unsigned int*>(ws);
+  a.wait_limit = kWaitLimit;
+
+  if (cudaFuncSetAttribute(attention_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmem) != cudaSuccess)
+    return US_ERR_CUDA;
+  const dim3 grid((unsigned)((s_q + 127) / 128), (unsigned)cnt[1], (unsigned)cnt[0]);
+  attention_fwd_kernel<<<grid, kAttnThreads, kAttnSmem, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, tp, a);
+  return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
+}

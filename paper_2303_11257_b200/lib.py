@@ -42,6 +42,11 @@ class us_batch(C.Structure):
     _fields_ = [("count", C.c_int64 * 2), ("a_stride", C.c_int64 * 2), ("b_stride", C.c_int64 * 2), ("out_stride", C.c_int64 * 2)]
 
 
+class us_attention_batch(C.Structure):
+    _fields_ = [("count", C.c_int64 * 2), ("q_stride", C.c_int64 * 2), ("k_stride", C.c_int64 * 2),
+                ("v_stride", C.c_int64 * 2), ("c_stride", C.c_int64 * 2), ("p_stride", C.c_int64 * 2)]
+
+
 class us_linear_call(C.Structure):
     _fields_ = [("op", C.c_int32), ("a", us_mat), ("b", us_mat), ("scale", C.c_float), ("ep", us_epilogue), ("out", us_mat)]
 
@@ -75,6 +80,8 @@ def _load() -> C.CDLL:
         fn = getattr(lib, name)
         fn.argtypes = [MP, MP, F, MP, C.POINTER(us_batch), V, SZ, V]
         fn.restype = C.c_int
+    lib.us_attention_fwd.argtypes = [MP, MP, MP, F, F, F, MP, MP, C.POINTER(us_attention_batch), V, SZ, V]
+    lib.us_attention_fwd.restype = C.c_int
     lib.us_linear_fwd_static_ws.argtypes = [MP, MP, F, EP, MP, C.POINTER(C.c_void_p), V]
     lib.us_linear_fwd_static_ws.restype = C.c_int
     lib.us_linear_fwd_check.argtypes = [MP, MP, EP, MP, V, SZ]
@@ -248,6 +255,26 @@ def us_linear_bwd_x_batched(G, W, beta_x, dX, bt, ws, stream=None):
 
 def us_linear_bwd_w_batched(X, G, beta_w, dW, bt, ws, stream=None):
     return _linear_batched("us_linear_bwd_w_batched", X, G, beta_w, dW, bt, ws, stream)
+
+
+def attention_batch(count, q_stride, k_stride, v_stride, c_stride, p_stride=(0, 0)) -> us_attention_batch:
+    """us_attention_batch from (outer, inner) pairs of counts and element strides."""
+    b = us_attention_batch()
+    for i in range(2):
+        b.count[i] = count[i]
+        b.q_stride[i], b.k_stride[i], b.v_stride[i] = q_stride[i], k_stride[i], v_stride[i]
+        b.c_stride[i], b.p_stride[i] = c_stride[i], p_stride[i]
+    return b
+
+
+def us_attention_fwd(Q, K, V, alpha_scores, softmax_scale, alpha_context, Cx, P, bt, ws, stream=None):
+    """Fused scaled dot-product attention forward; P may be None (weights not stored)."""
+    pp = C.byref(mat(P)) if P is not None else None
+    _check("us_attention_fwd",
+           _lib.us_attention_fwd(C.byref(mat(Q)), C.byref(mat(K)), C.byref(mat(V)), alpha_scores, softmax_scale,
+                                 alpha_context, C.byref(mat(Cx)), pp, C.byref(bt), ws.data_ptr(),
+                                 ws.numel() * ws.element_size(), _stream(stream)))
+    return Cx
 
 
 def us_linear_fwd_static_ws(X, W, alpha, Y, ep=None, stream=None) -> int:

@@ -1,0 +1,145 @@
+"""Fused scaled dot-product attention forward (us_attention_fwd) against the oracle, element by element.
+
+The weights P are compared with ops.attention_fwd evaluated on the operands the device holds (16-bit
+output: within one ulp plus 3e-6 of the row scale, the allowance of the stand-alone softmax tests); the
+context C is compared with alpha_context * P V evaluated on the device's OWN stored weights, so that a
+legitimate one-ulp difference in a weight does not leak into the second check (2e-3 at unit scale, one ulp /
+one FP8 code of the output format on top).  Problems are strided head slices of a [tokens x 3 d] matrix as in
+the encoder layer, with ragged lengths, one and two halves of keys, and every output format of C."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import formats as F
+from oracle import ops as O
+from tests import util as U
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-3
+
+
+def _run(nseq, nhead, s, fmt, c_fmt, seed, store_p=True, scale=1.0):
+    from paper_2303_11257_b200 import lib as L, synth
+    hd, d, T = 64, nhead * 64, nseq * s
+    qkv = scale * synth.normal(seed, 0, (T, 3 * d))
+    QKV = U.to_device(qkv, fmt)
+    qkv_v = U.values_of(qkv, fmt)
+    Cx = U.empty(T, d, c_fmt)
+    P = U.empty(nseq * nhead * s, s, fmt) if store_p else None
+    ws = L.new_workspace()
+    a_s, sm, a_c = hd ** -0.5, float(s), s ** -0.5
+    st = (s * 3 * d, hd)
+    bt = L.attention_batch((nseq, nhead), st, st, st, (s * d, hd), (nhead * s * s, s * s))
+    L.us_attention_fwd(QKV[:s, 0:hd], QKV[:s, d:d + hd], QKV[:s, 2 * d:2 * d + hd], a_s, sm, a_c,
+                       Cx[:s, :hd], P[:s] if store_p else None, bt, ws)
+    assert L.us_workspace_status(ws) == 0
+    return qkv_v, Cx, P, (a_s, sm, a_c)
+
+
+def _heads(M, nseq, s, nhead, which):
+    d = nhead * 64
+    return M[:, which * d:(which + 1) * d].reshape(nseq, s, nhead, 64).transpose(0, 2, 1, 3)
+
+
+def _check_c(Cx, c_ref, c_fmt, nseq, s, nhead):
+    ref = c_ref.transpose(0, 2, 1, 3).reshape(nseq * s, nhead * 64)
+    got = U.host_values(Cx)
+    tol = TOL * max(1.0, np.abs(ref).max())
+    if c_fmt in ("e4m3", "e5m2"):
+        fm = F.FORMATS[c_fmt]
+        dist = U.code_distance(F.quantise_codes(got, fm), F.quantise_codes(ref, fm), c_fmt)
+        ok = (dist <= 1) | (np.abs(got - F.quantise(ref, fm)) <= tol)
+        assert ok.all(), f"C: code distance {dist.max()} at {(~ok).sum()} places"
+    else:
+        lim = tol + (U.ulp_of(ref, c_fmt) if c_fmt != "f32" else 0.0)
+        err = np.abs(got - ref)
+        assert (err <= lim).all(), f"C: {(err > lim).sum()} elements out, worst {err.max():.3e}"
+
+
+@pytest.mark.parametrize("fmt", ["bf16", "fp16"])
+@pytest.mark.parametrize("nseq,nhead,s", [(2, 3, 128), (1, 2, 200), (2, 2, 512), (1, 1, 72), (1, 2, 264), (3, 1, 8)])
+def test_weights_and_context_against_the_oracle(fmt, nseq, nhead, s):
+    c_fmt = "e4m3"
+    qkv_v, Cx, P, (a_s, sm, a_c) = _run(nseq, nhead, s, fmt, c_fmt, seed=61)
+    Q, K, V = (_heads(qkv_v, nseq, s, nhead, i) for i in range(3))
+    p_ref, _ = O.attention_fwd(Q, K, V, a_s, sm, a_c, "f64")            # unrounded weights
+    p_dev = U.host_values(P).reshape(nseq, nhead, s, s)
+    lim = U.ulp_of(p_ref, fmt) + 3e-6 * sm
+    err = np.abs(p_dev - p_ref)
+    assert (err <= lim).all(), f"P: {(err > lim).sum()} elements beyond one ulp, worst {err.max():.3e}"
+    assert np.allclose(p_dev.sum(axis=-1), sm, rtol=4e-3)                # rows of s * softmax sum to s
+    _check_c(Cx, np.float64(np.float32(a_c)) * (p_dev @ V), c_fmt, nseq, s, nhead)
+
+
+@pytest.mark.parametrize("c_fmt", ["f32", "bf16", "fp16", "e4m3", "e5m2"])
+def test_every_context_format_and_weights_not_stored(c_fmt):
+    nseq, nhead, s = 2, 2, 192
+    qkv_v, Cx, P, (a_s, sm, a_c) = _run(nseq, nhead, s, "bf16", c_fmt, seed=62, store_p=False)
+    Q, K, V = (_heads(qkv_v, nseq, s, nhead, i) for i in range(3))
+    p_ref, c_ref = O.attention_fwd(Q, K, V, a_s, sm, a_c, "bf16")
+    # without the device's weights at hand, allow for one-ulp differences in them: sum_j ulp(p_j) |v_j| * alpha_c
+    slack = np.float64(np.float32(a_c)) * (U.ulp_of(p_ref, "bf16") @ np.abs(V))
+    ref = c_ref.transpose(0, 2, 1, 3).reshape(nseq * s, nhead * 64)
+    got = U.host_values(Cx)
+    lim = TOL + 0.05 * slack.transpose(0, 2, 1, 3).reshape(ref.shape) + \
+        (U.ulp_of(ref, c_fmt) if c_fmt != "f32" else 0.0)
+    err = np.abs(got - ref)
+    assert (err <= lim).all(), f"C ({c_fmt}): {(err > lim).sum()} out, worst {err.max():.3e}"
+
+
+def test_peaked_rows_large_scores():
+    """Scores of standard deviation ~8: rows dominated by one key, weights from 0 to several hundred."""
+    nseq, nhead, s = 1, 2, 320
+    qkv_v, Cx, P, (a_s, sm, a_c) = _run(nseq, nhead, s, "bf16", "bf16", seed=63, scale=2.8)
+    Q, K, V = (_heads(qkv_v, nseq, s, nhead, i) for i in range(3))
+    p_ref, _ = O.attention_fwd(Q, K, V, a_s, sm, a_c, "f64")
+    p_dev = U.host_values(P).reshape(nseq, nhead, s, s)
+    assert p_ref.max() > 100
+    # exp of a float32 argument of magnitude up to ~60: relative error up to 60 * 2^-23
+    lim = U.ulp_of(p_ref, "bf16") + 3e-6 * sm + 1.5e-5 * p_ref
+    assert (np.abs(p_dev - p_ref) <= lim).all()
+    _check_c(Cx, np.float64(np.float32(a_c)) * (p_dev @ V), "bf16", nseq, s, nhead)
+
+
+def test_bert_large_attention_shape_sampled_problems():
+    """16 sequences x 16 heads x 512 tokens: first / last and sampled (sequence, head) problems in full."""
+    nseq, nhead, s = 16, 16, 512
+    qkv_v, Cx, P, (a_s, sm, a_c) = _run(nseq, nhead, s, "bf16", "e4m3", seed=64)
+    rng = np.random.default_rng(5)
+    probs = [(0, 0), (0, 15), (15, 0), (15, 15)] + [(int(rng.integers(16)), int(rng.integers(16))) for _ in range(6)]
+    Cv = U.host_values(Cx)
+    for (i, j) in probs:
+        r = slice(i * s, (i + 1) * s)
+        q, k, v = (qkv_v[r, o * 1024 + j * 64:o * 1024 + (j + 1) * 64] for o in range(3))
+        p_ref, _ = O.attention_fwd(q, k, v, a_s, sm, a_c, "f64")
+        p_dev = U.host_values(P[(i * nhead + j) * s:(i * nhead + j + 1) * s])
+        assert (np.abs(p_dev - p_ref) <= U.ulp_of(p_ref, "bf16") + 3e-6 * sm).all(), (i, j)
+        ref = np.float64(np.float32(a_c)) * (p_dev @ v)
+        fm = F.FORMATS["e4m3"]
+        got = Cv[r, j * 64:(j + 1) * 64]
+        dist = U.code_distance(F.quantise_codes(got, fm), F.quantise_codes(ref, fm), "e4m3")
+        ok = (dist <= 1) | (np.abs(got - F.quantise(ref, fm)) <= TOL * max(1.0, np.abs(ref).max()))
+        assert ok.all(), (i, j, dist.max())
+
+
+def test_argument_checks():
+    from paper_2303_11257_b200 import lib as L
+    ws = L.new_workspace()
+    q = U.empty(128, 64, "bf16"); k = U.empty(128, 64, "bf16"); c = U.empty(128, 64, "bf16")
+    bt = L.attention_batch((1, 1), (0, 0), (0, 0), (0, 0), (0, 0))
+    wide = U.empty(128, 128, "bf16")
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_attention_fwd(wide, wide, wide, 0.125, 128.0, 0.1, wide, None, bt, ws)
+    assert e.value.status == L.US_ERR_UNSUPPORTED                    # head width 128
+    k_long = U.empty(640, 64, "bf16")
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_attention_fwd(q, k_long, k_long, 0.125, 640.0, 0.1, c, None, bt, ws)
+    assert e.value.status == L.US_ERR_UNSUPPORTED                    # more than 512 keys
+    q8 = U.empty(128, 64, "e4m3")
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_attention_fwd(q8, q8, q8, 0.125, 128.0, 0.1, c, None, bt, ws)
+    assert e.value.status == L.US_ERR_UNSUPPORTED                    # FP8 operands
+    with pytest.raises(L.UnitScaleError) as e:
+        L.us_attention_fwd(q, k, U.empty(64, 64, "bf16"), 0.125, 128.0, 0.1, c, None, bt, ws)
+    assert e.value.status == L.US_ERR_INVALID_ARG                    # V rows != K rows
+    L.us_attention_fwd(q[:0], k, k, 0.125, 128.0, 0.1, c[:0], None, bt, ws)   # no queries: nothing to do
