@@ -655,11 +655,11 @@ def run_encoder(args, rank, world, local, torch, dev, peaks):
     sampler.start()
     results = {}
     windows = []
-    for attention in ("bf16", "fp8"):
+    for name, attention, fused in (("bf16", "bf16", False), ("fp8", "fp8", False), ("bf16, fused forward attention", "bf16", True)):
         host = (synth.normal(0, 0, (T, d)), synth.normal(0, 1, (d, 3 * d)), synth.normal(0, 2, (d, d)),
                 synth.normal(0, 3, (d, d_ff)), synth.normal(0, 4, (d_ff, d)), synth.normal(0, 5, (T, d)))
         tensors = [torch.from_numpy(t).to(dev) for t in host]
-        layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, d_ff, attention=attention, device=dev)
+        layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, d_ff, attention=attention, device=dev, fused_attention=fused)
         layer.step(*tensors)
         layer.check()
         g = torch.cuda.CUDAGraph()
@@ -678,7 +678,7 @@ def run_encoder(args, rank, world, local, torch, dev, peaks):
         windows.append((w0, time.time()))
         layer.check()
         ms = e0.elapsed_time(e1) / args.steps
-        results[attention] = {"ms_per_step": ms, "tflops": layer.flops() / (ms * 1e-3) / 1e12, "launches": layer.launches_per_step,
+        results[name] = {"ms_per_step": ms, "tflops": layer.flops() / (ms * 1e-3) / 1e12, "launches": layer.launches_per_step,
                               "tokens_per_s": T / (ms * 1e-3)}
         flops = layer.flops()
         del layer, g

@@ -6,14 +6,15 @@
 //   * tcgen05.mma (kind::f16, M = 128, N = 256, twice) leaves the whole score block, 128 x 512
 //     float32, in tensor memory (all 512 columns): the scores never reach shared or global memory
 //     and are never rounded;
-//   * four warps (one TMEM lane = one query row per thread) make three passes over their row in
-//     tensor memory: maximum; sum of exponentials; weights, scaled, rounded to the operand format and
-//     written to shared memory in the K-major swizzled layout of an MMA A operand, over the bytes Q
-//     and K occupied (both are dead by then);
+//   * eight warps (two per TMEM lane quarter, one query row per lane, alternate 32-column chunks each)
+//     make three passes over their rows in tensor memory: maximum; exponentials, written back over the
+//     scores (tcgen05.st), and their sum; weights, scaled, rounded to the operand format and written
+//     to shared memory in the K-major swizzled layout of an MMA A operand, over the bytes Q and K
+//     occupied (both are dead by then);
 //   * a second chain of MMAs (M = 128, N = 64, K = keys) multiplies the weights by V into tensor
 //     memory columns 0..63 (the scores are dead by then); the same shared-memory tiles leave by TMA
 //     store as the stored P the backward pass needs;
-//   * the four warps scale the context and store it in the output format.
+//   * the eight warps scale the context and store it in the output format.
 // Every wait on an mbarrier is bounded; a wait that runs out raises the status word (as in the GEMM
 // kernels) and the CTA leaves after its own copies have landed and its tensor memory is freed.
 #include <cuda.h>
@@ -32,12 +33,13 @@ namespace {
 
 constexpr int kAttnD = 64;                 // head width
 constexpr int kAttnMaxKeys = 512;          // 128 x 512 float32 scores fill the 512 TMEM columns
-constexpr int kAttnThreads = 192;          // warp 0: TMA + MMA issue; warp 1: TMEM owner; warps 2-5: softmax
+constexpr int kSoftmaxWarps = 8;
+constexpr int kAttnThreads = 64 + 32 * kSoftmaxWarps;   // warp 0: TMA + MMA issue; warp 1: TMEM owner; warps 2-9: softmax
 constexpr uint32_t kQBytes = 128 * 128;    // 128 rows x 64 x 2 bytes
 constexpr uint32_t kKeyBlockBytes = 128 * 128;   // P tile of one 64-key block: 128 rows x 128 bytes
 constexpr uint32_t kPBytes = 8 * kKeyBlockBytes; // 128 KB; Q and K (16 + 64 KB) live in its first 80 KB until the scores exist
 constexpr uint32_t kVBytes = 512 * 128;
-constexpr uint32_t kAttnSmem = kPBytes + kVBytes + 1024 /* alignment */ + 128 /* barriers, slots */;
+constexpr uint32_t kAttnSmem = kPBytes + kVBytes + 1024 /* alignment */ + 128 /* barriers, slots */ + 2048 /* row maxima and sums */;
 
 struct AttnParams {
   int s_q, s_k;
@@ -69,6 +71,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
   const uint32_t bar_qk = bars, bar_v = bars + 8, bar_s = bars + 16, bar_p = bars + 24, bar_o = bars + 32;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kPBytes + kVBytes + 64);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kPBytes + kVBytes + 68);
+  volatile float* row_max = reinterpret_cast<volatile float*>(gen + kPBytes + kVBytes + 128);   // [2][128]
+  volatile float* row_sum = row_max + 256;                                                        // [2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * 128, b1 = blockIdx.y, b0 = blockIdx.z;
@@ -77,7 +81,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
 
   if (threadIdx.x == 0) {
     ptx::mbar_init(bar_qk, 1); ptx::mbar_init(bar_v, 1); ptx::mbar_init(bar_s, 1);
-    ptx::mbar_init(bar_p, 4); ptx::mbar_init(bar_o, 1);
+    ptx::mbar_init(bar_p, kSoftmaxWarps); ptx::mbar_init(bar_o, 1);
     *abort_flag = 0;
     ptx::mbar_init_fence();
   }
@@ -137,49 +141,61 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
       ptx::bulk_wait_group_read<0>();                      // the stored P has left shared memory
     }
   } else if (warp >= 2) {
-    // ------------------------------------------------------------------ softmax and output, one query row per thread
-    const int q = warp & 3, r = q * 32 + lane;              // TMEM lane quarter of this warp; row within the tile
+    // ------------------------------------------------------------------ softmax and output
+    // Two warps share each TMEM lane quarter (= 32 query rows, one per lane): warp (q, part) works on the
+    // 32-column chunks c = 2 i + part of its rows, and the two exchange their partial row maximum and row
+    // sum through shared memory.
+    const int q = warp & 3, part = (warp - 2) >> 2, r = q * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(q * 32) << 16);
-    bool ok = wait_bounded(bar_s, 0, abort_flag, a.status, a.wait_limit);
-    ok = __all_sync(0xffffffffu, ok);
+    const bool have_scores = wait_bounded(bar_s, 0, abort_flag, a.status, a.wait_limit);
+    // every softmax thread reaches this barrier whatever its wait returned, and the reduction hands all of them
+    // the same answer, so either all or none go on to the barriers below
+    bool ok = !ptx::named_barrier_any(1, 32 * kSoftmaxWarps, !have_scores);
     if (ok) {
       ptx::tc_fence_after_sync();
-      const int nchunk = 2 * nkb;                           // 32-column chunks, whole key blocks
       float v[32];
-      float m = -3.0e38f;
       // columns at and beyond s_k hold products with zero-filled key rows: they are kept out of the maximum and
       // the sum by replacing them with a very negative score, whose weight is exactly zero
-      auto load_chunk = [&](int c) {
+      auto load_scores = [&](int c) {
         ptx::tmem_ld_32x32(t_row + 32u * c, v);
         if (32 * c + 32 > a.s_k) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) if (32 * c + i >= a.s_k) v[i] = -3.0e38f;
         }
       };
-      for (int c = 0; c < nchunk; ++c) {
-        load_chunk(c);
+      float m4[4] = {-3.0e38f, -3.0e38f, -3.0e38f, -3.0e38f};
+      for (int c = part; c < 2 * nkb; c += 2) {
+        load_scores(c);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) m = fmaxf(m, v[i]);
+        for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], v[i]);
       }
-      const float mk = m * a.exp_scale;
-      float sum = 0.f;
-      for (int c = 0; c < nchunk; ++c) {
-        load_chunk(c);
+      row_max[part * 128 + r] = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+      ptx::named_barrier_sync(1, 32 * kSoftmaxWarps);
+      const float mk = fmaxf(row_max[r], row_max[128 + r]) * a.exp_scale;
+      float s4[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int c = part; c < 2 * nkb; c += 2) {
+        load_scores(c);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) sum += ex2(fmaf(v[i], a.exp_scale, -mk));
+        for (int i = 0; i < 32; ++i) {
+          v[i] = ex2(fmaf(v[i], a.exp_scale, -mk));
+          s4[i & 3] += v[i];
+        }
+        ptx::tmem_st_32x32(t_row + 32u * c, v);              // the exponentials replace the scores
       }
-      const float inv = a.softmax_scale / sum;
+      ptx::tmem_st_wait();
+      row_sum[part * 128 + r] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+      ptx::named_barrier_sync(1, 32 * kSoftmaxWarps);
+      const float inv = a.softmax_scale / (row_sum[r] + row_sum[128 + r]);
       const uint32_t row_off = (uint32_t)r * 128u, sw = (uint32_t)(r & 7);
-      for (int c = 0; c < nchunk; ++c) {
-        load_chunk(c);
+      for (int c = part; c < 2 * nkb; c += 2) {
+        ptx::tmem_ld_32x32(t_row + 32u * c, v);
         const uint32_t blk = p_s + (uint32_t)(c >> 1) * kKeyBlockBytes + row_off;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           uint32_t w[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const float p0 = ex2(fmaf(v[8 * g + 2 * j], a.exp_scale, -mk)) * inv;       // masked columns: ex2(-huge) = 0
-            const float p1 = ex2(fmaf(v[8 * g + 2 * j + 1], a.exp_scale, -mk)) * inv;
+            const float p0 = v[8 * g + 2 * j] * inv, p1 = v[8 * g + 2 * j + 1] * inv;
             w[j] = a.op_bf16 ? pack_bf16x2(p0, p1) : pack_f16x2(p0, p1);
           }
           const uint32_t chunk16 = (uint32_t)((c & 1) * 4 + g);
@@ -190,21 +206,19 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(bar_p);
-      // ---------------------------------------------------------------- context
+      // ---------------------------------------------------------------- context: this warp's 32 of the 64 columns
       ok = wait_bounded(bar_o, 0, abort_flag, a.status, a.wait_limit);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         ptx::tc_fence_after_sync();
         const int row = q0 + r;
-        char* dst = static_cast<char*>(a.c) + ((int64_t)b0 * a.c_stride0 + (int64_t)b1 * a.c_stride1 + (int64_t)row * a.c_ld) *
-                                                  dtype_size(a.c_dt);
+        const int es = dtype_size(a.c_dt);
+        char* dst = static_cast<char*>(a.c) +
+                    ((int64_t)b0 * a.c_stride0 + (int64_t)b1 * a.c_stride1 + (int64_t)row * a.c_ld + 32 * part) * es;
+        ptx::tmem_ld_32x32(t_row + 32u * part, v);
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          ptx::tmem_ld_32x32(t_row + 32u * h, v);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] *= a.alpha_context;
-          if (row < a.s_q) store_vec<32>(dst + 32 * h * dtype_size(a.c_dt), a.c_dt, v);
-        }
+        for (int i = 0; i < 32; ++i) v[i] *= a.alpha_context;
+        if (row < a.s_q) store_vec<32>(dst, a.c_dt, v);
       }
     }
   }

@@ -37,9 +37,15 @@ E4, E5 = torch.float8_e4m3fn, torch.float8_e5m2
 
 class UnitScaledEncoderLayer:
     def __init__(self, nseq: int, slen: int, d: int, nhead: int, d_ff: int, tau: float = 0.5,
-                 attention: str = "bf16", norm: str | None = None, eps: float = 1e-5, device="cuda"):
+                 attention: str = "bf16", norm: str | None = None, eps: float = 1e-5, device="cuda",
+                 fused_attention: bool = False):
         assert d % nhead == 0 and norm in (None, "post")
         self.attention, self.norm, self.eps = attention, norm, eps
+        # fused_attention: scores, scaled softmax and context of the forward pass as one us_attention_fwd launch
+        # (16-bit attention operands, heads of 64, at most 512 tokens per sequence); the scores are then never stored
+        self.fused_attention = fused_attention
+        if fused_attention and not (attention in ("bf16", "fp16") and d // nhead == 64 and slen <= 512):
+            raise ValueError("fused attention needs 16-bit attention operands, heads of 64 and sequences of at most 512 tokens")
         if attention == "fp8":
             act_dt, grad_dt, wide_dt = E4, E5, torch.bfloat16
         else:
@@ -49,7 +55,7 @@ class UnitScaledEncoderLayer:
         e = lambda r, c, dt: torch.empty((r, c), dtype=dt, device=device)
         self.Xq, self.Wqkv_q, self.Wo_q = e(T, d, E4), e(d, 3 * d, E4), e(d, d, E4)
         self.QKV = e(T, 3 * d, act_dt)
-        self.S = e(nseq * nhead * slen, slen, wide_dt)
+        self.S = None if fused_attention else e(nseq * nhead * slen, slen, wide_dt)
         self.P = e(nseq * nhead * slen, slen, act_dt)
         self.Cq = e(T, d, E4)
         self.R1 = e(T, d, torch.bfloat16)
@@ -82,7 +88,8 @@ class UnitScaledEncoderLayer:
         self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
                        dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
         # fused cast, attention forward, FFN forward + backward, attention backward (one cast fewer with FP8 attention)
-        self.launches_per_step = 1 + 5 + 7 + (10 if attention == "fp8" else 11) + (7 if norm == "post" else 0)
+        self.launches_per_step = 1 + (3 if fused_attention else 5) + 7 + (10 if attention == "fp8" else 11) + (7 if norm == "post" else 0)
+        self.bt_fused = L.attention_batch(n, qkv, qkv, qkv, td, sq)
 
     def _heads(self, M, which):
         """Problem (0, 0) of a [T x 3d] matrix: rows of the first sequence, columns of head 0 of Q / K / V."""
@@ -102,9 +109,13 @@ class UnitScaledEncoderLayer:
                             [self.Wqkv_q, self.Wo_q, self.Xq, f.W1q, f.W2q] + ([] if post else [f.Gq]), stream)
         L.us_linear_fwd(self.Xq, self.Wqkv_q, sc["alpha_qkv"], self.QKV, ws, None, stream)
         Q, K, V = (self._heads(self.QKV, i) for i in range(3))
-        L.us_linear_bwd_x_batched(Q, K, sc["alpha_s"], self.S[:s], self.bt["scores"], ws, stream)
-        L.us_softmax_fwd(self.S, sc["sm"], self.P, stream)
-        L.us_linear_fwd_batched(self.P[:s], V, sc["alpha_c"], self.Cq[:s, : self.hd], self.bt["ctx"], ws, stream)
+        if self.fused_attention:
+            L.us_attention_fwd(Q, K, V, sc["alpha_s"], sc["sm"], sc["alpha_c"], self.Cq[:s, : self.hd], self.P[:s],
+                               self.bt_fused, ws, stream)
+        else:
+            L.us_linear_bwd_x_batched(Q, K, sc["alpha_s"], self.S[:s], self.bt["scores"], ws, stream)
+            L.us_softmax_fwd(self.S, sc["sm"], self.P, stream)
+            L.us_linear_fwd_batched(self.P[:s], V, sc["alpha_c"], self.Cq[:s, : self.hd], self.bt["ctx"], ws, stream)
         ep = L.epilogue(skip=X, skip_coef=self.c_skip, out_coef=self.c_branch)
         L.us_linear_fwd(self.Cq, self.Wo_q, sc["alpha_o"], self.U1 if post else self.R1, ws, ep, stream)
         if post:

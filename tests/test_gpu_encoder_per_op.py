@@ -21,12 +21,12 @@ pytestmark = pytest.mark.gpu
 TOL = 2e-3
 
 
-def _run(nseq, slen, d, nhead, f, seed, attention):
+def _run(nseq, slen, d, nhead, f, seed, attention, fused=False):
     from paper_2303_11257_b200 import encoder, synth
     T = nseq * slen
     host = (synth.normal(seed, 0, (T, d)), synth.normal(seed, 1, (d, 3 * d)), synth.normal(seed, 2, (d, d)),
             synth.normal(seed, 3, (d, f)), synth.normal(seed, 4, (f, d)), synth.normal(seed, 5, (T, d)))
-    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, f, attention=attention)
+    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, f, attention=attention, fused_attention=fused)
     layer.step(*[torch.from_numpy(t).cuda() for t in host])
     layer.check()
     return layer, host
@@ -65,7 +65,8 @@ def _per_op(layer, host, problems, rows, wrows):
     assert np.array_equal(U.codes_of(layer.Wo_q), F.quantise_codes(Wo, F.E4M3))
     Xq, Wqkv_q, Wo_q = H(layer.Xq), H(layer.Wqkv_q), H(layer.Wo_q)
     QKV, Cq = H(layer.QKV), H(layer.Cq)
-    f_act, f_wide, f_grad = _fmt_of(layer.QKV), _fmt_of(layer.S), _fmt_of(layer.dS)
+    f_act, f_wide, f_grad = _fmt_of(layer.QKV), _fmt_of(layer.dP), _fmt_of(layer.dS)
+    fused = layer.S is None          # fused attention forward: the scores are never stored
     # ---- QKV projection
     _check(QKV[rows], O.linear_fwd(Xq[rows], Wqkv_q, sc["alpha_qkv"]), f_act, TOL, "QKV")
     dC, dQKV = H(layer.dC), H(layer.dQKV)
@@ -75,10 +76,15 @@ def _per_op(layer, host, problems, rows, wrows):
         q, k, v = (QKV[r, o + j * hd:o + (j + 1) * hd] for o in (0, d, 2 * d))
         c = slice(j * hd, (j + 1) * hd)
         tag = f"problem ({i}, {j})"
-        Sp, Pp, dPp, dSp = H(layer.S[pr]), H(layer.P[pr]), H(layer.dP[pr]), H(layer.dS[pr])   # score-sized tensors: this problem only
+        Pp, dPp, dSp = H(layer.P[pr]), H(layer.dP[pr]), H(layer.dS[pr])   # score-sized tensors: this problem only
         # forward: scores, scaled softmax, context
-        _check(Sp, O.linear_bwd_x(q, k, sc["alpha_s"]), f_wide, TOL, "S " + tag)
-        _check(Pp, O.softmax_fwd(Sp, sc["sm"]), f_act, 3e-6 * sc["sm"], "P " + tag)
+        if fused:
+            p_ref, _ = O.attention_fwd(q, k, v, sc["alpha_s"], sc["sm"], sc["alpha_c"], "f64")     # from unrounded scores
+            _check(Pp, p_ref, f_act, 3e-6 * sc["sm"], "P (fused) " + tag)
+        else:
+            Sp = H(layer.S[pr])
+            _check(Sp, O.linear_bwd_x(q, k, sc["alpha_s"]), f_wide, TOL, "S " + tag)
+            _check(Pp, O.softmax_fwd(Sp, sc["sm"]), f_act, 3e-6 * sc["sm"], "P " + tag)
         ref_c = O.linear_fwd(Pp, v, sc["alpha_c"])
         _check(Cq[r, c], ref_c, "e4m3", TOL * max(1.0, np.abs(ref_c).max()), "C " + tag)
         # backward: dP = beta dC V^T, dV = beta P^T dC, dS, dQ = beta dS K, dK = beta dS^T Q
@@ -142,11 +148,20 @@ def test_encoder_layer_every_op_small(cfg, attention):
     _per_op(layer, host, problems, np.arange(nseq * slen), np.arange(max(d, f)))
 
 
-@pytest.mark.parametrize("attention", ["bf16", "fp8"])
-def test_encoder_layer_every_op_bert_large_shape(attention):
+@pytest.mark.parametrize("attention", ["bf16", "fp16"])
+@pytest.mark.parametrize("cfg", [(2, 128, 256, 4, 512), (3, 80, 192, 3, 400)])
+def test_encoder_layer_every_op_small_fused_attention(cfg, attention):
+    nseq, slen, d, nhead, f = cfg
+    layer, host = _run(nseq, slen, d, nhead, f, seed=53, attention=attention, fused=True)
+    problems = [(i, j) for i in range(nseq) for j in range(nhead)]
+    _per_op(layer, host, problems, np.arange(nseq * slen), np.arange(max(d, f)))
+
+
+@pytest.mark.parametrize("attention,fused", [("bf16", False), ("fp8", False), ("bf16", True)])
+def test_encoder_layer_every_op_bert_large_shape(attention, fused):
     """Config 5 at its stated size (16 sequences x 512 tokens, d = 1024, 16 heads x 64, d_ff = 4096)."""
     nseq, slen, d, nhead, f = 16, 512, 1024, 16, 4096
-    layer, host = _run(nseq, slen, d, nhead, f, seed=52, attention=attention)
+    layer, host = _run(nseq, slen, d, nhead, f, seed=52, attention=attention, fused=fused)
     rng = np.random.default_rng(7)
     problems = [(0, 0), (0, nhead - 1), (nseq - 1, 0), (nseq - 1, nhead - 1)] + \
                [(int(rng.integers(nseq)), int(rng.integers(nhead))) for _ in range(4)]
