@@ -153,55 +153,72 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
     bool ok = !ptx::named_barrier_any(1, 32 * kSoftmaxWarps, !have_scores);
     if (ok) {
       ptx::tc_fence_after_sync();
-      float v[32];
+      // One sweep over this warp's chunks c = part, part + 2, ...: the load of the next chunk is in flight
+      // while body(c, registers) works on the current one.
+      const int c_end = 2 * nkb;
+      auto sweep = [&](auto&& body) {
+        uint32_t ra[32], rb[32];
+        int c = part;
+        if (c < c_end) ptx::tmem_ld_32x32_issue(t_row + 32u * c, ra);
+        while (c < c_end) {
+          ptx::tmem_ld_fence(ra);
+          if (c + 2 < c_end) ptx::tmem_ld_32x32_issue(t_row + 32u * (c + 2), rb);
+          body(c, ra);
+          c += 2;
+          if (c >= c_end) break;
+          ptx::tmem_ld_fence(rb);
+          if (c + 2 < c_end) ptx::tmem_ld_32x32_issue(t_row + 32u * (c + 2), ra);
+          body(c, rb);
+          c += 2;
+        }
+      };
       // columns at and beyond s_k hold products with zero-filled key rows: they are kept out of the maximum and
       // the sum by replacing them with a very negative score, whose weight is exactly zero
-      auto load_scores = [&](int c) {
-        ptx::tmem_ld_32x32(t_row + 32u * c, v);
+      auto mask = [&](int c, uint32_t (&x)[32]) {
         if (32 * c + 32 > a.s_k) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) if (32 * c + i >= a.s_k) v[i] = -3.0e38f;
+          for (int i = 0; i < 32; ++i) if (32 * c + i >= a.s_k) x[i] = __float_as_uint(-3.0e38f);
         }
       };
       float m4[4] = {-3.0e38f, -3.0e38f, -3.0e38f, -3.0e38f};
-      for (int c = part; c < 2 * nkb; c += 2) {
-        load_scores(c);
+      sweep([&](int c, uint32_t (&x)[32]) {
+        mask(c, x);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], v[i]);
-      }
+        for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(x[i]));
+      });
       row_max[part * 128 + r] = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       ptx::named_barrier_sync(1, 32 * kSoftmaxWarps);
       const float mk = fmaxf(row_max[r], row_max[128 + r]) * a.exp_scale;
       float s4[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int c = part; c < 2 * nkb; c += 2) {
-        load_scores(c);
+      sweep([&](int c, uint32_t (&x)[32]) {
+        mask(c, x);
+        float e[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          v[i] = ex2(fmaf(v[i], a.exp_scale, -mk));
-          s4[i & 3] += v[i];
+          e[i] = ex2(fmaf(__uint_as_float(x[i]), a.exp_scale, -mk));
+          s4[i & 3] += e[i];
         }
-        ptx::tmem_st_32x32(t_row + 32u * c, v);              // the exponentials replace the scores
-      }
+        ptx::tmem_st_32x32(t_row + 32u * c, e);              // the exponentials replace the scores
+      });
       ptx::tmem_st_wait();
       row_sum[part * 128 + r] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
       ptx::named_barrier_sync(1, 32 * kSoftmaxWarps);
       const float inv = a.softmax_scale / (row_sum[r] + row_sum[128 + r]);
       const uint32_t row_off = (uint32_t)r * 128u, sw = (uint32_t)(r & 7);
-      for (int c = part; c < 2 * nkb; c += 2) {
-        ptx::tmem_ld_32x32(t_row + 32u * c, v);
+      sweep([&](int c, uint32_t (&x)[32]) {
         const uint32_t blk = p_s + (uint32_t)(c >> 1) * kKeyBlockBytes + row_off;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           uint32_t w[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const float p0 = v[8 * g + 2 * j] * inv, p1 = v[8 * g + 2 * j + 1] * inv;
+            const float p0 = __uint_as_float(x[8 * g + 2 * j]) * inv, p1 = __uint_as_float(x[8 * g + 2 * j + 1]) * inv;
             w[j] = a.op_bf16 ? pack_bf16x2(p0, p1) : pack_f16x2(p0, p1);
           }
           const uint32_t chunk16 = (uint32_t)((c & 1) * 4 + g);
           ptx::sts128(blk + ((chunk16 ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
         }
-      }
+      });
       ptx::fence_proxy_async_smem();                         // the MMA and the TMA store read these bytes
       ptx::tc_fence_before_sync();
       __syncwarp();
@@ -215,6 +232,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
         const int es = dtype_size(a.c_dt);
         char* dst = static_cast<char*>(a.c) +
                     ((int64_t)b0 * a.c_stride0 + (int64_t)b1 * a.c_stride1 + (int64_t)row * a.c_ld + 32 * part) * es;
+        float v[32];
         ptx::tmem_ld_32x32(t_row + 32u * part, v);
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] *= a.alpha_context;
