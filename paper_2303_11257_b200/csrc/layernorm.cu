@@ -14,6 +14,7 @@
 #include "common.cuh"
 #include "host.h"
 #include "rowwise.cuh"
+#include "sm100.cuh"
 
 namespace us {
 
@@ -281,95 +282,212 @@ __global__ void __launch_bounds__(kLnThreads, 2) ln_fwd16_kernel(const LnArgs a)
   }
 }
 
-// G32: the gradient is float32 (the gradient of a layer's output often is): it is loaded at the top of the
-// iteration into float registers instead of being prefetched packed; X is still prefetched.
-template <int NCH, bool G32>
+// G32: the gradient is float32 (the gradient of a layer's output often is) instead of the 16-bit type of X.
+//
+// The rows reach the SM through a ring of kLnStages slots per warp in shared memory, filled by bulk
+// copies (cp.async.bulk, completion counted on one mbarrier per slot): with one row per warp in
+// registers the kernel is bound by memory latency (a few tens of KB in flight per SM), the ring keeps
+// kLnStages rows per warp in flight.  A wait on a slot is bounded; if it ever runs out the warp reads
+// that row and all later ones with ordinary loads (same result), and before leaving it gives the
+// copies it issued time to land.
+constexpr int kLnStages = 3;
+constexpr uint32_t kLnWaitLimit = 1u << 20;
+
+// XBF: X (and a 16-bit gradient) are BF16 rather than F16; fixed at compile time, because a run-time choice
+// in the unpacking costs more instructions than the arithmetic it feeds.
+template <int NCH, bool G32, bool XBF>
 __global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
-  extern __shared__ __align__(16) float ln_smem[];                         // w[cols] as float32, then [warps][cols] for the combine
-  float* w_s = ln_smem;
-  float* comb = ln_smem + a.cols;
-  for (int j = threadIdx.x; j < a.cols; j += blockDim.x) w_s[j] = load_one(a.w, a.w_dt, j);
-  __syncthreads();
+  extern __shared__ __align__(16) float ln_smem[];             // w[cols] as float32, [warps][cols] for the combine, the ring, its mbarriers
+  float* w_s = ln_smem;                                        // NCH * 256 floats
+  float* comb = ln_smem + NCH * 256;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const uint32_t xb = (uint32_t)a.cols * 2u, gb = (uint32_t)a.cols * (G32 ? 4u : 2u), slot = xb + gb;
+  char* ring_gen = reinterpret_cast<char*>(comb + (size_t)nw * a.cols) + (size_t)warp * kLnStages * slot;
+  const uint32_t ring = ptx::smem_addr(ring_gen);
+  const uint32_t bars = ptx::smem_addr(reinterpret_cast<char*>(comb + (size_t)nw * a.cols) + (size_t)nw * kLnStages * slot) +
+                        8u * (uint32_t)(warp * kLnStages);
+  if (!G32 && lane == 0) {                                     // (no ring, hence no mbarriers, with a float32 gradient)
+    for (int st = 0; st < kLnStages; ++st) ptx::mbar_init(bars + 8u * st, 1);
+    ptx::mbar_init_fence();
+  }
+  // w in shared memory, laid out for conflict-free 16-byte reads: a lane's eight consecutive weights
+  // (columns 8 q .. 8 q + 7) are split into a low and a high half; low halves at [4 q, 4 q + 4), high halves
+  // kLnHi floats further.
+  const int kLnHi = NCH * 32 * 4;
+  for (int j = threadIdx.x; j < a.cols; j += blockDim.x)
+    w_s[(j >> 3) * 4 + (j & 3) + ((j & 4) ? kLnHi : 0)] = load_one(a.w, a.w_dt, j);
+  __syncthreads();
   const int64_t stride = (int64_t)gridDim.x * nw;
   const float inv_n = 1.0f / (float)a.cols;
-  float sw[NCH][8], sc[NCH][8];
+  f32x2 sw[NCH][4], sc[NCH][4];                                // column sums of g * xhat and of g, as float32 pairs
 #pragma unroll
   for (int c = 0; c < NCH; ++c)
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { sw[c][i] = 0.f; sc[c][i] = 0.f; }
+    for (int j = 0; j < 4; ++j) { sw[c][j] = pack2(0.f, 0.f); sc[c][j] = pack2(0.f, 0.f); }
   int64_t row = (int64_t)blockIdx.x * nw + warp;
-  uint4 cx[NCH], cg[G32 ? 1 : NCH], nx[NCH], ng[G32 ? 1 : NCH];
-  if (row < a.rows) {
-    load_row16<NCH>(a.x, row * a.x_ld, lane, a.cols, cx);
-    if (!G32) load_row16<G32 ? 1 : NCH>(a.g, row * a.g_ld, lane, a.cols, cg);
-  }
-  for (; row < a.rows; row += stride) {
-    if (row + stride < a.rows) {
-      load_row16<NCH>(a.x, (row + stride) * a.x_ld, lane, a.cols, nx);
-      if (!G32) load_row16<G32 ? 1 : NCH>(a.g, (row + stride) * a.g_ld, lane, a.cols, ng);
-    }
+  auto issue = [&](int64_t r, int st) {                        // lane 0
+    const uint32_t bar = bars + 8u * st;
+    ptx::mbar_expect_tx(bar, slot);
+    ptx::bulk_load_1d(ring + st * slot, static_cast<const char*>(a.x) + r * a.x_ld * 2, xb, bar);
+    ptx::bulk_load_1d(ring + st * slot + xb, static_cast<const char*>(a.g) + r * a.g_ld * (G32 ? 4 : 2), gb, bar);
+  };
+  int issued = 0;                                              // rows asked for so far (warp-uniform)
+  if (!G32)
+    for (; issued < kLnStages && row + issued * stride < a.rows; ++issued)
+      if (lane == 0) issue(row + issued * stride, issued);
+  // direct: ordinary loads instead of the ring -- after a wait ran out, and always for a float32 gradient
+  // (rows of 6 bytes per element: the ring then costs a CTA per SM and measured slower than plain loads)
+  bool direct = G32;
+  int it = 0, unconsumed = 0;                                  // unconsumed: first row whose copy was never waited for
+  uint4 cx[NCH], cg[G32 ? 1 : NCH], nx[G32 ? NCH : 1];
+  for (; row < a.rows; row += stride, ++it) {
+    const int st = it % kLnStages;
+    const uint32_t parity = (uint32_t)(it / kLnStages) & 1u;
     float gf[G32 ? NCH : 1][8];
-    if (G32) {
+    if (!direct) {
+      bool ok = false;
+      for (uint32_t k = 0; k < kLnWaitLimit && !(ok = ptx::mbar_try_wait(bars + 8u * st, parity)); ++k) {}
+      direct = !__all_sync(0xffffffffu, ok);
+      if (direct) unconsumed = it;
+    }
+    if (!direct) {
+      const char* sx = ring_gen + (size_t)st * slot;
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
         const int col = (c * 32 + lane) * 8;
-        if (col < a.cols) load_vec<8>(static_cast<const char*>(a.g) + (row * a.g_ld + col) * 4, US_F32, gf[G32 ? c : 0]);
+        if (col < a.cols) {
+          cx[c] = *reinterpret_cast<const uint4*>(sx + col * 2);
+          if (G32) {
+            const float4 g0 = *reinterpret_cast<const float4*>(sx + xb + col * 4), g1 = *reinterpret_cast<const float4*>(sx + xb + col * 4 + 16);
+            gf[G32 ? c : 0][0] = g0.x; gf[G32 ? c : 0][1] = g0.y; gf[G32 ? c : 0][2] = g0.z; gf[G32 ? c : 0][3] = g0.w;
+            gf[G32 ? c : 0][4] = g1.x; gf[G32 ? c : 0][5] = g1.y; gf[G32 ? c : 0][6] = g1.z; gf[G32 ? c : 0][7] = g1.w;
+          } else {
+            cg[G32 ? 0 : c] = *reinterpret_cast<const uint4*>(sx + xb + col * 2);
+          }
+        } else {
+          cx[c] = make_uint4(0, 0, 0, 0);
+          if (!G32) cg[G32 ? 0 : c] = make_uint4(0, 0, 0, 0);
+        }
+      }
+      __syncwarp();                                            // every lane holds its part: the slot can be refilled
+      const int64_t nxt = row + (int64_t)kLnStages * stride;
+      if (nxt < a.rows) {
+        if (lane == 0) issue(nxt, st);
+        ++issued;
+      }
+    } else {
+      if constexpr (G32) {
+        // X of this row was fetched one iteration ahead (packed, in registers); the float32 gradient is read now
+        if (it == 0) load_row16<NCH>(a.x, row * a.x_ld, lane, a.cols, cx);
+        else {
+#pragma unroll
+          for (int c = 0; c < NCH; ++c) cx[c] = nx[c];
+        }
+        if (row + stride < a.rows) load_row16<NCH>(a.x, (row + stride) * a.x_ld, lane, a.cols, nx);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const int col = (c * 32 + lane) * 8;
+          if (col < a.cols) load_vec<8>(static_cast<const char*>(a.g) + (row * a.g_ld + col) * 4, US_F32, gf[c]);
+        }
+      } else {
+        load_row16<NCH>(a.x, row * a.x_ld, lane, a.cols, cx);
+        load_row16<NCH>(a.g, row * a.g_ld, lane, a.cols, cg);
       }
     }
-    float x[NCH][8];
+    // From here on the row is worked on as pairs of float32 in 64-bit registers (add / mul / fma .f32x2):
+    // the kernel is bound by instruction issue, and the packed forms halve the arithmetic instructions.
+    f32x2 xp[NCH][4];
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) unpack16x8(cx[c], a.x_dt, x[c]);
-    float mu, rstd;
-    stats_regs<NCH>(x, lane, a.cols, a.eps, mu, rstd);
-    float su = 0.f, sux = 0.f;
+    for (int c = 0; c < NCH; ++c) {
+      const uint32_t wx[4] = {cx[c].x, cx[c].y, cx[c].z, cx[c].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float2 f = XBF ? unpack_bf16x2(wx[j]) : unpack_f16x2(wx[j]);
+        xp[c][j] = pack2(f.x, f.y);
+      }
+    }
+    auto g_pair = [&](int c, int j) -> f32x2 {                 // gradient values 2 j, 2 j + 1 of chunk c
+      if (G32) return pack2(gf[G32 ? c : 0][2 * j], gf[G32 ? c : 0][2 * j + 1]);
+      const uint4& r = cg[G32 ? 0 : c];
+      const uint32_t w = j == 0 ? r.x : j == 1 ? r.y : j == 2 ? r.z : r.w;
+      const float2 f = XBF ? unpack_bf16x2(w) : unpack_f16x2(w);
+      return pack2(f.x, f.y);
+    };
+    auto w_pairs = [&](int col, f32x2 (&w2)[4]) {
+      const ulonglong2 lo = *reinterpret_cast<const ulonglong2*>(w_s + (col >> 1)), hi = *reinterpret_cast<const ulonglong2*>(w_s + (col >> 1) + kLnHi);
+      w2[0] = lo.x; w2[1] = lo.y; w2[2] = hi.x; w2[3] = hi.y;
+    };
+    // mean, then variance about the mean (chunks beyond the row's end hold zeros and are left out of the second sum)
+    f32x2 acc = pack2(0.f, 0.f);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc = add2(acc, xp[c][j]);
+    float lo, hi;
+    unpack2(acc, lo, hi);
+    const float mu = warp_sum(lo + hi) * inv_n;
+    const f32x2 neg_mu = splat2(-mu);
+    acc = pack2(0.f, 0.f);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      if ((c * 32 + lane) * 8 < a.cols) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { const f32x2 dm = add2(xp[c][j], neg_mu); acc = fma2(dm, dm, acc); }
+      }
+    }
+    unpack2(acc, lo, hi);
+    const float rstd = rsqrtf(warp_sum(lo + hi) * inv_n + a.eps);
+    const f32x2 rstd2 = splat2(rstd), shift2 = splat2(-mu * rstd);
+    f32x2 su2 = pack2(0.f, 0.f), sux2 = pack2(0.f, 0.f);
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
       const int col = (c * 32 + lane) * 8;
       if (col < a.cols) {
-        float g[8];
-        if (G32) {
+        f32x2 w2[4];
+        w_pairs(col, w2);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) g[i] = gf[G32 ? c : 0][i];
-        } else {
-          unpack16x8(cg[G32 ? 0 : c], a.g_dt, g);
-        }
-        const float4 w0 = *reinterpret_cast<const float4*>(w_s + col), w1 = *reinterpret_cast<const float4*>(w_s + col + 4);
-        const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const float xh = (x[c][i] - mu) * rstd, uu = g[i] * w[i];
-          x[c][i] = xh;
-          su += uu;
-          sux = fmaf(uu, xh, sux);
-          sw[c][i] = fmaf(g[i], xh, sw[c][i]);
-          sc[c][i] += g[i];
+        for (int j = 0; j < 4; ++j) {
+          const f32x2 g2 = g_pair(c, j);
+          const f32x2 xh = fma2(xp[c][j], rstd2, shift2);      // normalised input, kept for the second loop
+          xp[c][j] = xh;
+          const f32x2 uu = mul2(g2, w2[j]);
+          su2 = add2(su2, uu);
+          sux2 = fma2(uu, xh, sux2);
+          sw[c][j] = fma2(g2, xh, sw[c][j]);
+          sc[c][j] = add2(sc[c][j], g2);
         }
       }
     }
-    const float mean_u = warp_sum(su) * inv_n, mean_ux = warp_sum(sux) * inv_n;
+    unpack2(su2, lo, hi);
+    const float mean_u = warp_sum(lo + hi) * inv_n;
+    unpack2(sux2, lo, hi);
+    const float mean_ux = warp_sum(lo + hi) * inv_n;
     const float k = a.beta_x * rstd;
+    const f32x2 k2 = splat2(k), c0 = splat2(-k * mean_u), c1 = splat2(-k * mean_ux);
     const int64_t out_off = row * a.out_ld;
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
       const int col = (c * 32 + lane) * 8;
       if (col < a.cols) {
-        float g[8], d[8];
-        if (G32) {
+        f32x2 w2[4];
+        w_pairs(col, w2);
+        float d[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) g[i] = gf[G32 ? c : 0][i];
-        } else {
-          unpack16x8(cg[G32 ? 0 : c], a.g_dt, g);
+        for (int j = 0; j < 4; ++j) {
+          // k (g w - mean_u - xh mean_ux)
+          const f32x2 t = fma2(mul2(g_pair(c, j), w2[j]), k2, c0);
+          unpack2(fma2(xp[c][j], c1, t), d[2 * j], d[2 * j + 1]);
         }
-        const float4 w0 = *reinterpret_cast<const float4*>(w_s + col), w1 = *reinterpret_cast<const float4*>(w_s + col + 4);
-        const float w[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) d[i] = k * (g[i] * w[i] - mean_u - x[c][i] * mean_ux);
         store8(a.out, a.out_dt, out_off, col, a.cols, true, d);
       }
     }
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) { cx[c] = nx[c]; if (!G32) cg[G32 ? 0 : c] = ng[G32 ? 0 : c]; }
+  }
+  if (direct && lane == 0) {
+    // copies issued but never consumed: one per slot at most
+    for (int k = unconsumed; k < issued; ++k) {
+      const uint32_t bar = bars + 8u * (k % kLnStages), parity = (uint32_t)(k / kLnStages) & 1u;
+      for (uint32_t n = 0; n < kLnWaitLimit && !ptx::mbar_try_wait(bar, parity); ++n) {}
+    }
   }
   float* dst = a.partial + (size_t)blockIdx.x * 2 * a.cols;
 #pragma unroll
@@ -380,7 +498,8 @@ __global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
       const int col = (c * 32 + lane) * 8;
       if (col < a.cols) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) comb[(size_t)warp * a.cols + col + i] = pass == 0 ? sw[c][i] : sc[c][i];
+        for (int j = 0; j < 4; ++j)
+          *reinterpret_cast<f32x2*>(comb + (size_t)warp * a.cols + col + 2 * j) = pass == 0 ? sw[c][j] : sc[c][j];
       }
     }
     __syncthreads();
@@ -393,22 +512,32 @@ __global__ void __launch_bounds__(128, 3) ln_bwd16_kernel(const LnArgs a) {
 }
 
 // dw_j = beta * sum over CTAs of partial[cta][0][j], dc_j likewise from partial[cta][1][j].
-// One CTA per 32 columns of the 2 * cols sums: 8 groups of 32 threads each add every 8th partial row
-// in order, then the groups are added in order.
-__global__ void __launch_bounds__(256) ln_bwd_reduce_kernel(const float* partial, int nparts, int cols, float beta,
-                                                            void* dw, int dw_dt, void* dc, int dc_dt) {
-  __shared__ float acc[8][32];
+// One CTA per 32 columns of the 2 * cols sums: 32 groups of 32 threads each add every 32nd partial row
+// in order (four independent partial sums per thread, combined in a fixed order), then the groups are
+// added in order.
+constexpr int kLnReduceGroups = 32;
+__global__ void __launch_bounds__(32 * kLnReduceGroups) ln_bwd_reduce_kernel(const float* partial, int nparts, int cols, float beta,
+                                                                             void* dw, int dw_dt, void* dc, int dc_dt) {
+  __shared__ float acc[kLnReduceGroups][32];
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int j = blockIdx.x * 32 + tx;               // index into [2][cols]
-  float s = 0.f;
-  if (j < 2 * cols)
-    for (int p = ty; p < nparts; p += 8) s += partial[(size_t)p * 2 * cols + j];
-  acc[ty][tx] = s;
+  float s4[4] = {0.f, 0.f, 0.f, 0.f};
+  if (j < 2 * cols) {
+    int p = ty;
+    for (; p + 3 * kLnReduceGroups < nparts; p += 4 * kLnReduceGroups) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) s4[u] += partial[(size_t)(p + u * kLnReduceGroups) * 2 * cols + j];
+    }
+#pragma unroll
+    for (int u = 0; u < 3; ++u)                     // at most three rows are left for this group
+      if (p + u * kLnReduceGroups < nparts) s4[u] += partial[(size_t)(p + u * kLnReduceGroups) * 2 * cols + j];
+  }
+  acc[ty][tx] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
   __syncthreads();
   if (ty == 0 && j < 2 * cols) {
     float t = 0.f;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) t += acc[q][tx];
+    for (int q = 0; q < kLnReduceGroups; ++q) t += acc[q][tx];
     t *= beta;
     if (j < cols) store_one(dw, dw_dt, j, t);
     else store_one(dc, dc_dt, j - cols, t);
@@ -529,16 +658,22 @@ extern "C" us_status us_layer_norm_bwd(const us_mat* X, const us_mat* w, const u
   if (a.vec_ok && nch <= 4 && (a.x_dt == US_BF16 || a.x_dt == US_F16) && (a.g_dt == a.x_dt || a.g_dt == US_F32)) {
     const bool g32 = a.g_dt == US_F32;
     nparts = ln_bwd_grid(X->rows > 0 ? X->rows : 1, kLnFastWarps, kLnFastPerSm);
-    const size_t smem = (size_t)(1 + kLnFastWarps) * a.cols * sizeof(float);
-#define US_LN_BWD16(N)                                                                             \
-  do {                                                                                            \
-    if (g32) ln_bwd16_kernel<N, true><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);                \
-    else ln_bwd16_kernel<N, false><<<nparts, 32 * kLnFastWarps, smem, st>>>(a);                   \
-  } while (0)
-    if (nch <= 1) US_LN_BWD16(1);
-    else if (nch <= 2) US_LN_BWD16(2);
-    else US_LN_BWD16(4);
-#undef US_LN_BWD16
+    const size_t smem = ((size_t)(nch <= 1 ? 1 : nch <= 2 ? 2 : 4) * 256 + (size_t)kLnFastWarps * a.cols) * sizeof(float) +
+                        (g32 ? (size_t)0 : (size_t)kLnFastWarps * kLnStages * (a.cols * 4 + 8));
+    const bool xbf = a.x_dt == US_BF16;
+    const int n = nch <= 1 ? 1 : nch <= 2 ? 2 : 4;
+    void (*fn)(const LnArgs) = nullptr;
+#define US_LN_PICK(N)                                                                                   \
+  fn = g32 ? (xbf ? ln_bwd16_kernel<N, true, true> : ln_bwd16_kernel<N, true, false>)                   \
+           : (xbf ? ln_bwd16_kernel<N, false, true> : ln_bwd16_kernel<N, false, false>)
+    if (n == 1) US_LN_PICK(1);
+    else if (n == 2) US_LN_PICK(2);
+    else US_LN_PICK(4);
+#undef US_LN_PICK
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return US_ERR_CUDA;
+    fn<<<nparts, 32 * kLnFastWarps, smem, st>>>(a);
   } else if (nch <= 4) {
     const size_t smem = (size_t)kLnWarps * a.cols * sizeof(float);
     if (nch <= 1) ln_bwd_kernel<1><<<grid, kLnThreads, smem, st>>>(a);
@@ -552,6 +687,6 @@ extern "C" us_status us_layer_norm_bwd(const us_mat* X, const us_mat* w, const u
   }
   if (cudaGetLastError() != cudaSuccess) return US_ERR_CUDA;
   const int rgrid = (2 * a.cols + 31) / 32;
-  ln_bwd_reduce_kernel<<<rgrid, 256, 0, st>>>(a.partial, nparts, a.cols, beta_wc, dw->ptr, dw->dtype, dc->ptr, dc->dtype);
+  ln_bwd_reduce_kernel<<<rgrid, 32 * kLnReduceGroups, 0, st>>>(a.partial, nparts, a.cols, beta_wc, dw->ptr, dw->dtype, dc->ptr, dc->dtype);
   return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }

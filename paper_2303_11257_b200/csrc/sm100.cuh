@@ -81,6 +81,14 @@ __device__ __forceinline__ void tma_store_4d(const void* tmap, uint32_t src, int
                : "memory");
 }
 
+// Untiled bulk copy global -> this CTA's shared memory; both addresses and the size are multiples of 16 bytes.
+// Completion is counted in bytes on the mbarrier.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
 // Same load issued by a CTA of a cooperating pair (cta_group::2): the bytes are counted on the
 // mbarrier of the pair's even CTA (`bar` must already address that CTA).  No multicast.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap, uint32_t bar, int32_t x, int32_t y) {
