@@ -1,7 +1,8 @@
 // Fused scaled dot-product attention, forward (appendix "Unit scaling and attention"; paragraph
 // "Softmax (followed by matmul)"): per (sequence, head) problem
 //     S = alpha_scores * Q K^T,   P = softmax_scale * softmax(S) per row,   C = alpha_context * P V
-// in ONE kernel.  A CTA owns 128 query rows of one problem and all of its (at most 512) keys:
+// in ONE persistent kernel (one CTA per SM walks the tiles).  A tile is 128 query rows of one problem and
+// all of its (at most 512) keys:
 //   * Q [128 x 64] and K [<=512 x 64] arrive by TMA (128-byte swizzle), V [<=512 x 64] behind them;
 //   * tcgen05.mma (kind::f16, M = 128, N = 256, twice) leaves the whole score block, 128 x 512
 //     float32, in tensor memory (all 512 columns): the scores never reach shared or global memory
@@ -9,12 +10,16 @@
 //   * eight warps (two per TMEM lane quarter, one query row per lane, alternate 32-column chunks each)
 //     make three passes over their rows in tensor memory: maximum; exponentials, written back over the
 //     scores (tcgen05.st), and their sum; weights, scaled, rounded to the operand format and written
-//     to shared memory in the K-major swizzled layout of an MMA A operand, over the bytes Q and K
-//     occupied (both are dead by then);
-//   * a second chain of MMAs (M = 128, N = 64, K = keys) multiplies the weights by V into tensor
-//     memory columns 0..63 (the scores are dead by then); the same shared-memory tiles leave by TMA
-//     store as the stored P the backward pass needs;
+//     to shared memory in the K-major swizzled layout of an MMA A operand, a quarter of the keys (128)
+//     at a time into two 32 KB buffers used in turn;
+//   * as each quarter lands, a second chain of MMAs (M = 128, N = 64, K = 128 keys) multiplies it by V
+//     into tensor memory columns 0..63 (whose scores are dead by then), and the same shared-memory
+//     tiles leave by TMA store as the stored P the backward pass needs; a buffer is reused once its
+//     MMAs and its store have read it;
 //   * the eight warps scale the context and store it in the output format.
+// The roles overlap across tiles: Q and K of the next tile are fetched as soon as the score MMAs have
+// read the current ones, V as soon as the last context MMA has, and the weight stores of a tile drain
+// while the next tile's softmax runs.
 // Every wait on an mbarrier is bounded; a wait that runs out raises the status word (as in the GEMM
 // kernels) and the CTA leaves after its own copies have landed and its tensor memory is freed.
 #include <cuda.h>
@@ -37,12 +42,15 @@ constexpr int kSoftmaxWarps = 8;
 constexpr int kAttnThreads = 64 + 32 * kSoftmaxWarps;   // warp 0: TMA + MMA issue; warp 1: TMEM owner; warps 2-9: softmax
 constexpr uint32_t kQBytes = 128 * 128;    // 128 rows x 64 x 2 bytes
 constexpr uint32_t kKeyBlockBytes = 128 * 128;   // P tile of one 64-key block: 128 rows x 128 bytes
-constexpr uint32_t kPBytes = 8 * kKeyBlockBytes; // 128 KB; Q and K (16 + 64 KB) live in its first 80 KB until the scores exist
+constexpr uint32_t kQuarterBytes = 2 * kKeyBlockBytes;   // weights of 128 keys; two such buffers take the quarters of a tile in turn
+constexpr uint32_t kKBytes = 512 * 128;
 constexpr uint32_t kVBytes = 512 * 128;
-constexpr uint32_t kAttnSmem = kPBytes + kVBytes + 1024 /* alignment */ + 128 /* barriers, slots */ + 2048 /* row maxima and sums */;
+constexpr uint32_t kAttnSmem = kQBytes + kKBytes + kVBytes + 2 * kQuarterBytes + 1024 /* alignment */ + 128 /* barriers, slots */ +
+                               2048 /* row maxima and sums */;
 
 struct AttnParams {
   int s_q, s_k;
+  int q_tiles, nb1, nb0;    // 128-row query tiles per problem; problems in the inner / outer batch dimension
   float exp_scale;          // alpha_scores * log2(e)
   float softmax_scale;
   float alpha_context;
@@ -60,28 +68,40 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// Tile n of a CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ... of q_tiles * nb1 * nb0, query tile fastest.
+__device__ __forceinline__ void attn_tile_coords(const AttnParams& a, int tile, int& q0, int& b1, int& b0) {
+  const int qt = tile % a.q_tiles, pr = tile / a.q_tiles;
+  q0 = qt * 128; b1 = pr % a.nb1; b0 = pr / a.nb1;
+}
+
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_constant__ CUtensorMap tk,
                      const __grid_constant__ CUtensorMap tv, const __grid_constant__ CUtensorMap tp, const AttnParams a) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - ptx::smem_addr(smem_raw));
-  const uint32_t q_s = base, k_s = base + kQBytes, p_s = base, v_s = base + kPBytes;
-  const uint32_t bars = v_s + kVBytes;
-  const uint32_t bar_qk = bars, bar_v = bars + 8, bar_s = bars + 16, bar_p = bars + 24, bar_o = bars + 32;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kPBytes + kVBytes + 64);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kPBytes + kVBytes + 68);
-  volatile float* row_max = reinterpret_cast<volatile float*>(gen + kPBytes + kVBytes + 128);   // [2][128]
-  volatile float* row_sum = row_max + 256;                                                        // [2][128]
+  const uint32_t q_s = base, k_s = q_s + kQBytes, v_s = k_s + kKBytes, pq_s = v_s + kVBytes;
+  constexpr uint32_t kData = kQBytes + kKBytes + kVBytes + 2 * kQuarterBytes;
+  const uint32_t bars = base + kData;
+  const uint32_t bar_qk = bars, bar_v = bars + 8, bar_s = bars + 16, bar_o = bars + 24, bar_tmem_free = bars + 32;
+  auto bar_full = [&](int b) { return bars + 40u + 8u * b; };     // weights of a quarter are in buffer b
+  auto bar_free = [&](int b) { return bars + 56u + 8u * b; };     // buffer b has been read by its MMAs and by its store
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kData + 80);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kData + 84);
+  volatile float* row_max = reinterpret_cast<volatile float*>(gen + kData + 128);   // [2][128]
+  volatile float* row_sum = row_max + 256;                                            // [2][128]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int q0 = blockIdx.x * 128, b1 = blockIdx.y, b0 = blockIdx.z;
+  const int num_tiles = a.q_tiles * a.nb1 * a.nb0;
   const int nkb = (a.s_k + 63) >> 6;                 // 64-key blocks with at least one key
+  const int nq = (nkb + 1) >> 1;                     // quarters (two key blocks, 128 keys) with at least one key
   const bool two_halves = a.s_k > 256;
+  const uint32_t kv_bytes = (two_halves ? 2u : 1u) * 256u * 128u;
 
   if (threadIdx.x == 0) {
-    ptx::mbar_init(bar_qk, 1); ptx::mbar_init(bar_v, 1); ptx::mbar_init(bar_s, 1);
-    ptx::mbar_init(bar_p, kSoftmaxWarps); ptx::mbar_init(bar_o, 1);
+    ptx::mbar_init(bar_qk, 1); ptx::mbar_init(bar_v, 1); ptx::mbar_init(bar_s, 1); ptx::mbar_init(bar_o, 1);
+    ptx::mbar_init(bar_tmem_free, kSoftmaxWarps);
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(bar_full(b), kSoftmaxWarps); ptx::mbar_init(bar_free(b), 2); }
     *abort_flag = 0;
     ptx::mbar_init_fence();
   }
@@ -93,93 +113,151 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
 
   if (warp == 0) {
     if (lane == 0) {
-      // ---------------------------------------------------------------- loads
-      ptx::mbar_expect_tx(bar_qk, kQBytes + (two_halves ? 2u : 1u) * 256u * 128u);
-      ptx::tma_load_4d(q_s, &tq, bar_qk, 0, q0, b1, b0);
-      ptx::tma_load_4d(k_s, &tk, bar_qk, 0, 0, b1, b0);
-      if (two_halves) ptx::tma_load_4d(k_s + 256u * 128u, &tk, bar_qk, 0, 256, b1, b0);
-      ptx::mbar_expect_tx(bar_v, (two_halves ? 2u : 1u) * 256u * 128u);
-      ptx::tma_load_4d(v_s, &tv, bar_v, 0, 0, b1, b0);
-      if (two_halves) ptx::tma_load_4d(v_s + 256u * 128u, &tv, bar_v, 0, 256, b1, b0);
-      // ---------------------------------------------------------------- S = Q K^T
-      bool ok = wait_bounded(bar_qk, 0, abort_flag, a.status, a.wait_limit);
-      if (ok) {
+      // ---------------------------------------------------------------- TMA loads and both MMA chains
+      auto load_qk = [&](int tile) {
+        int q0, b1, b0;
+        attn_tile_coords(a, tile, q0, b1, b0);
+        ptx::mbar_expect_tx(bar_qk, kQBytes + kv_bytes);
+        ptx::tma_load_4d(q_s, &tq, bar_qk, 0, q0, b1, b0);
+        ptx::tma_load_4d(k_s, &tk, bar_qk, 0, 0, b1, b0);
+        if (two_halves) ptx::tma_load_4d(k_s + 256u * 128u, &tk, bar_qk, 0, 256, b1, b0);
+      };
+      auto load_v = [&](int tile) {
+        int q0, b1, b0;
+        attn_tile_coords(a, tile, q0, b1, b0);
+        ptx::mbar_expect_tx(bar_v, kv_bytes);
+        ptx::tma_load_4d(v_s, &tv, bar_v, 0, 0, b1, b0);
+        if (two_halves) ptx::tma_load_4d(v_s + 256u * 128u, &tv, bar_v, 0, 256, b1, b0);
+      };
+      bool qk_pending = false, v_pending = false;             // a load has been issued and not yet waited for ...
+      uint32_t qk_phase = 0, v_phase = 0;                      // ... on this phase of its barrier
+      if ((int)blockIdx.x < num_tiles) { load_qk(blockIdx.x); load_v(blockIdx.x); qk_pending = v_pending = true; }
+      uint32_t fill0 = 0, fill1 = 0;                           // uses of each weight buffer so far
+      bool ok = true;
+      int n = 0;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++n) {
+        const uint32_t ph = (uint32_t)n & 1u;
+        const int next = tile + (int)gridDim.x;
+        ok = wait_bounded(bar_qk, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        qk_pending = false;
+        if (n > 0) {                                           // the previous tile's context has left tensor memory
+          ok = wait_bounded(bar_tmem_free, ph ^ 1u, abort_flag, a.status, a.wait_limit);
+          if (!ok) break;
+        }
         ptx::tc_fence_after_sync();
         const uint64_t qd = ptx::smem_desc_sw128(q_s, 16, 1024);
         for (int h = 0; h < (two_halves ? 2 : 1); ++h) {
           const uint64_t kd = ptx::smem_desc_sw128(k_s + (uint32_t)h * 256u * 128u, 16, 1024);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)                     // 16 of the 64 head columns (32 bytes) per MMA
+          for (int k = 0; k < 4; ++k)                          // 16 of the 64 head columns (32 bytes) per MMA
             ptx::mma_ss<false>(tmem + 256u * h, qd + 2u * k, kd + 2u * k, a.idesc_s, k > 0);
         }
         ptx::mma_commit(bar_s);
-        // -------------------------------------------------------------- C = P V once the weights are in shared memory
-        ok = wait_bounded(bar_p, 0, abort_flag, a.status, a.wait_limit) &&
-             wait_bounded(bar_v, 0, abort_flag, a.status, a.wait_limit);
-      }
-      if (ok) {
-        ptx::tc_fence_after_sync();
-        for (int kb = 0; kb < nkb; ++kb) {
-          const uint64_t pd = ptx::smem_desc_sw128(p_s + (uint32_t)kb * kKeyBlockBytes, 16, 1024);
-          const uint64_t vd = ptx::smem_desc_sw128(v_s + (uint32_t)kb * 8192u, 8192, 1024);
+        // Q and K may be overwritten once those MMAs have read them: fetch the next tile's
+        ok = wait_bounded(bar_s, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        if (next < num_tiles) { load_qk(next); qk_pending = true; qk_phase = ph ^ 1u; }
+        ok = wait_bounded(bar_v, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        v_pending = false;
+        // ---------------------------------------------------------------- C = P V, quarter by quarter
+        for (int qd4 = 0; ok && qd4 < nq; ++qd4) {
+          const int b = qd4 & 1;
+          ok = wait_bounded(bar_full(b), (b ? fill1 : fill0) & 1u, abort_flag, a.status, a.wait_limit);
+          if (!ok) break;
+          if (b) ++fill1; else ++fill0;
+          ptx::tc_fence_after_sync();
+          for (int kbl = 0; kbl < 2; ++kbl) {
+            const int kb = 2 * qd4 + kbl;
+            if (kb >= nkb) break;
+            const uint64_t pd = ptx::smem_desc_sw128(pq_s + (uint32_t)b * kQuarterBytes + (uint32_t)kbl * kKeyBlockBytes, 16, 1024);
+            const uint64_t vd = ptx::smem_desc_sw128(v_s + (uint32_t)kb * 8192u, 8192, 1024);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)                     // 16 keys per MMA: 32 bytes along a P row, 16 rows of V
-            ptx::mma_ss<false>(tmem, pd + 2u * k, vd + 128u * k, a.idesc_c, (kb | k) != 0);
+            for (int k = 0; k < 4; ++k)                        // 16 keys per MMA: 32 bytes along a P row, 16 rows of V
+              ptx::mma_ss<false>(tmem, pd + 2u * k, vd + 128u * k, a.idesc_c, (kb | k) != 0);
+          }
+          ptx::mma_commit(bar_free(b));                        // one of the two arrivals that free the buffer
         }
+        if (!ok) break;
         ptx::mma_commit(bar_o);
-        if (a.store_p) {
-          for (int kb = 0; kb < nkb; ++kb)
-            ptx::tma_store_4d(&tp, p_s + (uint32_t)kb * kKeyBlockBytes, kb * 64, q0, b1, b0);
-          ptx::bulk_commit_group();
-        }
+        // V may be overwritten once the last of those MMAs has read it
+        ok = wait_bounded(bar_o, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        if (next < num_tiles) { load_v(next); v_pending = true; v_phase = ph ^ 1u; }
       }
       if (*abort_flag) {
         // loads that were issued land before the CTA gives up its shared memory
-        for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_qk, 0); ++it) {}
-        for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_v, 0); ++it) {}
+        if (qk_pending) for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_qk, qk_phase); ++it) {}
+        if (v_pending) for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_v, v_phase); ++it) {}
       }
-      ptx::bulk_wait_group_read<0>();                      // the stored P has left shared memory
     }
-  } else if (warp >= 2) {
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- the stored weights leave by TMA store
+      uint32_t fill0 = 0, fill1 = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        int q0, b1, b0;
+        attn_tile_coords(a, tile, q0, b1, b0);
+        for (int qd4 = 0; ok && qd4 < nq; ++qd4) {
+          const int b = qd4 & 1;
+          ok = wait_bounded(bar_full(b), (b ? fill1 : fill0) & 1u, abort_flag, a.status, a.wait_limit);
+          if (!ok) break;
+          if (b) ++fill1; else ++fill0;
+          if (a.store_p) {
+            for (int kbl = 0; kbl < 2; ++kbl) {
+              const int kb = 2 * qd4 + kbl;
+              if (kb < nkb)
+                ptx::tma_store_4d(&tp, pq_s + (uint32_t)b * kQuarterBytes + (uint32_t)kbl * kKeyBlockBytes, kb * 64, q0, b1, b0);
+            }
+            ptx::bulk_commit_group();
+            ptx::bulk_wait_group_read<0>();                    // the store has read the buffer
+          }
+          ptx::mbar_arrive(bar_free(b));                       // the other arrival that frees it
+        }
+      }
+      ptx::bulk_wait_group_read<0>();
+    }
+  } else {
     // ------------------------------------------------------------------ softmax and output
     // Two warps share each TMEM lane quarter (= 32 query rows, one per lane): warp (q, part) works on the
     // 32-column chunks c = 2 i + part of its rows, and the two exchange their partial row maximum and row
     // sum through shared memory.
     const int q = warp & 3, part = (warp - 2) >> 2, r = q * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(q * 32) << 16);
-    const bool have_scores = wait_bounded(bar_s, 0, abort_flag, a.status, a.wait_limit);
-    // every softmax thread reaches this barrier whatever its wait returned, and the reduction hands all of them
-    // the same answer, so either all or none go on to the barriers below
-    bool ok = !ptx::named_barrier_any(1, 32 * kSoftmaxWarps, !have_scores);
-    if (ok) {
-      ptx::tc_fence_after_sync();
-      // One sweep over this warp's chunks c = part, part + 2, ...: the load of the next chunk is in flight
-      // while body(c, registers) works on the current one.
-      const int c_end = 2 * nkb;
-      auto sweep = [&](auto&& body) {
-        uint32_t ra[32], rb[32];
-        int c = part;
-        if (c < c_end) ptx::tmem_ld_32x32_issue(t_row + 32u * c, ra);
-        while (c < c_end) {
-          ptx::tmem_ld_fence(ra);
-          if (c + 2 < c_end) ptx::tmem_ld_32x32_issue(t_row + 32u * (c + 2), rb);
-          body(c, ra);
-          c += 2;
-          if (c >= c_end) break;
-          ptx::tmem_ld_fence(rb);
-          if (c + 2 < c_end) ptx::tmem_ld_32x32_issue(t_row + 32u * (c + 2), ra);
-          body(c, rb);
-          c += 2;
-        }
-      };
-      // columns at and beyond s_k hold products with zero-filled key rows: they are kept out of the maximum and
-      // the sum by replacing them with a very negative score, whose weight is exactly zero
-      auto mask = [&](int c, uint32_t (&x)[32]) {
-        if (32 * c + 32 > a.s_k) {
+    const int c_end = 2 * nkb;
+    // One sweep over this warp's chunks c = part, part + 2, ...
+    auto sweep = [&](auto&& body) {
+#pragma unroll 1
+      for (int c = part; c < c_end; c += 2) {
+        uint32_t x[32];
+        ptx::tmem_ld_32x32_issue(t_row + 32u * c, x);
+        ptx::tmem_ld_fence(x);
+        body(c, x);
+      }
+    };
+    // columns at and beyond s_k hold products with zero-filled key rows: they are kept out of the maximum and
+    // the sum by replacing them with a very negative score, whose weight is exactly zero
+    auto mask = [&](int c, uint32_t (&x)[32]) {
+      if (32 * c + 32 > a.s_k) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) if (32 * c + i >= a.s_k) x[i] = __float_as_uint(-3.0e38f);
-        }
-      };
+        for (int i = 0; i < 32; ++i) if (32 * c + i >= a.s_k) x[i] = __float_as_uint(-3.0e38f);
+      }
+    };
+    uint32_t fill0 = 0, fill1 = 0;
+    bool aborted = false;                                      // this warp gave up on a wait (it still joins the barriers below)
+    int n = 0;
+#pragma unroll 1
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++n) {
+      const uint32_t ph = (uint32_t)n & 1u;
+      const bool have_scores = !aborted && wait_bounded(bar_s, ph, abort_flag, a.status, a.wait_limit);
+      // every softmax thread reaches this barrier in every tile whatever its waits returned, and the reduction
+      // hands all of them the same answer, so either all or none go on to the barriers below
+      if (ptx::named_barrier_any(1, 32 * kSoftmaxWarps, !have_scores)) break;
+      ptx::tc_fence_after_sync();
+      int q0, b1, b0;
+      attn_tile_coords(a, tile, q0, b1, b0);
       float m4[4] = {-3.0e38f, -3.0e38f, -3.0e38f, -3.0e38f};
       sweep([&](int c, uint32_t (&x)[32]) {
         mask(c, x);
@@ -192,48 +270,65 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
       float s4[4] = {0.f, 0.f, 0.f, 0.f};
       sweep([&](int c, uint32_t (&x)[32]) {
         mask(c, x);
-        float e[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          e[i] = ex2(fmaf(__uint_as_float(x[i]), a.exp_scale, -mk));
-          s4[i & 3] += e[i];
+          const float e = ex2(fmaf(__uint_as_float(x[i]), a.exp_scale, -mk));
+          s4[i & 3] += e;
+          x[i] = __float_as_uint(e);
         }
-        ptx::tmem_st_32x32(t_row + 32u * c, e);              // the exponentials replace the scores
+        ptx::tmem_st_32x32_bits(t_row + 32u * c, x);           // the exponentials replace the scores
       });
       ptx::tmem_st_wait();
       row_sum[part * 128 + r] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
       ptx::named_barrier_sync(1, 32 * kSoftmaxWarps);
       const float inv = a.softmax_scale / (row_sum[r] + row_sum[128 + r]);
       const uint32_t row_off = (uint32_t)r * 128u, sw = (uint32_t)(r & 7);
-      sweep([&](int c, uint32_t (&x)[32]) {
-        const uint32_t blk = p_s + (uint32_t)(c >> 1) * kKeyBlockBytes + row_off;
+      // weights, a quarter (128 keys, four chunks, two of them this warp's) at a time into the two buffers in turn
+#pragma unroll 1
+      for (int qd4 = 0; qd4 < nq && !aborted; ++qd4) {
+        const int b = qd4 & 1;
+        bool free_ok = wait_bounded(bar_free(b), ((b ? fill1 : fill0) & 1u) ^ 1u, abort_flag, a.status, a.wait_limit);
+        free_ok = __all_sync(0xffffffffu, free_ok);
+        if (!free_ok) { aborted = true; break; }
+        if (b) ++fill1; else ++fill0;
+#pragma unroll 1
+        for (int c = 4 * qd4 + part; c < 4 * qd4 + 4 && c < c_end; c += 2) {
+          float v[32];
+          ptx::tmem_ld_32x32(t_row + 32u * c, v);
+          const uint32_t blk = pq_s + (uint32_t)b * kQuarterBytes + (uint32_t)((c >> 1) & 1) * kKeyBlockBytes + row_off;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint32_t w[4];
+          for (int g = 0; g < 4; ++g) {
+            uint32_t w[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float p0 = __uint_as_float(x[8 * g + 2 * j]) * inv, p1 = __uint_as_float(x[8 * g + 2 * j + 1]) * inv;
-            w[j] = a.op_bf16 ? pack_bf16x2(p0, p1) : pack_f16x2(p0, p1);
+            for (int j = 0; j < 4; ++j) {
+              const float p0 = v[8 * g + 2 * j] * inv, p1 = v[8 * g + 2 * j + 1] * inv;
+              w[j] = a.op_bf16 ? pack_bf16x2(p0, p1) : pack_f16x2(p0, p1);
+            }
+            const uint32_t chunk16 = (uint32_t)((c & 1) * 4 + g);
+            ptx::sts128(blk + ((chunk16 ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
           }
-          const uint32_t chunk16 = (uint32_t)((c & 1) * 4 + g);
-          ptx::sts128(blk + ((chunk16 ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
         }
-      });
-      ptx::fence_proxy_async_smem();                         // the MMA and the TMA store read these bytes
-      ptx::tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(bar_p);
+        ptx::fence_proxy_async_smem();                         // the MMA and the TMA store read these bytes
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar_full(b));
+      }
+      if (aborted) continue;
       // ---------------------------------------------------------------- context: this warp's 32 of the 64 columns
-      ok = wait_bounded(bar_o, 0, abort_flag, a.status, a.wait_limit);
+      bool ok = wait_bounded(bar_o, ph, abort_flag, a.status, a.wait_limit);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok) {
-        ptx::tc_fence_after_sync();
+      if (!ok) { aborted = true; continue; }
+      ptx::tc_fence_after_sync();
+      {
         const int row = q0 + r;
         const int es = dtype_size(a.c_dt);
         char* dst = static_cast<char*>(a.c) +
                     ((int64_t)b0 * a.c_stride0 + (int64_t)b1 * a.c_stride1 + (int64_t)row * a.c_ld + 32 * part) * es;
         float v[32];
         ptx::tmem_ld_32x32(t_row + 32u * part, v);
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar_tmem_free);        // the next tile's scores may overwrite the context
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] *= a.alpha_context;
         if (row < a.s_q) store_vec<32>(dst, a.c_dt, v);
@@ -345,7 +440,12 @@ extern "C" us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us
 
   if (cudaFuncSetAttribute(attention_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmem) != cudaSuccess)
     return US_ERR_CUDA;
-  const dim3 grid((unsigned)((s_q + 127) / 128), (unsigned)cnt[1], (unsigned)cnt[0]);
+  a.q_tiles = (int)((s_q + 127) / 128); a.nb1 = (int)cnt[1]; a.nb0 = (int)cnt[0];
+  const int64_t tiles = (int64_t)a.q_tiles * cnt[1] * cnt[0];
+  if (tiles > 0x7fffffff) return US_ERR_INVALID_ARG;
+  const int sms = host::sm_count();
+  if (sms <= 0) return US_ERR_CUDA;
+  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);    // persistent: one CTA per SM walks the tiles
   attention_fwd_kernel<<<grid, kAttnThreads, kAttnSmem, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, tp, a);
   return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }
