@@ -1,9 +1,12 @@
 """Runs a few eager passes of the FFN block so that a profiler can attach to individual launches.
 
     python -m paper_2303_11257_b200.profile_case [--tokens 8192] [--passes 2] [--operand fp8]
+    python -m paper_2303_11257_b200.profile_case --case attention [--passes 2]
 
 Each pass is the launches of UnitScaledFFN.step (one fused cast, six GEMMs) at d_model = 1024, d_ff = 4096.  At the default
 size the process holds well under 2 GB on the device and a pass lasts a fraction of a millisecond.
+--case attention: passes of the fused attention forward launch (us_attention_fwd) at 16 sequences x 16 heads x 512
+tokens x 64 (BF16 operands, E4M3 context, weights stored): about 0.3 GB on the device.
 """
 from __future__ import annotations
 
@@ -11,7 +14,24 @@ import argparse
 
 import torch
 
-from . import ffn, synth
+from . import ffn, lib as L, synth
+
+
+def attention(passes: int):
+    nseq, nhead, s, hd = 16, 16, 512, 64
+    d, T = nhead * hd, nseq * s
+    qkv = torch.from_numpy(synth.normal(0, 0, (T, 3 * d))).cuda().to(torch.bfloat16)
+    P = torch.empty(nseq * nhead * s, s, device="cuda", dtype=torch.bfloat16)
+    Cq = torch.empty(T, d, device="cuda", dtype=torch.uint8).view(torch.float8_e4m3fn)
+    ws = L.new_workspace("cuda")
+    st, td, sq = (s * 3 * d, hd), (s * d, hd), (nhead * s * s, s * s)
+    bt = L.attention_batch((nseq, nhead), st, st, st, td, sq)
+    sc = L.us_scales_attention(s, hd)
+    for _ in range(passes):
+        L.us_attention_fwd(qkv[:s, 0:hd], qkv[:s, d:d + hd], qkv[:s, 2 * d:2 * d + hd], sc["alpha_s"], sc["sm"], sc["alpha_c"],
+                           Cq[:s, :hd], P[:s], bt, ws)
+    assert L.us_workspace_status(ws) == 0
+    print("ok attention", passes)
 
 
 def main():
@@ -19,7 +39,10 @@ def main():
     ap.add_argument("--tokens", type=int, default=8192)
     ap.add_argument("--passes", type=int, default=2)
     ap.add_argument("--operand", default="fp8")
+    ap.add_argument("--case", default="ffn", choices=["ffn", "attention"])
     a = ap.parse_args()
+    if a.case == "attention":
+        return attention(a.passes)
     shape = synth.FFNShape("profile", a.tokens, 1024, 4096)
     tensors = [torch.from_numpy(t).cuda() for t in synth.ffn_tensors(shape, seed=0)]
     blk = ffn.UnitScaledFFN(shape.tokens, shape.d_model, shape.d_ff, operand=a.operand)
