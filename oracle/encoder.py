@@ -9,8 +9,9 @@ weights, E5 gradients); the attention matmuls take 16-bit operands (att = "bf16"
 att = "fp8", FP8 operands like every other matmul (section "Experiments": all matmul inputs are
 quantised): Q, K, V and the softmax output P as E4, the gradients dC, dS and dQ, dK, dV as E5, while
 the softmax input S and the gradient dP of its output, which feed no matmul, stay in BF16.  Every
-stored intermediate is rounded to the format it is stored in; with fused_scores the scores are not
-stored between the first matmul and the softmax and therefore not rounded.
+stored intermediate is rounded to the format it is stored in; with fused_scores the scores (and, in the
+backward pass, the gradient of the softmax output) are not stored between the matmul that makes them and
+the softmax (gradient) that consumes them, and therefore not rounded.
 
 norm = "post" adds the post-norm arrangement of the appendix "Model architectures"
 (res^PostNorm(f, z) = layernorm(interp(z, f(z)))): each of the two residual sums goes through a scaled
@@ -66,7 +67,8 @@ def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16"
     """norm = None: R2 = res(ffn, res(attention, X)), G = dL/dR2 (the FFN block's output r.ffn.R).
     norm = "post": ln = (w1, c1, w2, c2), each [d]; R1 = LN1(U1), R2 = LN2(U2) with U the residual sums.
     fused_scores: the scores S feed the softmax directly and are never stored, hence never rounded
-    (ops.attention_fwd); r.S then holds the unrounded scores."""
+    (ops.attention_fwd), and likewise the gradient dP of the weights in the backward pass
+    (ops.attention_bwd_scores); r.S and r.dP then hold the unrounded values."""
     T, d = X.shape
     hd = d // nhead
     f32 = lambda v: float(np.float32(v))
@@ -122,10 +124,14 @@ def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16"
     r.dC, _ = O.store(O.linear_bwd_x(g1q, Wo_q, b_o), f_grad)
     r.dWo, _ = O.store(O.linear_bwd_w(r.Cq, g1q, b_w), "f32")
     dC4 = _heads(r.dC, nseq, slen, nhead, hd, 0, d)
-    dP4, _ = O.store(f32(b_P) * (dC4 @ V.transpose(0, 1, 3, 2)), f_wide)           # beta_1 G W^T with W = V
     dV4 = f32(b_V) * (P4.transpose(0, 1, 3, 2) @ dC4)                           # beta_2 X^T G with X = P
-    dS4, _ = O.store(O.softmax_bwd(P4, dP4, sm, sm), f_grad)
-    dQ4 = f32(b_Q) * (dS4 @ K)
+    if fused_scores:
+        dP4 = f32(b_P) * (dC4 @ V.transpose(0, 1, 3, 2))                          # kept unrounded, like the scores
+        dS4, dQ4 = O.attention_bwd_scores(dC4, P4, K, V, b_P, sm, sm, b_Q, f_grad)
+    else:
+        dP4, _ = O.store(f32(b_P) * (dC4 @ V.transpose(0, 1, 3, 2)), f_wide)       # beta_1 G W^T with W = V
+        dS4, _ = O.store(O.softmax_bwd(P4, dP4, sm, sm), f_grad)
+        dQ4 = f32(b_Q) * (dS4 @ K)
     dK4 = f32(b_K) * (dS4.transpose(0, 1, 3, 2) @ Q)
     r.dP, r.dS = dP4.reshape(-1, slen), dS4.reshape(-1, slen)
     dQKV = np.concatenate([_unheads(t, nseq, slen, nhead, hd) for t in (dQ4, dK4, dV4)], axis=1)

@@ -168,6 +168,23 @@ def attention_fwd(Q, K, V, alpha_scores, softmax_scale, alpha_context, p_dtype: 
     return P, _f32(alpha_context) * (P @ V)
 
 
+def attention_bwd_scores(dC, P, K, V, beta_p, softmax_alpha, softmax_beta, beta_q, ds_dtype: str):
+    """Backward of attention_fwd down to the queries, with the gradient of the weights kept unrounded:
+
+        dP = beta_p * dC V^T                                  dC [s_q x d], V [s_k x d]      (never stored)
+        dS = store(softmax_beta * p (dP - sum_k p_k dP_k), ds_dtype),  p = P / softmax_alpha   [s_q x s_k]
+        dQ = beta_q * dS K                                    K [s_k x d]                      [s_q x d]
+
+    (matmul*_grad_1 with W = V for dP and the forward matmul form with W = K for dQ, section "Example"; the softmax
+    gradient of the table row "softmax").  P is the forward pass's stored output.  dS is a matmul input (of dQ here and
+    of dK = beta dS^T Q elsewhere) and is rounded to its operand format; dP feeds no matmul and no memory.
+    Returns (dS as stored, dQ unrounded).  Leading batch axes are allowed."""
+    dC, P, K, V = (np.asarray(t, np.float64) for t in (dC, P, K, V))
+    dP = _f32(beta_p) * (dC @ np.swapaxes(V, -1, -2))
+    dS, _ = store(softmax_bwd(P, dP, softmax_alpha, softmax_beta), ds_dtype)
+    return dS, _f32(beta_q) * (dS @ K)
+
+
 # --------------------------------------------------------------------------- softmax cross-entropy
 
 def softmax_xent_fwd(X, t):

@@ -96,3 +96,38 @@ def test_encoder_layer_with_unrounded_scores_differs_only_from_the_scores_on():
     assert np.array_equal(b.P, P.reshape(-1, slen))
     assert np.array_equal(b.Cq, F.quantise(E._unheads(C, nseq, slen, nhead, hd), F.FORMATS["e4m3"]))
     assert np.abs(a.P - b.P).max() < 0.05 * np.abs(a.P).max()             # close, not identical
+
+
+def test_backward_to_the_scores_by_finite_differences():
+    """dS and dQ of attention_bwd_scores are beta-scaled gradients of L = sum(G * (P V)) with P = alpha softmax(S):
+    central differences in S for dS (through the unscaled softmax, table row "softmax") and the plain products for dQ."""
+    rng = np.random.default_rng(5)
+    sq, sk, d = 3, 6, 4
+    Q, K, V = rng.standard_normal((sq, d)), rng.standard_normal((sk, d)), rng.standard_normal((sk, d))
+    G = rng.standard_normal((sq, d))
+    alpha, beta, b_p, b_q = 6.0, 6.0, 0.5, 0.25
+    S = 0.5 * Q @ K.T
+    P = O.softmax_fwd(S, alpha)
+    dS, dQ = O.attention_bwd_scores(G, P, K, V, b_p, alpha, beta, b_q, "f64")
+    fd = np.zeros_like(S)
+    h = 1e-6
+    for i in range(sq):
+        for j in range(sk):
+            E = np.zeros_like(S); E[i, j] = h
+            f = lambda s_: np.sum(G * (special.softmax(s_, axis=-1) @ V))       # unscaled ops
+            fd[i, j] = (f(S + E) - f(S - E)) / (2 * h)
+    assert np.allclose(dS, beta * b_p * fd, atol=1e-8)
+    assert np.allclose(dQ, b_q * dS @ K, rtol=1e-14)
+
+
+def test_backward_rows_sum_to_zero_and_uniform_gradient_vanishes():
+    rng = np.random.default_rng(6)
+    s, d = 40, 8
+    P = O.softmax_fwd(rng.standard_normal((5, s)), float(s))
+    K, V = rng.standard_normal((s, d)), rng.standard_normal((s, d))
+    dS, _ = O.attention_bwd_scores(rng.standard_normal((5, d)), P, K, V, d ** -0.5, float(s), float(s), d ** -0.5, "f64")
+    assert np.abs(dS.sum(axis=1)).max() < 1e-12                      # softmax gradients are orthogonal to 1
+    # every value row equal: dP is constant along a row, so dS = 0
+    Vc = np.tile(rng.standard_normal((1, d)), (s, 1))
+    dS0, dQ0 = O.attention_bwd_scores(rng.standard_normal((5, d)), P, K, Vc, 1.0, float(s), float(s), 1.0, "bf16")
+    assert np.abs(dS0).max() < 1e-12 and np.abs(dQ0).max() < 1e-10
