@@ -329,6 +329,32 @@ us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us_mat* V, fl
                            float alpha_context, const us_mat* C, const us_mat* P, const us_attention_batch* batch,
                            void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * us_attention_bwd: the backward pass of us_attention_fwd down to the queries, in one launch:
+ *
+ *   dP = beta_p * dC V^T                                           score-sized, never stored and never rounded
+ *   dS = softmax_beta * p (dP - sum_k p_k dP_k),  p = P / softmax_alpha    rounded to the operands' 16-bit format
+ *   dQ = beta_q * dS K
+ *
+ * dC [s_q x 64] is the gradient of the context, P [s_q x s_k] the weights the forward call stored, K and V [s_k x 64].
+ * dS [s_q x s_k] is written for the caller's dK = beta dS^T Q matmul (dV = beta P^T dC needs only P and dC); dQ
+ * [s_q x 64] in any us_dtype.  dC, P, K, V and dS: all BF16 or all F16.  Shapes, limits, batch description (one stride
+ * pair per tensor), alignment, workspace and errors as for us_attention_fwd; softmax_alpha must be positive.
+ */
+typedef struct {
+  int64_t count[2];
+  int64_t dc_stride[2];
+  int64_t p_stride[2];
+  int64_t k_stride[2];
+  int64_t v_stride[2];
+  int64_t ds_stride[2];
+  int64_t dq_stride[2];
+} us_attention_bwd_batch;
+
+us_status us_attention_bwd(const us_mat* dC, const us_mat* P, const us_mat* K, const us_mat* V, float beta_p,
+                           float softmax_alpha, float softmax_beta, float beta_q, const us_mat* dS, const us_mat* dQ,
+                           const us_attention_bwd_batch* batch, void* ws, size_t ws_bytes, void* stream);
+
 /* ------------------------------------------------------------ scaled softmax
  *
  * Row-wise scaled softmax and its gradient (table "Table of unit scaling factors", row softmax:

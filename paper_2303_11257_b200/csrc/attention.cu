@@ -340,6 +340,257 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
   if (warp == 1) { ptx::tc_fence_after_sync(); ptx::tmem_dealloc(tmem, 512); }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Backward pass down to the queries, one persistent kernel of the same shape as the forward one: per tile of 128
+// query rows
+//     dP = beta_p * dC V^T            score-sized, float32 in tensor memory only (never stored, never rounded)
+//     dS = k * P (dP - sum_j P_j dP_j / alpha)     the scaled-softmax gradient, from the forward pass's stored P
+//     dQ = beta_q * dS K
+// dC [128 x 64] and V arrive by TMA, the MMAs of dC V^T fill the 512 TMEM columns; the tile of P (128 x 512, the layout
+// the forward kernel stored it from) arrives in shared memory; eight warps pass twice over their rows (row sums of
+// P dP; then dS, rounded and written over P in place); K replaces V in its buffer as soon as the first MMA chain has
+// read V, and a second chain multiplies dS (A operand, from the same shared-memory tile) by K into TMEM columns
+// 0..63; the tile of dS leaves by TMA store (the dK matmul reads it), the eight warps scale and store dQ.
+struct AttnBwdParams {
+  int s_q, s_k;
+  int q_tiles, nb1, nb0;
+  float inv_alpha;          // 1 / softmax_alpha
+  float ds_scale;           // softmax_beta * beta_p / softmax_alpha
+  float beta_q;
+  void* dq; int dq_dt; int64_t dq_ld, dq_stride0, dq_stride1;
+  int op_bf16;
+  uint32_t idesc_s, idesc_c;
+  unsigned int* status;
+  uint32_t wait_limit;
+};
+
+constexpr uint32_t kTileBytes = 8 * kKeyBlockBytes;      // a 128 x 512 tile of 16-bit weights: 128 KB
+constexpr uint32_t kAttnBwdSmem = kQBytes + kKBytes + kTileBytes + 1024 + 128 + 1024;
+
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_constant__ CUtensorMap tv,
+                     const __grid_constant__ CUtensorMap tk, const __grid_constant__ CUtensorMap tp,
+                     const __grid_constant__ CUtensorMap tds, const AttnBwdParams a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (ptx::smem_addr(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - ptx::smem_addr(smem_raw));
+  const uint32_t dc_s = base, kv_s = dc_s + kQBytes, ps_s = kv_s + kKBytes;
+  constexpr uint32_t kData = kQBytes + kKBytes + kTileBytes;
+  const uint32_t bars = base + kData;
+  const uint32_t bar_in = bars, bar_pin = bars + 8, bar_dp = bars + 16, bar_k = bars + 24, bar_ds = bars + 32,
+                 bar_dq = bars + 40, bar_tmem_free = bars + 48, bar_ps_free = bars + 56;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kData + 64);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kData + 68);
+  volatile float* row_sum = reinterpret_cast<volatile float*>(gen + kData + 128);     // [2][128]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_tiles = a.q_tiles * a.nb1 * a.nb0;
+  const int nkb = (a.s_k + 63) >> 6;
+  const bool two_halves = a.s_k > 256;
+  const uint32_t kv_bytes = (two_halves ? 2u : 1u) * 256u * 128u;
+  auto coords = [&](int tile, int& q0, int& b1, int& b0) {
+    const int qt = tile % a.q_tiles, pr = tile / a.q_tiles;
+    q0 = qt * 128; b1 = pr % a.nb1; b0 = pr / a.nb1;
+  };
+
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(bar_in, 1); ptx::mbar_init(bar_pin, 1); ptx::mbar_init(bar_dp, 1); ptx::mbar_init(bar_k, 1);
+    ptx::mbar_init(bar_ds, kSoftmaxWarps); ptx::mbar_init(bar_dq, 1); ptx::mbar_init(bar_tmem_free, kSoftmaxWarps);
+    ptx::mbar_init(bar_ps_free, 1);
+    *abort_flag = 0;
+    ptx::mbar_init_fence();
+  }
+  if (warp == 1) { ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), 512); ptx::tmem_relinquish(); }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- TMA loads and both MMA chains
+      auto load_in = [&](int tile) {                           // dC tile and V
+        int q0, b1, b0;
+        coords(tile, q0, b1, b0);
+        ptx::mbar_expect_tx(bar_in, kQBytes + kv_bytes);
+        ptx::tma_load_4d(dc_s, &tdc, bar_in, 0, q0, b1, b0);
+        ptx::tma_load_4d(kv_s, &tv, bar_in, 0, 0, b1, b0);
+        if (two_halves) ptx::tma_load_4d(kv_s + 256u * 128u, &tv, bar_in, 0, 256, b1, b0);
+      };
+      auto load_p = [&](int tile) {                            // the tile of stored weights, key block by key block
+        int q0, b1, b0;
+        coords(tile, q0, b1, b0);
+        ptx::mbar_expect_tx(bar_pin, (uint32_t)nkb * kKeyBlockBytes);
+        for (int kb = 0; kb < nkb; ++kb) ptx::tma_load_4d(ps_s + (uint32_t)kb * kKeyBlockBytes, &tp, bar_pin, kb * 64, q0, b1, b0);
+      };
+      // phase of the latest load issued on each barrier (a wait on a phase that has completed returns at once)
+      bool in_issued = false, p_issued = false, k_issued = false;
+      uint32_t in_phase = 0, p_phase = 0, k_phase = 0;
+      if ((int)blockIdx.x < num_tiles) { load_in(blockIdx.x); load_p(blockIdx.x); in_issued = p_issued = true; }
+      bool ok = true;
+      int n = 0;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++n) {
+        const uint32_t ph = (uint32_t)n & 1u;
+        const int next = tile + (int)gridDim.x;
+        int q0, b1, b0;
+        coords(tile, q0, b1, b0);
+        ok = wait_bounded(bar_in, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        if (n > 0) {                                           // the previous tile's dQ has left tensor memory
+          ok = wait_bounded(bar_tmem_free, ph ^ 1u, abort_flag, a.status, a.wait_limit);
+          if (!ok) break;
+        }
+        ptx::tc_fence_after_sync();
+        const uint64_t cd = ptx::smem_desc_sw128(dc_s, 16, 1024);
+        for (int h = 0; h < (two_halves ? 2 : 1); ++h) {
+          const uint64_t vd = ptx::smem_desc_sw128(kv_s + (uint32_t)h * 256u * 128u, 16, 1024);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) ptx::mma_ss<false>(tmem + 256u * h, cd + 2u * k, vd + 2u * k, a.idesc_s, k > 0);
+        }
+        ptx::mma_commit(bar_dp);
+        // V has been read: K takes its place
+        ok = wait_bounded(bar_dp, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        ptx::mbar_expect_tx(bar_k, kv_bytes);
+        ptx::tma_load_4d(kv_s, &tk, bar_k, 0, 0, b1, b0);
+        if (two_halves) ptx::tma_load_4d(kv_s + 256u * 128u, &tk, bar_k, 0, 256, b1, b0);
+        k_issued = true; k_phase = ph;
+        ok = wait_bounded(bar_k, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        ok = wait_bounded(bar_ds, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        ptx::tc_fence_after_sync();
+        for (int kb = 0; kb < nkb; ++kb) {
+          const uint64_t sd = ptx::smem_desc_sw128(ps_s + (uint32_t)kb * kKeyBlockBytes, 16, 1024);
+          const uint64_t kd = ptx::smem_desc_sw128(kv_s + (uint32_t)kb * 8192u, 8192, 1024);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) ptx::mma_ss<false>(tmem, sd + 2u * k, kd + 128u * k, a.idesc_c, (kb | k) != 0);
+        }
+        ptx::mma_commit(bar_dq);
+        // dC, K and (for the MMAs) the dS tile have been read once those MMAs are done
+        ok = wait_bounded(bar_dq, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        if (next < num_tiles) { load_in(next); in_phase = ph ^ 1u; }
+        // ... and the tile's store has read it too: the next tile of P may land
+        ok = wait_bounded(bar_ps_free, ph, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        if (next < num_tiles) { load_p(next); p_phase = ph ^ 1u; }
+      }
+      if (*abort_flag) {
+        // loads that were issued land before the CTA gives up its shared memory
+        if (in_issued) for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_in, in_phase); ++it) {}
+        if (p_issued) for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_pin, p_phase); ++it) {}
+        if (k_issued) for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_k, k_phase); ++it) {}
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- dS leaves by TMA store
+      bool ok = true;
+      int n = 0;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++n) {
+        int q0, b1, b0;
+        coords(tile, q0, b1, b0);
+        ok = wait_bounded(bar_ds, (uint32_t)n & 1u, abort_flag, a.status, a.wait_limit);
+        if (!ok) break;
+        for (int kb = 0; kb < nkb; ++kb) ptx::tma_store_4d(&tds, ps_s + (uint32_t)kb * kKeyBlockBytes, kb * 64, q0, b1, b0);
+        ptx::bulk_commit_group();
+        ptx::bulk_wait_group_read<0>();
+        ptx::mbar_arrive(bar_ps_free);
+      }
+      ptx::bulk_wait_group_read<0>();
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax gradient and dQ
+    const int q = warp & 3, part = (warp - 2) >> 2, r = q * 32 + lane;
+    const uint32_t t_row = tmem + ((uint32_t)(q * 32) << 16);
+    const int c_end = 2 * nkb;
+    const uint32_t row_off = (uint32_t)r * 128u, sw = (uint32_t)(r & 7);
+    auto p_addr = [&](int c, int g) {                          // 16 bytes = columns 32 c + 8 g .. + 7 of this row
+      return ps_s + (uint32_t)(c >> 1) * kKeyBlockBytes + row_off + ((((uint32_t)((c & 1) * 4 + g)) ^ sw) << 4);
+    };
+    bool aborted = false;
+    int n = 0;
+#pragma unroll 1
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++n) {
+      const uint32_t ph = (uint32_t)n & 1u;
+      const bool have = !aborted && wait_bounded(bar_dp, ph, abort_flag, a.status, a.wait_limit) &&
+                        wait_bounded(bar_pin, ph, abort_flag, a.status, a.wait_limit);
+      if (ptx::named_barrier_any(1, 32 * kSoftmaxWarps, !have)) break;
+      ptx::tc_fence_after_sync();
+      int q0, b1, b0;
+      coords(tile, q0, b1, b0);
+      // pass 1: sum_j P_j dP_j over this warp's chunks (columns beyond s_k hold zeros in both factors)
+      float s4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+      for (int c = part; c < c_end; c += 2) {
+        float x[32];
+        ptx::tmem_ld_32x32(t_row + 32u * c, x);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const uint4 raw = ptx::lds128(p_addr(c, g));
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float2 pv = a.op_bf16 ? unpack_bf16x2(w[j]) : unpack_f16x2(w[j]);
+            s4[j] = fmaf(pv.x, x[8 * g + 2 * j], s4[j]);
+            s4[j] = fmaf(pv.y, x[8 * g + 2 * j + 1], s4[j]);
+          }
+        }
+      }
+      row_sum[part * 128 + r] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+      ptx::named_barrier_sync(1, 32 * kSoftmaxWarps);
+      const float mean = (row_sum[r] + row_sum[128 + r]) * a.inv_alpha;     // sum_j p_j dP_j in units of the raw accumulator
+      // pass 2: dS = ds_scale * P * (dP - mean), rounded, over P in place
+#pragma unroll 1
+      for (int c = part; c < c_end; c += 2) {
+        float x[32];
+        ptx::tmem_ld_32x32(t_row + 32u * c, x);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const uint32_t addr = p_addr(c, g);
+          const uint4 raw = ptx::lds128(addr);
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+          uint32_t o[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float2 pv = a.op_bf16 ? unpack_bf16x2(w[j]) : unpack_f16x2(w[j]);
+            const float d0 = a.ds_scale * pv.x * (x[8 * g + 2 * j] - mean), d1 = a.ds_scale * pv.y * (x[8 * g + 2 * j + 1] - mean);
+            o[j] = a.op_bf16 ? pack_bf16x2(d0, d1) : pack_f16x2(d0, d1);
+          }
+          ptx::sts128(addr, make_uint4(o[0], o[1], o[2], o[3]));
+        }
+      }
+      ptx::fence_proxy_async_smem();                           // the MMA and the TMA store read these bytes
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(bar_ds);
+      // ---------------------------------------------------------------- dQ: this warp's 32 of the 64 columns
+      bool ok = wait_bounded(bar_dq, ph, abort_flag, a.status, a.wait_limit);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { aborted = true; continue; }
+      ptx::tc_fence_after_sync();
+      {
+        const int row = q0 + r;
+        const int es = dtype_size(a.dq_dt);
+        char* dst = static_cast<char*>(a.dq) +
+                    ((int64_t)b0 * a.dq_stride0 + (int64_t)b1 * a.dq_stride1 + (int64_t)row * a.dq_ld + 32 * part) * es;
+        float v[32];
+        ptx::tmem_ld_32x32(t_row + 32u * part, v);
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(bar_tmem_free);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] *= a.beta_q;
+        if (row < a.s_q) store_vec<32>(dst, a.dq_dt, v);
+      }
+    }
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) { ptx::tc_fence_after_sync(); ptx::tmem_dealloc(tmem, 512); }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -447,5 +698,71 @@ extern "C" us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us
   if (sms <= 0) return US_ERR_CUDA;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);    // persistent: one CTA per SM walks the tiles
   attention_fwd_kernel<<<grid, kAttnThreads, kAttnSmem, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, tp, a);
+  return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
+}
+
+extern "C" us_status us_attention_bwd(const us_mat* dC, const us_mat* P, const us_mat* K, const us_mat* V, float beta_p,
+                                      float softmax_alpha, float softmax_beta, float beta_q, const us_mat* dS,
+                                      const us_mat* dQ, const us_attention_bwd_batch* batch, void* ws, size_t ws_bytes,
+                                      void* stream) {
+  using namespace us;
+  if (!dC || !P || !K || !V || !dS || !dQ || !batch) return US_ERR_INVALID_ARG;
+  const int64_t* cnt = batch->count;
+  if (cnt[0] < 1 || cnt[1] < 1 || cnt[0] > 65535 || cnt[1] > 65535) return US_ERR_INVALID_ARG;
+  const us_mat* all[6] = {dC, P, K, V, dS, dQ};
+  const int64_t* strides[6] = {batch->dc_stride, batch->p_stride, batch->k_stride, batch->v_stride, batch->ds_stride,
+                               batch->dq_stride};
+  for (int i = 0; i < 6; ++i) {
+    const us_mat* m = all[i];
+    if (m->rows < 0 || m->cols < 0 || m->ld < m->cols) return US_ERR_INVALID_ARG;
+    if (m->rows * m->cols > 0 && !m->ptr) return US_ERR_INVALID_ARG;
+    for (int j = 0; j < 2; ++j)
+      if (cnt[j] > 1 && strides[i][j] <= 0) return US_ERR_INVALID_ARG;
+  }
+  const int64_t s_q = dC->rows, s_k = K->rows;
+  if (K->cols != dC->cols || V->cols != dC->cols || V->rows != s_k || P->rows != s_q || P->cols != s_k || dS->rows != s_q ||
+      dS->cols != s_k || dQ->rows != s_q || dQ->cols != dC->cols)
+    return US_ERR_INVALID_ARG;
+  if (!(softmax_alpha > 0.f)) return US_ERR_INVALID_ARG;
+  const bool h16 = (dC->dtype == US_BF16 || dC->dtype == US_F16) && K->dtype == dC->dtype && V->dtype == dC->dtype &&
+                   P->dtype == dC->dtype && dS->dtype == dC->dtype;
+  if (!h16) return US_ERR_UNSUPPORTED;
+  if (dQ->dtype < US_F32 || dQ->dtype > US_E5M2) return US_ERR_UNSUPPORTED;
+  if (dC->cols != kAttnD || s_k > kAttnMaxKeys) return US_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < us_workspace_bytes()) return US_ERR_WORKSPACE;
+  if (s_q == 0 || s_k == 0) return US_OK;              // no queries: nothing to do; no keys: dS is empty and dQ is not written
+  const int q_es = (int)dtype_size(dQ->dtype);
+  for (int i = 0; i < 5; ++i)
+    if (!ok16(all[i], strides[i], cnt, 2)) return US_ERR_ALIGNMENT;
+  if (!ok16(dQ, batch->dq_stride, cnt, q_es)) return US_ERR_ALIGNMENT;
+
+  CUtensorMap tdc, tv, tk, tp, tds;
+  if (!attn_tmap(&tdc, dC, batch->dc_stride, cnt, 128) || !attn_tmap(&tv, V, batch->v_stride, cnt, 256) ||
+      !attn_tmap(&tk, K, batch->k_stride, cnt, 256) || !attn_tmap(&tp, P, batch->p_stride, cnt, 128) ||
+      !attn_tmap(&tds, dS, batch->ds_stride, cnt, 128))
+    return US_ERR_CUDA;
+
+  AttnBwdParams a{};
+  a.s_q = (int)s_q; a.s_k = (int)s_k;
+  a.q_tiles = (int)((s_q + 127) / 128); a.nb1 = (int)cnt[1]; a.nb0 = (int)cnt[0];
+  a.inv_alpha = 1.0f / softmax_alpha;
+  a.ds_scale = softmax_beta * beta_p / softmax_alpha;
+  a.beta_q = beta_q;
+  a.dq = dQ->ptr; a.dq_dt = dQ->dtype; a.dq_ld = dQ->ld;
+  a.dq_stride0 = cnt[0] > 1 ? batch->dq_stride[0] : 0; a.dq_stride1 = cnt[1] > 1 ? batch->dq_stride[1] : 0;
+  a.op_bf16 = dC->dtype == US_BF16;
+  const int fmt = a.op_bf16 ? 1 : 0;
+  a.idesc_s = make_idesc(fmt, fmt, false, false, 128, 256);
+  a.idesc_c = make_idesc(fmt, fmt, false, true, 128, 64);
+  a.status = static_cast<unsigned int*>(ws);
+  a.wait_limit = kWaitLimit;
+  const int64_t tiles = (int64_t)a.q_tiles * cnt[1] * cnt[0];
+  if (tiles > 0x7fffffff) return US_ERR_INVALID_ARG;
+  const int sms = host::sm_count();
+  if (sms <= 0) return US_ERR_CUDA;
+  if (cudaFuncSetAttribute(attention_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnBwdSmem) != cudaSuccess)
+    return US_ERR_CUDA;
+  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+  attention_bwd_kernel<<<grid, kAttnThreads, kAttnBwdSmem, static_cast<cudaStream_t>(stream)>>>(tdc, tv, tk, tp, tds, a);
   return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }

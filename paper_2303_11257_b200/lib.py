@@ -47,6 +47,11 @@ class us_attention_batch(C.Structure):
                 ("v_stride", C.c_int64 * 2), ("c_stride", C.c_int64 * 2), ("p_stride", C.c_int64 * 2)]
 
 
+class us_attention_bwd_batch(C.Structure):
+    _fields_ = [("count", C.c_int64 * 2), ("dc_stride", C.c_int64 * 2), ("p_stride", C.c_int64 * 2), ("k_stride", C.c_int64 * 2),
+                ("v_stride", C.c_int64 * 2), ("ds_stride", C.c_int64 * 2), ("dq_stride", C.c_int64 * 2)]
+
+
 class us_linear_call(C.Structure):
     _fields_ = [("op", C.c_int32), ("a", us_mat), ("b", us_mat), ("scale", C.c_float), ("ep", us_epilogue), ("out", us_mat)]
 
@@ -82,6 +87,8 @@ def _load() -> C.CDLL:
         fn.restype = C.c_int
     lib.us_attention_fwd.argtypes = [MP, MP, MP, F, F, F, MP, MP, C.POINTER(us_attention_batch), V, SZ, V]
     lib.us_attention_fwd.restype = C.c_int
+    lib.us_attention_bwd.argtypes = [MP, MP, MP, MP, F, F, F, F, MP, MP, C.POINTER(us_attention_bwd_batch), V, SZ, V]
+    lib.us_attention_bwd.restype = C.c_int
     lib.us_linear_fwd_static_ws.argtypes = [MP, MP, F, EP, MP, C.POINTER(C.c_void_p), V]
     lib.us_linear_fwd_static_ws.restype = C.c_int
     lib.us_linear_fwd_check.argtypes = [MP, MP, EP, MP, V, SZ]
@@ -275,6 +282,24 @@ def us_attention_fwd(Q, K, V, alpha_scores, softmax_scale, alpha_context, Cx, P,
                                  alpha_context, C.byref(mat(Cx)), pp, C.byref(bt), ws.data_ptr(),
                                  ws.numel() * ws.element_size(), _stream(stream)))
     return Cx
+
+
+def attention_bwd_batch(count, dc_stride, p_stride, k_stride, v_stride, ds_stride, dq_stride) -> us_attention_bwd_batch:
+    b = us_attention_bwd_batch()
+    for i in range(2):
+        b.count[i] = count[i]
+        b.dc_stride[i], b.p_stride[i], b.k_stride[i] = dc_stride[i], p_stride[i], k_stride[i]
+        b.v_stride[i], b.ds_stride[i], b.dq_stride[i] = v_stride[i], ds_stride[i], dq_stride[i]
+    return b
+
+
+def us_attention_bwd(dC, P, K, V, beta_p, softmax_alpha, softmax_beta, beta_q, dS, dQ, bt, ws, stream=None):
+    """Attention backward down to the queries: dS (for the dK matmul) and dQ from dC, the stored P, K and V."""
+    _check("us_attention_bwd",
+           _lib.us_attention_bwd(C.byref(mat(dC)), C.byref(mat(P)), C.byref(mat(K)), C.byref(mat(V)), beta_p, softmax_alpha,
+                                 softmax_beta, beta_q, C.byref(mat(dS)), C.byref(mat(dQ)), C.byref(bt), ws.data_ptr(),
+                                 ws.numel() * ws.element_size(), _stream(stream)))
+    return dQ
 
 
 def us_linear_fwd_static_ws(X, W, alpha, Y, ep=None, stream=None) -> int:

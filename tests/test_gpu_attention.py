@@ -143,3 +143,82 @@ def test_argument_checks():
         L.us_attention_fwd(q, k, U.empty(64, 64, "bf16"), 0.125, 128.0, 0.1, c, None, bt, ws)
     assert e.value.status == L.US_ERR_INVALID_ARG                    # V rows != K rows
     L.us_attention_fwd(q[:0], k, k, 0.125, 128.0, 0.1, c[:0], None, bt, ws)   # no queries: nothing to do
+
+
+# ------------------------------------------------------------------------------------------------ backward
+
+def _run_bwd(nseq, nhead, s, fmt, dq_fmt, seed, scale=1.0):
+    """Weights P as the oracle's forward pass rounds them (uploaded bit patterns), random dC; returns host values of the
+    operands and the device outputs."""
+    from paper_2303_11257_b200 import lib as L, synth
+    hd, d, T = 64, nhead * 64, nseq * s
+    qkv = scale * synth.normal(seed, 0, (T, 3 * d))
+    dc = synth.normal(seed, 1, (T, d))
+    QKV, dCt = U.to_device(qkv, fmt), U.to_device(dc, fmt)
+    qkv_v, dc_v = U.values_of(qkv, fmt), U.values_of(dc, fmt)
+    Q, K, V = (_heads(qkv_v, nseq, s, nhead, i) for i in range(3))
+    a_s, sm, a_c = hd ** -0.5, float(s), s ** -0.5
+    p_host, _ = O.attention_fwd(Q, K, V, a_s, sm, a_c, fmt)                    # as stored by a forward pass
+    P = U.to_device(p_host.reshape(-1, s), fmt)
+    dS = U.empty(nseq * nhead * s, s, fmt)
+    dQ = U.empty(T, d, dq_fmt)
+    ws = L.new_workspace()
+    b_p, b_q = hd ** -0.5, hd ** -0.5
+    st, td, sq = (s * 3 * d, hd), (s * d, hd), (nhead * s * s, s * s)
+    bt = L.attention_bwd_batch((nseq, nhead), td, sq, st, st, sq, td)
+    L.us_attention_bwd(dCt[:s, :hd], P[:s], QKV[:s, d:d + hd], QKV[:s, 2 * d:2 * d + hd], b_p, sm, sm, b_q, dS[:s], dQ[:s, :hd], bt, ws)
+    assert L.us_workspace_status(ws) == 0
+    dC4 = dc_v.reshape(nseq, s, nhead, 64).transpose(0, 2, 1, 3)
+    return dC4, p_host, K, V, dS, dQ, (b_p, sm, b_q)
+
+
+@pytest.mark.parametrize("fmt", ["bf16", "fp16"])
+@pytest.mark.parametrize("nseq,nhead,s", [(2, 3, 128), (1, 2, 200), (2, 2, 512), (1, 1, 72), (1, 2, 264), (3, 1, 8)])
+def test_backward_scores_and_queries_against_the_oracle(fmt, nseq, nhead, s):
+    dC4, p_host, K, V, dS, dQ, (b_p, sm, b_q) = _run_bwd(nseq, nhead, s, fmt, fmt, seed=71)
+    dp = np.float64(np.float32(b_p)) * (dC4 @ V.transpose(0, 1, 3, 2))          # unrounded, as in the kernel
+    ref = O.softmax_bwd(p_host, dp, sm, sm)
+    got = U.host_values(dS).reshape(ref.shape)
+    scale = np.abs(ref).max() + np.abs(dp).max()
+    lim = U.ulp_of(ref, fmt) + 3e-6 * scale * max(1.0, s / 512)
+    err = np.abs(got - ref)
+    assert (err <= lim).all(), f"dS: {(err > lim).sum()} elements out, worst {err.max():.3e}"
+    ref_q = (np.float64(np.float32(b_q)) * (got @ K)).transpose(0, 2, 1, 3).reshape(nseq * s, nhead * 64)   # from the device's own dS
+    gq = U.host_values(dQ)
+    lim_q = TOL * max(1.0, np.abs(ref_q).max()) + U.ulp_of(ref_q, fmt)
+    assert (np.abs(gq - ref_q) <= lim_q).all(), f"dQ: worst {np.abs(gq - ref_q).max():.3e}"
+    # and the whole chain against the oracle's single function, loosely (a one-ulp flip in dS moves dQ by ulp * |K|)
+    ds_o, dq_o = O.attention_bwd_scores(dC4, p_host, K, V, b_p, sm, sm, b_q, fmt)
+    assert np.abs(gq - dq_o.transpose(0, 2, 1, 3).reshape(gq.shape)).max() < 0.02 * max(1.0, np.abs(dq_o).max())
+
+
+@pytest.mark.parametrize("dq_fmt", ["f32", "e5m2"])
+def test_backward_query_gradient_formats(dq_fmt):
+    nseq, nhead, s = 2, 2, 192
+    dC4, p_host, K, V, dS, dQ, (b_p, sm, b_q) = _run_bwd(nseq, nhead, s, "bf16", dq_fmt, seed=72)
+    got = U.host_values(dS).reshape(nseq, nhead, s, s)
+    ref_q = (np.float64(np.float32(b_q)) * (got @ K)).transpose(0, 2, 1, 3).reshape(nseq * s, nhead * 64)
+    gq = U.host_values(dQ)
+    if dq_fmt == "f32":
+        assert np.abs(gq - ref_q).max() <= TOL * max(1.0, np.abs(ref_q).max())
+    else:
+        fm = F.FORMATS[dq_fmt]
+        dist = U.code_distance(F.quantise_codes(gq, fm), F.quantise_codes(ref_q, fm), dq_fmt)
+        assert ((dist <= 1) | (np.abs(gq - F.quantise(ref_q, fm)) <= TOL * max(1.0, np.abs(ref_q).max()))).all()
+
+
+def test_backward_bert_large_attention_shape_sampled_problems():
+    nseq, nhead, s = 16, 16, 512
+    dC4, p_host, K, V, dS, dQ, (b_p, sm, b_q) = _run_bwd(nseq, nhead, s, "bf16", "bf16", seed=73)
+    rng = np.random.default_rng(8)
+    probs = [(0, 0), (0, 15), (15, 0), (15, 15)] + [(int(rng.integers(16)), int(rng.integers(16))) for _ in range(4)]
+    gq = U.host_values(dQ)
+    for (i, j) in probs:
+        dp = np.float64(np.float32(b_p)) * (dC4[i, j] @ V[i, j].T)
+        ref = O.softmax_bwd(p_host[i, j], dp, sm, sm)
+        got = U.host_values(dS[(i * nhead + j) * s:(i * nhead + j + 1) * s])
+        lim = U.ulp_of(ref, "bf16") + 3e-6 * (np.abs(ref).max() + np.abs(dp).max())
+        assert (np.abs(got - ref) <= lim).all(), (i, j)
+        ref_q = np.float64(np.float32(b_q)) * (got @ K[i, j])
+        g = gq[i * s:(i + 1) * s, j * 64:(j + 1) * 64]
+        assert (np.abs(g - ref_q) <= TOL * max(1.0, np.abs(ref_q).max()) + U.ulp_of(ref_q, "bf16")).all(), (i, j)
