@@ -41,8 +41,9 @@ class UnitScaledEncoderLayer:
                  fused_attention: bool = False):
         assert d % nhead == 0 and norm in (None, "post")
         self.attention, self.norm, self.eps = attention, norm, eps
-        # fused_attention: scores, scaled softmax and context of the forward pass as one us_attention_fwd launch
-        # (16-bit attention operands, heads of 64, at most 512 tokens per sequence); the scores are then never stored
+        # fused_attention: scores, scaled softmax and context of the forward pass as one us_attention_fwd launch, and
+        # dP, the softmax gradient and dQ of the backward pass as one us_attention_bwd launch (16-bit attention operands,
+        # heads of 64, at most 512 tokens per sequence); the scores and the gradient dP are then never stored
         self.fused_attention = fused_attention
         if fused_attention and not (attention in ("bf16", "fp16") and d // nhead == 64 and slen <= 512):
             raise ValueError("fused attention needs 16-bit attention operands, heads of 64 and sequences of at most 512 tokens")
@@ -62,7 +63,7 @@ class UnitScaledEncoderLayer:
         self.ffn = F.UnitScaledFFN(T, d, d_ff, scales=F.FFNScales.unit(T, d, d_ff, tau), device=device)
         self.g1q = e(T, d, E5)
         self.dC = e(T, d, grad_dt)
-        self.dP = e(nseq * nhead * slen, slen, wide_dt)
+        self.dP = None if fused_attention else e(nseq * nhead * slen, slen, wide_dt)
         self.dS = e(nseq * nhead * slen, slen, grad_dt)
         self.dQKVq = e(T, 3 * d, E5)
         self.dQKV = self.dQKVq if attention == "fp8" else e(T, 3 * d, grad_dt)   # FP8: written as E5M2 directly
@@ -88,8 +89,9 @@ class UnitScaledEncoderLayer:
         self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
                        dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
         # fused cast, attention forward, FFN forward + backward, attention backward (one cast fewer with FP8 attention)
-        self.launches_per_step = 1 + (3 if fused_attention else 5) + 7 + (10 if attention == "fp8" else 11) + (7 if norm == "post" else 0)
+        self.launches_per_step = 1 + (3 if fused_attention else 5) + 7 + (10 if attention == "fp8" else 9 if fused_attention else 11) + (7 if norm == "post" else 0)
         self.bt_fused = L.attention_batch(n, qkv, qkv, qkv, td, sq)
+        self.bt_fused_bwd = L.attention_bwd_batch(n, td, sq, qkv, qkv, sq, qkv)
 
     def _heads(self, M, which):
         """Problem (0, 0) of a [T x 3d] matrix: rows of the first sequence, columns of head 0 of Q / K / V."""
@@ -150,10 +152,15 @@ class UnitScaledEncoderLayer:
         L.us_linear_bwd_x(self.g1q, self.Wo_q, sc["beta_o"], self.dC, ws, None, cur)
         dC_h = self.dC[:s, : self.hd]
         beside(lambda st: L.us_linear_bwd_w_batched(self.P[:s], dC_h, sc["beta_V"], self._heads(self.dQKV, 2), self.bt["dV"], ws, st))
-        L.us_linear_bwd_x_batched(dC_h, V, sc["beta_P"], self.dP[:s], self.bt["dP"], ws, cur)
-        L.us_softmax_bwd(self.P, self.dP, sc["sm"], sc["sm"], self.dS, cur)
-        beside(lambda st: L.us_linear_bwd_w_batched(self.dS[:s], Q, sc["beta_K"], self._heads(self.dQKV, 1), self.bt["dK"], ws, st))
-        L.us_linear_fwd_batched(self.dS[:s], K, sc["beta_Q"], self._heads(self.dQKV, 0), self.bt["dQ"], ws, cur)
+        if self.fused_attention:
+            L.us_attention_bwd(dC_h, self.P[:s], K, V, sc["beta_P"], sc["sm"], sc["sm"], sc["beta_Q"], self.dS[:s],
+                               self._heads(self.dQKV, 0), self.bt_fused_bwd, ws, cur)
+            beside(lambda st: L.us_linear_bwd_w_batched(self.dS[:s], Q, sc["beta_K"], self._heads(self.dQKV, 1), self.bt["dK"], ws, st))
+        else:
+            L.us_linear_bwd_x_batched(dC_h, V, sc["beta_P"], self.dP[:s], self.bt["dP"], ws, cur)
+            L.us_softmax_bwd(self.P, self.dP, sc["sm"], sc["sm"], self.dS, cur)
+            beside(lambda st: L.us_linear_bwd_w_batched(self.dS[:s], Q, sc["beta_K"], self._heads(self.dQKV, 1), self.bt["dK"], ws, st))
+            L.us_linear_fwd_batched(self.dS[:s], K, sc["beta_Q"], self._heads(self.dQKV, 0), self.bt["dQ"], ws, cur)
         if par:
             cur.wait_stream(side)                                   # dQ, dK, dV all written
         if self.dQKV is not self.dQKVq:

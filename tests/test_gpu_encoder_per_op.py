@@ -65,7 +65,8 @@ def _per_op(layer, host, problems, rows, wrows):
     assert np.array_equal(U.codes_of(layer.Wo_q), F.quantise_codes(Wo, F.E4M3))
     Xq, Wqkv_q, Wo_q = H(layer.Xq), H(layer.Wqkv_q), H(layer.Wo_q)
     QKV, Cq = H(layer.QKV), H(layer.Cq)
-    f_act, f_wide, f_grad = _fmt_of(layer.QKV), _fmt_of(layer.dP), _fmt_of(layer.dS)
+    f_act, f_grad = _fmt_of(layer.QKV), _fmt_of(layer.dS)
+    f_wide = _fmt_of(layer.dP) if layer.dP is not None else None
     fused = layer.S is None          # fused attention forward: the scores are never stored
     # ---- QKV projection
     _check(QKV[rows], O.linear_fwd(Xq[rows], Wqkv_q, sc["alpha_qkv"]), f_act, TOL, "QKV")
@@ -76,7 +77,7 @@ def _per_op(layer, host, problems, rows, wrows):
         q, k, v = (QKV[r, o + j * hd:o + (j + 1) * hd] for o in (0, d, 2 * d))
         c = slice(j * hd, (j + 1) * hd)
         tag = f"problem ({i}, {j})"
-        Pp, dPp, dSp = H(layer.P[pr]), H(layer.dP[pr]), H(layer.dS[pr])   # score-sized tensors: this problem only
+        Pp, dSp = H(layer.P[pr]), H(layer.dS[pr])   # score-sized tensors: this problem only
         # forward: scores, scaled softmax, context
         if fused:
             p_ref, _ = O.attention_fwd(q, k, v, sc["alpha_s"], sc["sm"], sc["alpha_c"], "f64")     # from unrounded scores
@@ -90,7 +91,11 @@ def _per_op(layer, host, problems, rows, wrows):
         # backward: dP = beta dC V^T, dV = beta P^T dC, dS, dQ = beta dS K, dK = beta dS^T Q
         dc = dC[r, c]
         ref = O.linear_bwd_x(dc, v, sc["beta_P"])
-        _check(dPp, ref, f_wide, TOL * max(1.0, np.abs(ref).max()), "dP " + tag)
+        if fused:
+            dPp = ref                                  # never stored: the softmax gradient sees it unrounded
+        else:
+            dPp = H(layer.dP[pr])
+            _check(dPp, ref, f_wide, TOL * max(1.0, np.abs(ref).max()), "dP " + tag)
         ref = O.linear_bwd_w(Pp, dc, sc["beta_V"])
         _check(dQKV[r, 2 * d + j * hd:2 * d + (j + 1) * hd], ref, f_grad, TOL * max(1.0, np.abs(ref).max()), "dV " + tag)
         ref = O.softmax_bwd(Pp, dPp, sc["sm"], sc["sm"])
