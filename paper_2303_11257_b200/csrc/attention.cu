@@ -378,7 +378,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
   constexpr uint32_t kData = kQBytes + kKBytes + kTileBytes;
   const uint32_t bars = base + kData;
   const uint32_t bar_in = bars, bar_pin = bars + 8, bar_dp = bars + 16, bar_k = bars + 24, bar_ds = bars + 32,
-                 bar_dq = bars + 40, bar_tmem_free = bars + 48, bar_ps_free = bars + 56;
+                 bar_dq = bars + 40, bar_tmem_free = bars + 48;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + kData + 64);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + kData + 68);
   volatile float* row_sum = reinterpret_cast<volatile float*>(gen + kData + 128);     // [2][128]
@@ -396,7 +396,6 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
   if (threadIdx.x == 0) {
     ptx::mbar_init(bar_in, 1); ptx::mbar_init(bar_pin, 1); ptx::mbar_init(bar_dp, 1); ptx::mbar_init(bar_k, 1);
     ptx::mbar_init(bar_ds, kSoftmaxWarps); ptx::mbar_init(bar_dq, 1); ptx::mbar_init(bar_tmem_free, kSoftmaxWarps);
-    ptx::mbar_init(bar_ps_free, 1);
     *abort_flag = 0;
     ptx::mbar_init_fence();
   }
@@ -417,16 +416,10 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
         ptx::tma_load_4d(kv_s, &tv, bar_in, 0, 0, b1, b0);
         if (two_halves) ptx::tma_load_4d(kv_s + 256u * 128u, &tv, bar_in, 0, 256, b1, b0);
       };
-      auto load_p = [&](int tile) {                            // the tile of stored weights, key block by key block
-        int q0, b1, b0;
-        coords(tile, q0, b1, b0);
-        ptx::mbar_expect_tx(bar_pin, (uint32_t)nkb * kKeyBlockBytes);
-        for (int kb = 0; kb < nkb; ++kb) ptx::tma_load_4d(ps_s + (uint32_t)kb * kKeyBlockBytes, &tp, bar_pin, kb * 64, q0, b1, b0);
-      };
       // phase of the latest load issued on each barrier (a wait on a phase that has completed returns at once)
-      bool in_issued = false, p_issued = false, k_issued = false;
-      uint32_t in_phase = 0, p_phase = 0, k_phase = 0;
-      if ((int)blockIdx.x < num_tiles) { load_in(blockIdx.x); load_p(blockIdx.x); in_issued = p_issued = true; }
+      bool in_issued = false, k_issued = false;
+      uint32_t in_phase = 0, k_phase = 0;
+      if ((int)blockIdx.x < num_tiles) { load_in(blockIdx.x); in_issued = true; }
       bool ok = true;
       int n = 0;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++n) {
@@ -471,34 +464,43 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
         ok = wait_bounded(bar_dq, ph, abort_flag, a.status, a.wait_limit);
         if (!ok) break;
         if (next < num_tiles) { load_in(next); in_phase = ph ^ 1u; }
-        // ... and the tile's store has read it too: the next tile of P may land
-        ok = wait_bounded(bar_ps_free, ph, abort_flag, a.status, a.wait_limit);
-        if (!ok) break;
-        if (next < num_tiles) { load_p(next); p_phase = ph ^ 1u; }
       }
       if (*abort_flag) {
         // loads that were issued land before the CTA gives up its shared memory
         if (in_issued) for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_in, in_phase); ++it) {}
-        if (p_issued) for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_pin, p_phase); ++it) {}
         if (k_issued) for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_k, k_phase); ++it) {}
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      // ---------------------------------------------------------------- dS leaves by TMA store
-      bool ok = true;
-      int n = 0;
-      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++n) {
+      // ---------------------------------------------------------------- the weight tile: P in by TMA load, dS out by TMA store
+      auto load_p = [&](int tile) {                            // key block by key block
         int q0, b1, b0;
         coords(tile, q0, b1, b0);
-        ok = wait_bounded(bar_ds, (uint32_t)n & 1u, abort_flag, a.status, a.wait_limit);
+        ptx::mbar_expect_tx(bar_pin, (uint32_t)nkb * kKeyBlockBytes);
+        for (int kb = 0; kb < nkb; ++kb) ptx::tma_load_4d(ps_s + (uint32_t)kb * kKeyBlockBytes, &tp, bar_pin, kb * 64, q0, b1, b0);
+      };
+      bool ok = true, p_issued = false;
+      uint32_t p_phase = 0;
+      if ((int)blockIdx.x < num_tiles) { load_p(blockIdx.x); p_issued = true; }
+      int n = 0;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++n) {
+        const uint32_t ph = (uint32_t)n & 1u;
+        const int next = tile + (int)gridDim.x;
+        int q0, b1, b0;
+        coords(tile, q0, b1, b0);
+        ok = wait_bounded(bar_ds, ph, abort_flag, a.status, a.wait_limit);
         if (!ok) break;
         for (int kb = 0; kb < nkb; ++kb) ptx::tma_store_4d(&tds, ps_s + (uint32_t)kb * kKeyBlockBytes, kb * 64, q0, b1, b0);
         ptx::bulk_commit_group();
-        ptx::bulk_wait_group_read<0>();
-        ptx::mbar_arrive(bar_ps_free);
+        ptx::bulk_wait_group_read<0>();                        // the store has read the tile ...
+        ok = wait_bounded(bar_dq, ph, abort_flag, a.status, a.wait_limit);     // ... and so have the dQ MMAs
+        if (!ok) break;
+        if (next < num_tiles) { load_p(next); p_phase = ph ^ 1u; }
       }
       ptx::bulk_wait_group_read<0>();
+      if (*abort_flag && p_issued)
+        for (uint32_t it = 0; it < a.wait_limit && !ptx::mbar_try_wait(bar_pin, p_phase); ++it) {}
     }
   } else {
     // ------------------------------------------------------------------ softmax gradient and dQ
