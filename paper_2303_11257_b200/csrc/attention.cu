@@ -593,27 +593,10 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
   if (warp == 1) { ptx::tc_fence_after_sync(); ptx::tmem_dealloc(tmem, 512); }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn attn_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(sym);
-  }
-  return fn;
-}
-
 // 4-d map (column, row, inner problem index, outer problem index) over 16-bit elements; box of 64 columns
 // (128 bytes, 128-byte swizzle) x box_rows rows of one problem.
 static bool attn_tmap(CUtensorMap* tm, const us_mat* m, const int64_t* stride, const int64_t* count, int box_rows) {
-  EncodeTiledFn fn = attn_encode_fn();
+  host::EncodeTiledFn fn = host::encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[4] = {(cuuint64_t)m->cols, (cuuint64_t)m->rows, (cuuint64_t)count[1], (cuuint64_t)count[0]};
   // a dimension of extent 1 still needs a valid (multiple of 16 bytes) stride

@@ -14,28 +14,11 @@
 namespace us {
 namespace {
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(sym);
-  }
-  return fn;
-}
-
 // Tensor map over a row-major matrix [rows x cols] of ES-byte elements with a box of `box_rows` rows
 // and `box_bytes` (128, or 64) bytes per row, swizzled with the pattern of that width.  Out-of-range parts of a box read as zero.
 static bool make_tmap(CUtensorMap* tm, const us_mat* m, int es, int box_rows, int box_bytes = 128,
                       const BatchDesc* bd = nullptr, const int64_t* bstride = nullptr) {
-  EncodeTiledFn fn = encode_fn();
+  host::EncodeTiledFn fn = host::encode_tiled_fn();
   if (!fn) return false;
   const CUtensorMapDataType type = es == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                                  : es == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT32;

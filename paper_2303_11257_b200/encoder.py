@@ -89,9 +89,14 @@ class UnitScaledEncoderLayer:
         self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
                        dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
         # fused cast, attention forward, FFN forward + backward, attention backward (one cast fewer with FP8 attention)
-        self.launches_per_step = 1 + (3 if fused_attention else 5) + 7 + (10 if attention == "fp8" else 9 if fused_attention else 11) + (7 if norm == "post" else 0)
+        self._launches = 1 + (3 if fused_attention else 5) + 7 + (10 if attention == "fp8" else 9 if fused_attention else 11) + (7 if norm == "post" else 0)
         self.bt_fused = L.attention_batch(n, qkv, qkv, qkv, td, sq)
         self.bt_fused_bwd = L.attention_bwd_batch(n, td, sq, qkv, qkv, sq, qkv)
+
+    @property
+    def launches_per_step(self) -> int:
+        """Kernel launches of one step (the FFN block takes three fewer while its grouped launch covers the shape)."""
+        return self._launches - (3 if self.norm is None and self.ffn.grouped else 0)
 
     def _heads(self, M, which):
         """Problem (0, 0) of a [T x 3d] matrix: rows of the first sequence, columns of head 0 of Q / K / V."""
@@ -122,7 +127,8 @@ class UnitScaledEncoderLayer:
         L.us_linear_fwd(self.Cq, self.Wo_q, sc["alpha_o"], self.U1 if post else self.R1, ws, ep, stream)
         if post:
             L.us_layer_norm_fwd(self.U1, ln[0], ln[1], self.eps, self.R1, stream)
-        f.forward(self.R1, stream)
+        if post or not f.grouped:
+            f.forward(self.R1, stream)
         # ---- backward
         if post:
             L.us_layer_norm_fwd(f.R, ln[2], ln[3], self.eps, self.R2, stream)
@@ -130,6 +136,11 @@ class UnitScaledEncoderLayer:
             f.backward(self.dU2, stream)                            # f.dX = dL/dR1
             L.us_layer_norm_bwd(self.U1, ln[0], f.dX, self.eps, 1.0, self.beta_ln, self.dU1, self.dln[0], self.dln[1], self.ln_ws, stream)
             g1 = self.dU1
+        elif f.grouped:
+            # G is known from the start, so the whole FFN block goes out as a cast of its input and three GEMM launches
+            f._cast(self.R1, f.Xq, stream)
+            f.step_from_casts(self.R1, G, stream)                   # f.R = layer output, f.dX = dL/dR1
+            g1 = f.dX
         else:
             f.backward(G, stream, cast_g=False)                     # f.dX = dL/dR1
             g1 = f.dX

@@ -201,21 +201,9 @@ class UnitScaledFFN:
         and join back into the current stream (this also records as parallel branches under graph capture)."""
         st = self.stages(X, W1, W2, G)
         if self.grouped and self.fused_casts:
-            by = {name: fn for name, _, fn in st}
-            for name in ("cast_all", "fwd1_gelu", "bwd_x2_gelu_grad"):
-                by[name](stream)
-            try:
-                L.us_linear_group(self.group_calls(X, G), self.ws, stream)
-                return self.dX, self.dW1, self.dW2
-            except L.UnitScaleError as e:
-                if e.status != L.US_ERR_UNSUPPORTED:
-                    raise
-                # a shape the grouped form does not cover (an output of at most 128 rows or columns): nothing was
-                # launched; the four GEMMs go out one by one, now and in later steps
-                self.grouped, self.launches_per_step = False, 7
-                for name in ("fwd2_residual", "bwd_w2", "bwd_x1_residual", "bwd_w1"):
-                    by[name](stream)
-                return self.dX, self.dW1, self.dW2
+            cast_all = next(fn for name, _, fn in st if name == "cast_all")
+            cast_all(stream)
+            return self.step_from_casts(X, G, stream)
         if not (self.concurrent and self.fused_casts and stream is None):
             for name, _, fn in st:
                 fn(stream)
@@ -237,6 +225,27 @@ class UnitScaledFFN:
         by["bwd_x1_residual"](s_c)
         cur.wait_stream(s_b)
         cur.wait_stream(s_c)
+        return self.dX, self.dW1, self.dW2
+
+    def step_from_casts(self, X, G, stream=None):
+        """The GEMMs of one pass when self.Xq, W1q, W2q, Gq already hold the quantised operands (FP8 mode): three
+        launches -- first GEMM + GELU, GELU-gradient GEMM, the other four as one group.  X and G are the unquantised
+        skip inputs of the two residual epilogues."""
+        by = {name: fn for name, _, fn in self.stages(X, None, None, G)}
+        by["fwd1_gelu"](stream)
+        by["bwd_x2_gelu_grad"](stream)
+        if self.grouped:
+            try:
+                L.us_linear_group(self.group_calls(X, G), self.ws, stream)
+                return self.dX, self.dW1, self.dW2
+            except L.UnitScaleError as e:
+                if e.status != L.US_ERR_UNSUPPORTED:
+                    raise
+                # a shape the grouped form does not cover (an output of at most 128 rows or columns): nothing was
+                # launched; the four GEMMs go out one by one, now and in later steps
+                self.grouped, self.launches_per_step = False, 7
+        for name in ("fwd2_residual", "bwd_w2", "bwd_x1_residual", "bwd_w1"):
+            by[name](stream)
         return self.dX, self.dW1, self.dW2
 
     def capture(self, X, W1, W2, G):
