@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(kThreads) ew_kernel(const EwArgs p) {
   const int64_t total = p.rows * p.chunks_per_row;
   for (int64_t c = blockIdx.x * (int64_t)kThreads + threadIdx.x; c < total;
        c += (int64_t)gridDim.x * kThreads) {
-    const int64_t row = c / p.chunks_per_row;
+    const int64_t row = p.rows == 1 ? 0 : c / p.chunks_per_row;      // tensors without row padding arrive as one long row
     const int64_t col = (c - row * p.chunks_per_row) * kVec;
     const int64_t i0 = row * p.in0.ld + col, i1 = row * p.in1.ld + col, io = row * p.out.ld + col;
     if (p.vec_ok && col + kVec <= p.cols) {
