@@ -74,6 +74,12 @@ __device__ __forceinline__ void attn_tile_coords(const AttnParams& a, int tile, 
   q0 = qt * 128; b1 = pr % a.nb1; b0 = pr / a.nb1;
 }
 
+// F8: operands (and the stored weights) are FP8 instead of 16-bit.  A head row is then 64 bytes: the TMA boxes stay 128
+// bytes wide and the bytes beyond the head read as zeros, so Q and K tiles keep the 128-byte-swizzled layout (their
+// MMAs stop after 64 bytes of K), a 128-byte row of weights holds 128 keys (one key block per quarter instead of
+// two), and V, an MN-major operand whose rows are 128 bytes with the upper half zero, multiplies into 128 TMEM columns
+// of which the first 64 are the context.
+template <bool F8>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_constant__ CUtensorMap tk,
                      const __grid_constant__ CUtensorMap tv, const __grid_constant__ CUtensorMap tp, const AttnParams a) {
@@ -93,8 +99,10 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = a.q_tiles * a.nb1 * a.nb0;
-  const int nkb = (a.s_k + 63) >> 6;                 // 64-key blocks with at least one key
-  const int nq = (nkb + 1) >> 1;                     // quarters (two key blocks, 128 keys) with at least one key
+  constexpr int kBlockKeys = F8 ? 128 : 64;          // keys in a 128-byte row of weights
+  constexpr int kQuarterBlocks = F8 ? 1 : 2;         // key blocks per quarter (128 keys)
+  const int nkb = (a.s_k + kBlockKeys - 1) / kBlockKeys;   // key blocks with at least one key
+  const int nq = (a.s_k + 127) >> 7;                 // quarters with at least one key
   const bool two_halves = a.s_k > 256;
   const uint32_t kv_bytes = (two_halves ? 2u : 1u) * 256u * 128u;
 
@@ -150,8 +158,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
         for (int h = 0; h < (two_halves ? 2 : 1); ++h) {
           const uint64_t kd = ptx::smem_desc_sw128(k_s + (uint32_t)h * 256u * 128u, 16, 1024);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)                          // 16 of the 64 head columns (32 bytes) per MMA
-            ptx::mma_ss<false>(tmem + 256u * h, qd + 2u * k, kd + 2u * k, a.idesc_s, k > 0);
+          for (int k = 0; k < (F8 ? 2 : 4); ++k)               // 32 bytes of the head columns per MMA
+            ptx::mma_ss<F8>(tmem + 256u * h, qd + 2u * k, kd + 2u * k, a.idesc_s, k > 0);
         }
         ptx::mma_commit(bar_s);
         // Q and K may be overwritten once those MMAs have read them: fetch the next tile's
@@ -168,14 +176,15 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
           if (!ok) break;
           if (b) ++fill1; else ++fill0;
           ptx::tc_fence_after_sync();
-          for (int kbl = 0; kbl < 2; ++kbl) {
-            const int kb = 2 * qd4 + kbl;
+          for (int kbl = 0; kbl < kQuarterBlocks; ++kbl) {
+            const int kb = kQuarterBlocks * qd4 + kbl;
             if (kb >= nkb) break;
+            constexpr uint32_t kVBlock = (uint32_t)kBlockKeys * 128u;      // V rows of one key block, 128 bytes each
             const uint64_t pd = ptx::smem_desc_sw128(pq_s + (uint32_t)b * kQuarterBytes + (uint32_t)kbl * kKeyBlockBytes, 16, 1024);
-            const uint64_t vd = ptx::smem_desc_sw128(v_s + (uint32_t)kb * 8192u, 8192, 1024);
+            const uint64_t vd = ptx::smem_desc_sw128(v_s + (uint32_t)kb * kVBlock, kVBlock, 1024);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)                        // 16 keys per MMA: 32 bytes along a P row, 16 rows of V
-              ptx::mma_ss<false>(tmem, pd + 2u * k, vd + 128u * k, a.idesc_c, (kb | k) != 0);
+            for (int k = 0; k < 4; ++k)                        // 32 bytes along a P row = a quarter of the block's V rows per MMA
+              ptx::mma_ss<F8>(tmem, pd + 2u * k, vd + (kVBlock / 64u) * k, a.idesc_c, (kb | k) != 0);
           }
           ptx::mma_commit(bar_free(b));                        // one of the two arrivals that free the buffer
         }
@@ -206,10 +215,10 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
           if (!ok) break;
           if (b) ++fill1; else ++fill0;
           if (a.store_p) {
-            for (int kbl = 0; kbl < 2; ++kbl) {
-              const int kb = 2 * qd4 + kbl;
+            for (int kbl = 0; kbl < kQuarterBlocks; ++kbl) {
+              const int kb = kQuarterBlocks * qd4 + kbl;
               if (kb < nkb)
-                ptx::tma_store_4d(&tp, pq_s + (uint32_t)b * kQuarterBytes + (uint32_t)kbl * kKeyBlockBytes, kb * 64, q0, b1, b0);
+                ptx::tma_store_4d(&tp, pq_s + (uint32_t)b * kQuarterBytes + (uint32_t)kbl * kKeyBlockBytes, kb * kBlockKeys, q0, b1, b0);
             }
             ptx::bulk_commit_group();
             ptx::bulk_wait_group_read<0>();                    // the store has read the buffer
@@ -226,7 +235,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
     // sum through shared memory.
     const int q = warp & 3, part = (warp - 2) >> 2, r = q * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(q * 32) << 16);
-    const int c_end = 2 * nkb;
+    const int c_end = 4 * nq;                                  // 32-column chunks, whole quarters
     // One sweep over this warp's chunks c = part, part + 2, ...
     auto sweep = [&](auto&& body) {
 #pragma unroll 1
@@ -295,17 +304,31 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tq, const __grid_consta
         for (int c = 4 * qd4 + part; c < 4 * qd4 + 4 && c < c_end; c += 2) {
           float v[32];
           ptx::tmem_ld_32x32(t_row + 32u * c, v);
-          const uint32_t blk = pq_s + (uint32_t)b * kQuarterBytes + (uint32_t)((c >> 1) & 1) * kKeyBlockBytes + row_off;
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint32_t w[4];
+          for (int i = 0; i < 32; ++i) v[i] *= inv;
+          if (F8) {
+            // one key block per quarter; this chunk's 32 weights are bytes 32 (c & 3) .. + 31 of the row
+            const uint32_t blk = pq_s + (uint32_t)b * kQuarterBytes + row_off;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float p0 = v[8 * g + 2 * j] * inv, p1 = v[8 * g + 2 * j + 1] * inv;
-              w[j] = a.op_bf16 ? pack_bf16x2(p0, p1) : pack_f16x2(p0, p1);
+            for (int g = 0; g < 2; ++g) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                w[j] = cvt_fp8x4<false>(v[16 * g + 4 * j], v[16 * g + 4 * j + 1], v[16 * g + 4 * j + 2], v[16 * g + 4 * j + 3]);
+              const uint32_t chunk16 = (uint32_t)((c & 3) * 2 + g);
+              ptx::sts128(blk + ((chunk16 ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
             }
-            const uint32_t chunk16 = (uint32_t)((c & 1) * 4 + g);
-            ptx::sts128(blk + ((chunk16 ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+          } else {
+            const uint32_t blk = pq_s + (uint32_t)b * kQuarterBytes + (uint32_t)((c >> 1) & 1) * kKeyBlockBytes + row_off;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                w[j] = a.op_bf16 ? pack_bf16x2(v[8 * g + 2 * j], v[8 * g + 2 * j + 1]) : pack_f16x2(v[8 * g + 2 * j], v[8 * g + 2 * j + 1]);
+              const uint32_t chunk16 = (uint32_t)((c & 1) * 4 + g);
+              ptx::sts128(blk + ((chunk16 ^ sw) << 4), make_uint4(w[0], w[1], w[2], w[3]));
+            }
           }
         }
         ptx::fence_proxy_async_smem();                         // the MMA and the TMA store read these bytes
@@ -593,18 +616,18 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
   if (warp == 1) { ptx::tc_fence_after_sync(); ptx::tmem_dealloc(tmem, 512); }
 }
 
-// 4-d map (column, row, inner problem index, outer problem index) over 16-bit elements; box of 64 columns
-// (128 bytes, 128-byte swizzle) x box_rows rows of one problem.
-static bool attn_tmap(CUtensorMap* tm, const us_mat* m, const int64_t* stride, const int64_t* count, int box_rows) {
+// 4-d map (column, row, inner problem index, outer problem index) over elements of es bytes (2, or 1 for FP8); box of 128
+// bytes (128-byte swizzle) x box_rows rows of one problem; columns of a box beyond the matrix read as zeros.
+static bool attn_tmap(CUtensorMap* tm, const us_mat* m, const int64_t* stride, const int64_t* count, int box_rows, int es = 2) {
   host::EncodeTiledFn fn = host::encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[4] = {(cuuint64_t)m->cols, (cuuint64_t)m->rows, (cuuint64_t)count[1], (cuuint64_t)count[0]};
   // a dimension of extent 1 still needs a valid (multiple of 16 bytes) stride
-  const cuuint64_t s1 = count[1] > 1 ? (cuuint64_t)stride[1] * 2 : 16, s0 = count[0] > 1 ? (cuuint64_t)stride[0] * 2 : 16;
-  cuuint64_t strides[3] = {(cuuint64_t)m->ld * 2, s1, s0};
-  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
+  const cuuint64_t s1 = count[1] > 1 ? (cuuint64_t)stride[1] * es : 16, s0 = count[0] > 1 ? (cuuint64_t)stride[0] * es : 16;
+  cuuint64_t strides[3] = {(cuuint64_t)m->ld * es, s1, s0};
+  cuuint32_t box[4] = {(cuuint32_t)(128 / es), (cuuint32_t)box_rows, 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, m->ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  return fn(tm, es == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_UINT16, 4, m->ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -642,22 +665,24 @@ extern "C" us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us
     for (int j = 0; j < 2; ++j)
       if (all[i] && cnt[j] > 1 && strides[i][j] <= 0) return US_ERR_INVALID_ARG;
   const bool h16 = (Q->dtype == US_BF16 || Q->dtype == US_F16) && K->dtype == Q->dtype && V->dtype == Q->dtype;
-  if (!h16 || (P && P->dtype != Q->dtype)) return US_ERR_UNSUPPORTED;
+  const bool f8 = Q->dtype == US_E4M3 && K->dtype == US_E4M3 && V->dtype == US_E4M3;       // activations: E4M3
+  if (!(h16 || f8) || (P && P->dtype != Q->dtype)) return US_ERR_UNSUPPORTED;
+  const int es = f8 ? 1 : 2;
   if (C->dtype < US_F32 || C->dtype > US_E5M2) return US_ERR_UNSUPPORTED;
   if (Q->cols != kAttnD || s_k > kAttnMaxKeys) return US_ERR_UNSUPPORTED;
   if (!ws || ws_bytes < us_workspace_bytes()) return US_ERR_WORKSPACE;
   if (s_q == 0 || s_k == 0) return s_k == 0 && s_q > 0 ? US_ERR_INVALID_ARG : US_OK;   // a softmax over no keys is undefined
   const int c_es = (int)dtype_size(C->dtype);
-  if (!ok16(Q, batch->q_stride, cnt, 2) || !ok16(K, batch->k_stride, cnt, 2) || !ok16(V, batch->v_stride, cnt, 2) ||
-      !ok16(C, batch->c_stride, cnt, c_es) || (P && !ok16(P, batch->p_stride, cnt, 2)))
+  if (!ok16(Q, batch->q_stride, cnt, es) || !ok16(K, batch->k_stride, cnt, es) || !ok16(V, batch->v_stride, cnt, es) ||
+      !ok16(C, batch->c_stride, cnt, c_es) || (P && !ok16(P, batch->p_stride, cnt, es)))
     return US_ERR_ALIGNMENT;
 
   CUtensorMap tq, tk, tv, tp;
-  if (!attn_tmap(&tq, Q, batch->q_stride, cnt, 128) || !attn_tmap(&tk, K, batch->k_stride, cnt, 256) ||
-      !attn_tmap(&tv, V, batch->v_stride, cnt, 256))
+  if (!attn_tmap(&tq, Q, batch->q_stride, cnt, 128, es) || !attn_tmap(&tk, K, batch->k_stride, cnt, 256, es) ||
+      !attn_tmap(&tv, V, batch->v_stride, cnt, 256, es))
     return US_ERR_CUDA;
   tp = tq;
-  if (P && !attn_tmap(&tp, P, batch->p_stride, cnt, 128)) return US_ERR_CUDA;
+  if (P && !attn_tmap(&tp, P, batch->p_stride, cnt, 128, es)) return US_ERR_CUDA;
 
   AttnParams a{};
   a.s_q = (int)s_q; a.s_k = (int)s_k;
@@ -668,13 +693,14 @@ extern "C" us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us
   a.c_stride0 = cnt[0] > 1 ? batch->c_stride[0] : 0; a.c_stride1 = cnt[1] > 1 ? batch->c_stride[1] : 0;
   a.op_bf16 = Q->dtype == US_BF16;
   a.store_p = P != nullptr;
-  const int fmt = a.op_bf16 ? 1 : 0;
+  const int fmt = f8 ? 0 : a.op_bf16 ? 1 : 0;           // kind::f8f6f4: 0 = E4M3; kind::f16: 0 = F16, 1 = BF16
   a.idesc_s = make_idesc(fmt, fmt, false, false, 128, 256);
-  a.idesc_c = make_idesc(fmt, fmt, false, true, 128, 64);
+  a.idesc_c = make_idesc(fmt, fmt, false, true, 128, f8 ? 128 : 64);   // FP8: V rows are 128 bytes, the upper half zero
   a.status = static_cast<unsigned int*>(ws);
   a.wait_limit = kWaitLimit;
 
-  if (cudaFuncSetAttribute(attention_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmem) != cudaSuccess)
+  auto kern = f8 ? attention_fwd_kernel<true> : attention_fwd_kernel<false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmem) != cudaSuccess)
     return US_ERR_CUDA;
   a.q_tiles = (int)((s_q + 127) / 128); a.nb1 = (int)cnt[1]; a.nb0 = (int)cnt[0];
   const int64_t tiles = (int64_t)a.q_tiles * cnt[1] * cnt[0];
@@ -682,7 +708,7 @@ extern "C" us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us
   const int sms = host::sm_count();
   if (sms <= 0) return US_ERR_CUDA;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);    // persistent: one CTA per SM walks the tiles
-  attention_fwd_kernel<<<grid, kAttnThreads, kAttnSmem, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, tp, a);
+  kern<<<grid, kAttnThreads, kAttnSmem, static_cast<cudaStream_t>(stream)>>>(tq, tk, tv, tp, a);
   return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }
 

@@ -135,14 +135,51 @@ def test_argument_checks():
     with pytest.raises(L.UnitScaleError) as e:
         L.us_attention_fwd(q, k_long, k_long, 0.125, 640.0, 0.1, c, None, bt, ws)
     assert e.value.status == L.US_ERR_UNSUPPORTED                    # more than 512 keys
-    q8 = U.empty(128, 64, "e4m3")
+    q8 = U.empty(128, 64, "e5m2")
     with pytest.raises(L.UnitScaleError) as e:
         L.us_attention_fwd(q8, q8, q8, 0.125, 128.0, 0.1, c, None, bt, ws)
-    assert e.value.status == L.US_ERR_UNSUPPORTED                    # FP8 operands
+    assert e.value.status == L.US_ERR_UNSUPPORTED                    # E5M2 (gradient format) operands in the forward pass
     with pytest.raises(L.UnitScaleError) as e:
         L.us_attention_fwd(q, k, U.empty(64, 64, "bf16"), 0.125, 128.0, 0.1, c, None, bt, ws)
     assert e.value.status == L.US_ERR_INVALID_ARG                    # V rows != K rows
     L.us_attention_fwd(q[:0], k, k, 0.125, 128.0, 0.1, c[:0], None, bt, ws)   # no queries: nothing to do
+
+
+@pytest.mark.parametrize("nseq,nhead,s", [(2, 3, 128), (1, 2, 208), (2, 2, 512), (1, 1, 80), (1, 2, 272), (3, 1, 16)])
+def test_fp8_operands_weights_and_context(nseq, nhead, s):
+    """Q, K, V and the stored weights as E4M3 (all matmul inputs quantised): P within one code of the oracle's
+    (weights up to s = 512 saturate at 448), the context against alpha_c * P V on the device's own stored P."""
+    qkv_v, Cx, P, (a_s, sm, a_c) = _run(nseq, nhead, s, "e4m3", "e4m3", seed=65)
+    Q, K, V = (_heads(qkv_v, nseq, s, nhead, i) for i in range(3))
+    p_ref, _ = O.attention_fwd(Q, K, V, a_s, sm, a_c, "f64")
+    fm = F.FORMATS["e4m3"]
+    p_dev = U.host_values(P).reshape(nseq, nhead, s, s)
+    dist = U.code_distance(U.codes_of(P).reshape(p_ref.shape), F.quantise_codes(p_ref, fm), "e4m3")
+    ok = (dist <= 1) | (np.abs(p_dev - F.quantise(p_ref, fm)) <= 3e-6 * sm)
+    assert ok.all(), f"P: code distance {dist.max()} at {(~ok).sum()} places"
+    assert (dist > 0).mean() < 2e-3
+    _check_c(Cx, np.float64(np.float32(a_c)) * (p_dev @ V), "e4m3", nseq, s, nhead)
+
+
+def test_fp8_operands_bert_large_attention_shape_sampled_problems():
+    nseq, nhead, s = 16, 16, 512
+    qkv_v, Cx, P, (a_s, sm, a_c) = _run(nseq, nhead, s, "e4m3", "e4m3", seed=66)
+    rng = np.random.default_rng(9)
+    probs = [(0, 0), (0, 15), (15, 0), (15, 15)] + [(int(rng.integers(16)), int(rng.integers(16))) for _ in range(4)]
+    Cv = U.host_values(Cx)
+    fm = F.FORMATS["e4m3"]
+    for (i, j) in probs:
+        r = slice(i * s, (i + 1) * s)
+        q, k, v = (qkv_v[r, o * 1024 + j * 64:o * 1024 + (j + 1) * 64] for o in range(3))
+        p_ref, _ = O.attention_fwd(q, k, v, a_s, sm, a_c, "f64")
+        Pt = P[(i * nhead + j) * s:(i * nhead + j + 1) * s]
+        p_dev = U.host_values(Pt)
+        dist = U.code_distance(U.codes_of(Pt), F.quantise_codes(p_ref, fm), "e4m3")
+        assert ((dist <= 1) | (np.abs(p_dev - F.quantise(p_ref, fm)) <= 3e-6 * sm)).all(), (i, j)
+        ref = np.float64(np.float32(a_c)) * (p_dev @ v)
+        got = Cv[r, j * 64:(j + 1) * 64]
+        dc = U.code_distance(F.quantise_codes(got, fm), F.quantise_codes(ref, fm), "e4m3")
+        assert ((dc <= 1) | (np.abs(got - F.quantise(ref, fm)) <= TOL * max(1.0, np.abs(ref).max()))).all(), (i, j)
 
 
 # ------------------------------------------------------------------------------------------------ backward
