@@ -390,6 +390,9 @@ struct AttnBwdParams {
 constexpr uint32_t kTileBytes = 8 * kKeyBlockBytes;      // a 128 x 512 tile of 16-bit weights: 128 KB
 constexpr uint32_t kAttnBwdSmem = kQBytes + kKBytes + kTileBytes + 1024 + 128 + 1024;
 
+// F8: dC and dS are E5M2 (gradients), P, K and V E4M3 (activations); layouts as in the forward kernel's FP8 form
+// (a 128-byte row of P / dS holds 128 keys; dC, V and K rows are 64 bytes in 128-byte boxes whose upper half is zero).
+template <bool F8>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_constant__ CUtensorMap tv,
                      const __grid_constant__ CUtensorMap tk, const __grid_constant__ CUtensorMap tp,
@@ -408,7 +411,8 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = a.q_tiles * a.nb1 * a.nb0;
-  const int nkb = (a.s_k + 63) >> 6;
+  constexpr int kBlockKeys = F8 ? 128 : 64;          // keys in a 128-byte row of P / dS
+  const int nkb = (a.s_k + kBlockKeys - 1) / kBlockKeys;
   const bool two_halves = a.s_k > 256;
   const uint32_t kv_bytes = (two_halves ? 2u : 1u) * 256u * 128u;
   auto coords = [&](int tile, int& q0, int& b1, int& b0) {
@@ -461,7 +465,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
         for (int h = 0; h < (two_halves ? 2 : 1); ++h) {
           const uint64_t vd = ptx::smem_desc_sw128(kv_s + (uint32_t)h * 256u * 128u, 16, 1024);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) ptx::mma_ss<false>(tmem + 256u * h, cd + 2u * k, vd + 2u * k, a.idesc_s, k > 0);
+          for (int k = 0; k < (F8 ? 2 : 4); ++k) ptx::mma_ss<F8>(tmem + 256u * h, cd + 2u * k, vd + 2u * k, a.idesc_s, k > 0);
         }
         ptx::mma_commit(bar_dp);
         // V has been read: K takes its place
@@ -477,10 +481,11 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
         if (!ok) break;
         ptx::tc_fence_after_sync();
         for (int kb = 0; kb < nkb; ++kb) {
+          constexpr uint32_t kKBlock = (uint32_t)kBlockKeys * 128u;        // K rows of one key block, 128 bytes each
           const uint64_t sd = ptx::smem_desc_sw128(ps_s + (uint32_t)kb * kKeyBlockBytes, 16, 1024);
-          const uint64_t kd = ptx::smem_desc_sw128(kv_s + (uint32_t)kb * 8192u, 8192, 1024);
+          const uint64_t kd = ptx::smem_desc_sw128(kv_s + (uint32_t)kb * kKBlock, kKBlock, 1024);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) ptx::mma_ss<false>(tmem, sd + 2u * k, kd + 128u * k, a.idesc_c, (kb | k) != 0);
+          for (int k = 0; k < 4; ++k) ptx::mma_ss<F8>(tmem, sd + 2u * k, kd + (kKBlock / 64u) * k, a.idesc_c, (kb | k) != 0);
         }
         ptx::mma_commit(bar_dq);
         // dC, K and (for the MMAs) the dS tile have been read once those MMAs are done
@@ -501,7 +506,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
         int q0, b1, b0;
         coords(tile, q0, b1, b0);
         ptx::mbar_expect_tx(bar_pin, (uint32_t)nkb * kKeyBlockBytes);
-        for (int kb = 0; kb < nkb; ++kb) ptx::tma_load_4d(ps_s + (uint32_t)kb * kKeyBlockBytes, &tp, bar_pin, kb * 64, q0, b1, b0);
+        for (int kb = 0; kb < nkb; ++kb) ptx::tma_load_4d(ps_s + (uint32_t)kb * kKeyBlockBytes, &tp, bar_pin, kb * kBlockKeys, q0, b1, b0);
       };
       bool ok = true, p_issued = false;
       uint32_t p_phase = 0;
@@ -514,7 +519,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
         coords(tile, q0, b1, b0);
         ok = wait_bounded(bar_ds, ph, abort_flag, a.status, a.wait_limit);
         if (!ok) break;
-        for (int kb = 0; kb < nkb; ++kb) ptx::tma_store_4d(&tds, ps_s + (uint32_t)kb * kKeyBlockBytes, kb * 64, q0, b1, b0);
+        for (int kb = 0; kb < nkb; ++kb) ptx::tma_store_4d(&tds, ps_s + (uint32_t)kb * kKeyBlockBytes, kb * kBlockKeys, q0, b1, b0);
         ptx::bulk_commit_group();
         ptx::bulk_wait_group_read<0>();                        // the store has read the tile ...
         ok = wait_bounded(bar_dq, ph, abort_flag, a.status, a.wait_limit);     // ... and so have the dQ MMAs
@@ -529,11 +534,29 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
     // ------------------------------------------------------------------ softmax gradient and dQ
     const int q = warp & 3, part = (warp - 2) >> 2, r = q * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(q * 32) << 16);
-    const int c_end = 2 * nkb;
+    const int c_end = (kBlockKeys / 32) * nkb;                 // 32-column chunks, whole key blocks
     const uint32_t row_off = (uint32_t)r * 128u, sw = (uint32_t)(r & 7);
-    auto p_addr = [&](int c, int g) {                          // 16 bytes = columns 32 c + 8 g .. + 7 of this row
-      return ps_s + (uint32_t)(c >> 1) * kKeyBlockBytes + row_off + ((((uint32_t)((c & 1) * 4 + g)) ^ sw) << 4);
+    constexpr int kPieces = F8 ? 2 : 4;                        // 16-byte pieces of a chunk: 16 FP8 or 8 16-bit values each
+    auto p_addr = [&](int c, int g) {                          // piece g of chunk c of this row
+      const int per_block = kBlockKeys / 32;                   // chunks in a key block
+      return ps_s + (uint32_t)(c / per_block) * kKeyBlockBytes + row_off +
+             ((((uint32_t)((c % per_block) * kPieces + g)) ^ sw) << 4);
     };
+    // the values of one piece as floats (8, or 16 for FP8)
+    auto piece_values = [&](const uint4& raw, float (&pv)[16]) {
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (F8) {
+          const float2 lo = unpack_fp8x2((uint16_t)(w[j] & 0xffffu), false), hi = unpack_fp8x2((uint16_t)(w[j] >> 16), false);
+          pv[4 * j] = lo.x; pv[4 * j + 1] = lo.y; pv[4 * j + 2] = hi.x; pv[4 * j + 3] = hi.y;
+        } else {
+          const float2 f = a.op_bf16 ? unpack_bf16x2(w[j]) : unpack_f16x2(w[j]);
+          pv[2 * j] = f.x; pv[2 * j + 1] = f.y;
+        }
+      }
+    };
+    constexpr int kPieceVals = F8 ? 16 : 8;
     bool aborted = false;
     int n = 0;
 #pragma unroll 1
@@ -552,15 +575,11 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
         float x[32];
         ptx::tmem_ld_32x32(t_row + 32u * c, x);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const uint4 raw = ptx::lds128(p_addr(c, g));
-          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        for (int g = 0; g < kPieces; ++g) {
+          float pv[16];
+          piece_values(ptx::lds128(p_addr(c, g)), pv);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float2 pv = a.op_bf16 ? unpack_bf16x2(w[j]) : unpack_f16x2(w[j]);
-            s4[j] = fmaf(pv.x, x[8 * g + 2 * j], s4[j]);
-            s4[j] = fmaf(pv.y, x[8 * g + 2 * j + 1], s4[j]);
-          }
+          for (int i = 0; i < kPieceVals; ++i) s4[i & 3] = fmaf(pv[i], x[kPieceVals * g + i], s4[i & 3]);
         }
       }
       row_sum[part * 128 + r] = (s4[0] + s4[1]) + (s4[2] + s4[3]);
@@ -572,16 +591,17 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap tdc, const __grid_const
         float x[32];
         ptx::tmem_ld_32x32(t_row + 32u * c, x);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
+        for (int g = 0; g < kPieces; ++g) {
           const uint32_t addr = p_addr(c, g);
-          const uint4 raw = ptx::lds128(addr);
-          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+          float pv[16], d[16];
+          piece_values(ptx::lds128(addr), pv);
+#pragma unroll
+          for (int i = 0; i < kPieceVals; ++i) d[i] = a.ds_scale * pv[i] * (x[kPieceVals * g + i] - mean);
           uint32_t o[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const float2 pv = a.op_bf16 ? unpack_bf16x2(w[j]) : unpack_f16x2(w[j]);
-            const float d0 = a.ds_scale * pv.x * (x[8 * g + 2 * j] - mean), d1 = a.ds_scale * pv.y * (x[8 * g + 2 * j + 1] - mean);
-            o[j] = a.op_bf16 ? pack_bf16x2(d0, d1) : pack_f16x2(d0, d1);
+            if (F8) o[j] = cvt_fp8x4<true>(d[4 * j], d[4 * j + 1], d[4 * j + 2], d[4 * j + 3]);     // gradients: E5M2
+            else o[j] = a.op_bf16 ? pack_bf16x2(d[2 * j], d[2 * j + 1]) : pack_f16x2(d[2 * j], d[2 * j + 1]);
           }
           ptx::sts128(addr, make_uint4(o[0], o[1], o[2], o[3]));
         }
@@ -737,20 +757,23 @@ extern "C" us_status us_attention_bwd(const us_mat* dC, const us_mat* P, const u
   if (!(softmax_alpha > 0.f)) return US_ERR_INVALID_ARG;
   const bool h16 = (dC->dtype == US_BF16 || dC->dtype == US_F16) && K->dtype == dC->dtype && V->dtype == dC->dtype &&
                    P->dtype == dC->dtype && dS->dtype == dC->dtype;
-  if (!h16) return US_ERR_UNSUPPORTED;
+  const bool f8 = dC->dtype == US_E5M2 && dS->dtype == US_E5M2 && P->dtype == US_E4M3 && K->dtype == US_E4M3 &&
+                  V->dtype == US_E4M3;                 // gradients E5M2, activations E4M3
+  if (!(h16 || f8)) return US_ERR_UNSUPPORTED;
+  const int es = f8 ? 1 : 2;
   if (dQ->dtype < US_F32 || dQ->dtype > US_E5M2) return US_ERR_UNSUPPORTED;
   if (dC->cols != kAttnD || s_k > kAttnMaxKeys) return US_ERR_UNSUPPORTED;
   if (!ws || ws_bytes < us_workspace_bytes()) return US_ERR_WORKSPACE;
   if (s_q == 0 || s_k == 0) return US_OK;              // no queries: nothing to do; no keys: dS is empty and dQ is not written
   const int q_es = (int)dtype_size(dQ->dtype);
   for (int i = 0; i < 5; ++i)
-    if (!ok16(all[i], strides[i], cnt, 2)) return US_ERR_ALIGNMENT;
+    if (!ok16(all[i], strides[i], cnt, es)) return US_ERR_ALIGNMENT;
   if (!ok16(dQ, batch->dq_stride, cnt, q_es)) return US_ERR_ALIGNMENT;
 
   CUtensorMap tdc, tv, tk, tp, tds;
-  if (!attn_tmap(&tdc, dC, batch->dc_stride, cnt, 128) || !attn_tmap(&tv, V, batch->v_stride, cnt, 256) ||
-      !attn_tmap(&tk, K, batch->k_stride, cnt, 256) || !attn_tmap(&tp, P, batch->p_stride, cnt, 128) ||
-      !attn_tmap(&tds, dS, batch->ds_stride, cnt, 128))
+  if (!attn_tmap(&tdc, dC, batch->dc_stride, cnt, 128, es) || !attn_tmap(&tv, V, batch->v_stride, cnt, 256, es) ||
+      !attn_tmap(&tk, K, batch->k_stride, cnt, 256, es) || !attn_tmap(&tp, P, batch->p_stride, cnt, 128, es) ||
+      !attn_tmap(&tds, dS, batch->ds_stride, cnt, 128, es))
     return US_ERR_CUDA;
 
   AttnBwdParams a{};
@@ -763,17 +786,19 @@ extern "C" us_status us_attention_bwd(const us_mat* dC, const us_mat* P, const u
   a.dq_stride0 = cnt[0] > 1 ? batch->dq_stride[0] : 0; a.dq_stride1 = cnt[1] > 1 ? batch->dq_stride[1] : 0;
   a.op_bf16 = dC->dtype == US_BF16;
   const int fmt = a.op_bf16 ? 1 : 0;
-  a.idesc_s = make_idesc(fmt, fmt, false, false, 128, 256);
-  a.idesc_c = make_idesc(fmt, fmt, false, true, 128, 64);
+  // FP8 (kind::f8f6f4: 0 = E4M3, 1 = E5M2): the A operands dC and dS are gradients, the B operands V and K activations
+  a.idesc_s = f8 ? make_idesc(1, 0, false, false, 128, 256) : make_idesc(fmt, fmt, false, false, 128, 256);
+  a.idesc_c = f8 ? make_idesc(1, 0, false, true, 128, 128) : make_idesc(fmt, fmt, false, true, 128, 64);
   a.status = static_cast<unsigned int*>(ws);
   a.wait_limit = kWaitLimit;
   const int64_t tiles = (int64_t)a.q_tiles * cnt[1] * cnt[0];
   if (tiles > 0x7fffffff) return US_ERR_INVALID_ARG;
   const int sms = host::sm_count();
   if (sms <= 0) return US_ERR_CUDA;
-  if (cudaFuncSetAttribute(attention_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnBwdSmem) != cudaSuccess)
+  auto kern = f8 ? attention_bwd_kernel<true> : attention_bwd_kernel<false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnBwdSmem) != cudaSuccess)
     return US_ERR_CUDA;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-  attention_bwd_kernel<<<grid, kAttnThreads, kAttnBwdSmem, static_cast<cudaStream_t>(stream)>>>(tdc, tv, tk, tp, tds, a);
+  kern<<<grid, kAttnThreads, kAttnBwdSmem, static_cast<cudaStream_t>(stream)>>>(tdc, tv, tk, tp, tds, a);
   return cudaGetLastError() == cudaSuccess ? US_OK : US_ERR_CUDA;
 }

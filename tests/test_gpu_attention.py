@@ -184,20 +184,21 @@ def test_fp8_operands_bert_large_attention_shape_sampled_problems():
 
 # ------------------------------------------------------------------------------------------------ backward
 
-def _run_bwd(nseq, nhead, s, fmt, dq_fmt, seed, scale=1.0):
+def _run_bwd(nseq, nhead, s, fmt, dq_fmt, seed, scale=1.0, gfmt=None):
     """Weights P as the oracle's forward pass rounds them (uploaded bit patterns), random dC; returns host values of the
-    operands and the device outputs."""
+    operands and the device outputs.  gfmt: format of the gradients dC and dS when it differs from fmt (FP8: E5M2)."""
     from paper_2303_11257_b200 import lib as L, synth
+    gfmt = gfmt or fmt
     hd, d, T = 64, nhead * 64, nseq * s
     qkv = scale * synth.normal(seed, 0, (T, 3 * d))
     dc = synth.normal(seed, 1, (T, d))
-    QKV, dCt = U.to_device(qkv, fmt), U.to_device(dc, fmt)
-    qkv_v, dc_v = U.values_of(qkv, fmt), U.values_of(dc, fmt)
+    QKV, dCt = U.to_device(qkv, fmt), U.to_device(dc, gfmt)
+    qkv_v, dc_v = U.values_of(qkv, fmt), U.values_of(dc, gfmt)
     Q, K, V = (_heads(qkv_v, nseq, s, nhead, i) for i in range(3))
     a_s, sm, a_c = hd ** -0.5, float(s), s ** -0.5
     p_host, _ = O.attention_fwd(Q, K, V, a_s, sm, a_c, fmt)                    # as stored by a forward pass
     P = U.to_device(p_host.reshape(-1, s), fmt)
-    dS = U.empty(nseq * nhead * s, s, fmt)
+    dS = U.empty(nseq * nhead * s, s, gfmt)
     dQ = U.empty(T, d, dq_fmt)
     ws = L.new_workspace()
     b_p, b_q = hd ** -0.5, hd ** -0.5
@@ -259,3 +260,23 @@ def test_backward_bert_large_attention_shape_sampled_problems():
         ref_q = np.float64(np.float32(b_q)) * (got @ K[i, j])
         g = gq[i * s:(i + 1) * s, j * 64:(j + 1) * 64]
         assert (np.abs(g - ref_q) <= TOL * max(1.0, np.abs(ref_q).max()) + U.ulp_of(ref_q, "bf16")).all(), (i, j)
+
+
+@pytest.mark.parametrize("nseq,nhead,s", [(2, 3, 128), (1, 2, 208), (2, 2, 512), (1, 1, 80), (3, 1, 16)])
+def test_backward_fp8_operands(nseq, nhead, s):
+    """dC and dS as E5M2, P, K, V as E4M3: dS within one code of the oracle's softmax gradient on the unrounded dP,
+    dQ against beta * dS K on the device's own stored dS."""
+    dC4, p_host, K, V, dS, dQ, (b_p, sm, b_q) = _run_bwd(nseq, nhead, s, "e4m3", "e5m2", seed=74, gfmt="e5m2")
+    dp = np.float64(np.float32(b_p)) * (dC4 @ V.transpose(0, 1, 3, 2))
+    ref = O.softmax_bwd(p_host, dp, sm, sm)
+    fm = F.FORMATS["e5m2"]
+    got = U.host_values(dS).reshape(ref.shape)
+    dist = U.code_distance(U.codes_of(dS).reshape(ref.shape), F.quantise_codes(ref, fm), "e5m2")
+    scale = np.abs(ref).max() + np.abs(dp).max()
+    ok = (dist <= 1) | (np.abs(got - F.quantise(ref, fm)) <= 3e-6 * scale)
+    assert ok.all(), f"dS: code distance {dist.max()} at {(~ok).sum()} places"
+    assert (dist > 0).mean() < 2e-3
+    ref_q = (np.float64(np.float32(b_q)) * (got @ K)).transpose(0, 2, 1, 3).reshape(nseq * s, nhead * 64)
+    gq = U.host_values(dQ)
+    dq = U.code_distance(F.quantise_codes(gq, fm), F.quantise_codes(ref_q, fm), "e5m2")
+    assert ((dq <= 1) | (np.abs(gq - F.quantise(ref_q, fm)) <= TOL * max(1.0, np.abs(ref_q).max()))).all()
