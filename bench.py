@@ -655,7 +655,7 @@ def run_encoder(args, rank, world, local, torch, dev, peaks):
     sampler.start()
     results = {}
     windows = []
-    for name, attention, fused in (("bf16", "bf16", False), ("fp8", "fp8", False), ("bf16, fused attention kernels", "bf16", True)):
+    for name, attention, fused in (("bf16", "bf16", False), ("fp8", "fp8", False), ("bf16, fused attention kernels", "bf16", True), ("fp8, fused attention kernels", "fp8", True)):
         host = (synth.normal(0, 0, (T, d)), synth.normal(0, 1, (d, 3 * d)), synth.normal(0, 2, (d, d)),
                 synth.normal(0, 3, (d, d_ff)), synth.normal(0, 4, (d_ff, d)), synth.normal(0, 5, (T, d)))
         tensors = [torch.from_numpy(t).to(dev) for t in host]

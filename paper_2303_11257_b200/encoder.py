@@ -42,11 +42,11 @@ class UnitScaledEncoderLayer:
         assert d % nhead == 0 and norm in (None, "post")
         self.attention, self.norm, self.eps = attention, norm, eps
         # fused_attention: scores, scaled softmax and context of the forward pass as one us_attention_fwd launch, and
-        # dP, the softmax gradient and dQ of the backward pass as one us_attention_bwd launch (16-bit attention operands,
-        # heads of 64, at most 512 tokens per sequence); the scores and the gradient dP are then never stored
+        # dP, the softmax gradient and dQ of the backward pass as one us_attention_bwd launch (heads of 64, at most 512
+        # tokens per sequence; 16-bit or FP8 attention operands); the scores and the gradient dP are then never stored
         self.fused_attention = fused_attention
-        if fused_attention and not (attention in ("bf16", "fp16") and d // nhead == 64 and slen <= 512):
-            raise ValueError("fused attention needs 16-bit attention operands, heads of 64 and sequences of at most 512 tokens")
+        if fused_attention and not (d // nhead == 64 and slen <= 512):
+            raise ValueError("fused attention needs heads of 64 and sequences of at most 512 tokens")
         if attention == "fp8":
             act_dt, grad_dt, wide_dt = E4, E5, torch.bfloat16
         else:
@@ -89,7 +89,7 @@ class UnitScaledEncoderLayer:
         self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
                        dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
         # fused cast, attention forward, FFN forward + backward, attention backward (one cast fewer with FP8 attention)
-        self._launches = 1 + (3 if fused_attention else 5) + 7 + (10 if attention == "fp8" else 9 if fused_attention else 11) + (7 if norm == "post" else 0)
+        self._launches = 1 + (3 if fused_attention else 5) + 7 + ((10 if attention == "fp8" else 11) - (2 if fused_attention else 0)) + (7 if norm == "post" else 0)
         self.bt_fused = L.attention_batch(n, qkv, qkv, qkv, td, sq)
         self.bt_fused_bwd = L.attention_bwd_batch(n, td, sq, qkv, qkv, sq, qkv)
 

@@ -153,7 +153,7 @@ def test_encoder_layer_every_op_small(cfg, attention):
     _per_op(layer, host, problems, np.arange(nseq * slen), np.arange(max(d, f)))
 
 
-@pytest.mark.parametrize("attention", ["bf16", "fp16"])
+@pytest.mark.parametrize("attention", ["bf16", "fp16", "fp8"])
 @pytest.mark.parametrize("cfg", [(2, 128, 256, 4, 512), (3, 80, 192, 3, 400)])
 def test_encoder_layer_every_op_small_fused_attention(cfg, attention):
     nseq, slen, d, nhead, f = cfg
@@ -162,7 +162,7 @@ def test_encoder_layer_every_op_small_fused_attention(cfg, attention):
     _per_op(layer, host, problems, np.arange(nseq * slen), np.arange(max(d, f)))
 
 
-@pytest.mark.parametrize("attention,fused", [("bf16", False), ("fp8", False), ("bf16", True)])
+@pytest.mark.parametrize("attention,fused", [("bf16", False), ("fp8", False), ("bf16", True), ("fp8", True)])
 def test_encoder_layer_every_op_bert_large_shape(attention, fused):
     """Config 5 at its stated size (16 sequences x 512 tokens, d = 1024, 16 heads x 64, d_ff = 4096)."""
     nseq, slen, d, nhead, f = 16, 512, 1024, 16, 4096
