@@ -301,7 +301,7 @@ us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, co
  * count[1] independent (sequence, head) problems in one launch:
  *
  *   S = alpha_scores * Q K^T                       Q [s_q x 64], K [s_k x 64]; S is never stored and never rounded
- *   P = softmax_scale * softmax(S), row by row     rounded to the operands' 16-bit format (it is a matmul input)
+ *   P = softmax_scale * softmax(S), row by row     rounded to the operands' format (it is a matmul input)
  *   C = alpha_context * P V                        V [s_k x 64]; C [s_q x 64] rounded to C's dtype
  *
  * with alpha_scores = 1 / sqrt(64), softmax_scale = s_k and alpha_context = s_k^-1/2 for the
@@ -309,7 +309,8 @@ us_status us_cast_fp8_multi(int count, const us_mat* src, const float* scale, co
  * problem (i, j) of a tensor starts stride[0] * i + stride[1] * j elements further (heads are 64-column
  * slices of a [tokens x 3 d] QKV matrix, C a 64-column slice of a [tokens x d] matrix).  P may be NULL;
  * otherwise the rounded weights are also written to P [s_q x s_k] (the backward pass needs them).
- * Q, K, V (and P): all BF16 or all F16, device memory; C: any us_dtype.  Head width must be 64 and
+ * Q, K, V (and P): all BF16, all F16 or all E4M3 (FP8 activations; weights above 448 saturate), device memory;
+ * C: any us_dtype.  Head width must be 64 and
  * s_k at most 512, else US_ERR_UNSUPPORTED; s_k = 0 with s_q > 0 is US_ERR_INVALID_ARG, s_q = 0 is
  * a no-op.  Base addresses, row pitches and the strides of dimensions with count > 1 must be multiples
  * of 16 bytes (US_ERR_ALIGNMENT); those strides must be positive and counts lie in 1..65535
@@ -333,12 +334,12 @@ us_status us_attention_fwd(const us_mat* Q, const us_mat* K, const us_mat* V, fl
  * us_attention_bwd: the backward pass of us_attention_fwd down to the queries, in one launch:
  *
  *   dP = beta_p * dC V^T                                           score-sized, never stored and never rounded
- *   dS = softmax_beta * p (dP - sum_k p_k dP_k),  p = P / softmax_alpha    rounded to the operands' 16-bit format
+ *   dS = softmax_beta * p (dP - sum_k p_k dP_k),  p = P / softmax_alpha    rounded to the gradients' format
  *   dQ = beta_q * dS K
  *
  * dC [s_q x 64] is the gradient of the context, P [s_q x s_k] the weights the forward call stored, K and V [s_k x 64].
  * dS [s_q x s_k] is written for the caller's dK = beta dS^T Q matmul (dV = beta P^T dC needs only P and dC); dQ
- * [s_q x 64] in any us_dtype.  dC, P, K, V and dS: all BF16 or all F16.  Shapes, limits, batch description (one stride
+ * [s_q x 64] in any us_dtype.  dC, P, K, V and dS: all BF16 or all F16; or FP8: dC and dS E5M2 (gradients), P, K, V E4M3.  Shapes, limits, batch description (one stride
  * pair per tensor), alignment, workspace and errors as for us_attention_fwd; softmax_alpha must be positive.
  */
 typedef struct {
