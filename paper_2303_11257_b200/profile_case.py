@@ -2,7 +2,7 @@
 
     python -m paper_2303_11257_b200.profile_case [--tokens 8192] [--passes 2] [--operand fp8]
     python -m paper_2303_11257_b200.profile_case --case attention [--passes 2]
-    python -m paper_2303_11257_b200.profile_case --case encoder [--passes 2] [--unfused]
+    python -m paper_2303_11257_b200.profile_case --case encoder [--passes 2] [--unfused] [--attention bf16|fp16|fp8]
 
 Each pass is the launches of UnitScaledFFN.step (one fused cast, six GEMMs) at d_model = 1024, d_ff = 4096.  At the default
 size the process holds well under 2 GB on the device and a pass lasts a fraction of a millisecond.
@@ -43,17 +43,17 @@ def attention(passes: int):
     print("ok attention", passes)
 
 
-def encoder_layer(passes: int, fused: bool):
+def encoder_layer(passes: int, fused: bool, attention: str = "bf16"):
     nseq, slen, d, nhead, d_ff = 16, 512, 1024, 16, 4096
     T = nseq * slen
     host = (synth.normal(0, 0, (T, d)), synth.normal(0, 1, (d, 3 * d)), synth.normal(0, 2, (d, d)),
             synth.normal(0, 3, (d, d_ff)), synth.normal(0, 4, (d_ff, d)), synth.normal(0, 5, (T, d)))
     tensors = [torch.from_numpy(t).cuda() for t in host]
-    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, d_ff, attention="bf16", fused_attention=fused)
+    layer = encoder.UnitScaledEncoderLayer(nseq, slen, d, nhead, d_ff, attention=attention, fused_attention=fused)
     for _ in range(passes):
         layer.step(*tensors, stream=torch.cuda.current_stream().cuda_stream)     # one stream: launches in issue order
     layer.check()
-    print("ok encoder", passes, "fused" if fused else "unfused")
+    print("ok encoder", passes, attention, "fused" if fused else "unfused")
 
 
 def main():
@@ -63,11 +63,12 @@ def main():
     ap.add_argument("--operand", default="fp8")
     ap.add_argument("--case", default="ffn", choices=["ffn", "attention", "encoder"])
     ap.add_argument("--unfused", action="store_true")
+    ap.add_argument("--attention", default="bf16", choices=["bf16", "fp16", "fp8"])
     a = ap.parse_args()
     if a.case == "attention":
         return attention(a.passes)
     if a.case == "encoder":
-        return encoder_layer(a.passes, not a.unfused)
+        return encoder_layer(a.passes, not a.unfused, a.attention)
     shape = synth.FFNShape("profile", a.tokens, 1024, 4096)
     tensors = [torch.from_numpy(t).cuda() for t in synth.ffn_tensors(shape, seed=0)]
     blk = ffn.UnitScaledFFN(shape.tokens, shape.d_model, shape.d_ff, operand=a.operand)

@@ -112,3 +112,42 @@ def test_residual_and_attention_scale_helpers(lib):
         assert c["alpha_c"] == c["beta_P"] == f32(alc) and f32(bxc) == f32(alc)
     with pytest.raises(lib.UnitScaleError):
         lib.us_scales_attention(0, 64)
+
+
+def test_attention_entry_points_validate_before_any_launch(lib):
+    """Host checks of us_attention_fwd / us_attention_bwd (0 OK, 1 invalid argument, 2 unsupported, 3 alignment,
+    4 workspace); nothing is launched, so fake device addresses are safe."""
+    raw = lib.raw()
+    M = lambda addr, dt, r, c, ld=None: lib.us_mat(addr, dt, r, c, ld or c)
+    q, k, v = M(0x10000, lib.US_BF16, 128, 64), M(0x20000, lib.US_BF16, 256, 64), M(0x30000, lib.US_BF16, 256, 64)
+    c, p = M(0x40000, lib.US_E4M3, 128, 64), M(0x50000, lib.US_BF16, 128, 256)
+    bt = lib.attention_batch((1, 1), (0, 0), (0, 0), (0, 0), (0, 0))
+    ws = (0x60000, 256)
+    call = lambda Q, K, V, Cx, P, a=0.125, sm=256.0, w=ws, b=bt: raw.us_attention_fwd(
+        C.byref(Q), C.byref(K), C.byref(V), a, sm, 0.0625, C.byref(Cx), C.byref(P) if P is not None else None, C.byref(b), w[0], w[1], None)
+    assert call(q, k, M(0x30000, lib.US_BF16, 128, 64), c, p) == 1              # V rows differ from K rows
+    assert call(q, k, v, M(0x40000, lib.US_E4M3, 64, 64), p) == 1               # context rows differ from query rows
+    assert call(q, k, v, c, M(0x50000, lib.US_BF16, 128, 128)) == 1             # P is not s_q x s_k
+    assert call(q, k, v, c, p, a=0.0) == 1                                      # scales must be positive
+    assert call(q, k, v, c, M(0x50000, lib.US_F16, 128, 256)) == 2              # P in another format than the operands
+    assert call(q, M(0x20000, lib.US_F16, 256, 64), v, c, p) == 2               # mixed operand formats
+    w128 = lambda a: M(a, lib.US_BF16, 128, 128)
+    assert call(w128(0x10000), w128(0x20000), w128(0x30000), w128(0x40000), None) == 2        # head width 128
+    assert call(q, M(0x20000, lib.US_BF16, 1024, 64), M(0x30000, lib.US_BF16, 1024, 64), c, None) == 2   # more than 512 keys
+    assert call(q, k, v, c, p, w=(None, 0)) == 4                                # no workspace
+    assert call(M(0x10002, lib.US_BF16, 128, 64), k, v, c, p) == 3              # misaligned base address
+    assert call(q, k, v, c, M(0x50000, lib.US_BF16, 128, 256, 260)) == 3        # row pitch of P not a multiple of 16 bytes
+    many = lib.attention_batch((2, 2), (0, 64), (8192, 64), (8192, 64), (8192, 64), (65536, 32768))
+    assert call(q, k, v, c, p, b=many) == 1                                     # zero stride with more than one problem
+    assert call(M(0x10000, lib.US_BF16, 0, 64), k, v, M(0x40000, lib.US_E4M3, 0, 64), None) == 0   # no queries: nothing to do
+
+    dc, ds, dq = M(0x70000, lib.US_BF16, 128, 64), M(0x80000, lib.US_BF16, 128, 256), M(0x90000, lib.US_BF16, 128, 64)
+    btb = lib.attention_bwd_batch((1, 1), *[(0, 0)] * 6)
+    bcall = lambda dC, P, K, V, dS, dQ, alpha=256.0: raw.us_attention_bwd(
+        C.byref(dC), C.byref(P), C.byref(K), C.byref(V), 0.125, alpha, 256.0, 0.125, C.byref(dS), C.byref(dQ), C.byref(btb), ws[0], ws[1], None)
+    assert bcall(dc, p, k, v, M(0x80000, lib.US_BF16, 128, 128), dq) == 1       # dS is not s_q x s_k
+    assert bcall(dc, p, k, v, ds, dq, alpha=0.0) == 1
+    assert bcall(dc, p, k, v, M(0x80000, lib.US_E5M2, 128, 256), dq) == 2       # 16-bit operands with an FP8 dS
+    e5 = lambda a, r, cc: M(a, lib.US_E5M2, r, cc)
+    e4 = lambda a, r, cc: M(a, lib.US_E4M3, r, cc)
+    assert bcall(e5(0x70000, 128, 64), e5(0x50000, 128, 256), e4(0x20000, 256, 64), e4(0x30000, 256, 64), e5(0x80000, 128, 256), dq) == 2   # P must be E4M3
