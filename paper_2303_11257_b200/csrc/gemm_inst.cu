@@ -103,8 +103,12 @@ static us_status pick_epilogue(const us_mat* A, const us_mat* B, const GemmParam
 template <int ES, bool A_MN, bool B_MN>
 us_status launch_gemm(const us_mat* A, const us_mat* B, GemmParams& p, const EpiMats& em, int epi, const BatchDesc& bd,
                       cudaStream_t stream) {
-  // CTA pairs with 256 x 256 tiles whenever such a tile is not mostly empty; 128 x 128 tiles otherwise.
-  const bool pair = p.N > 128 && p.M > kBM;
+  // CTA pairs with 256 x 256 tiles whenever such a tile is not mostly empty and there are enough of them to occupy at
+  // least half of the machine's CTA pairs; 128 x 128 tiles otherwise (a 1024 x 1024 output is 16 pair tiles on 74
+  // pairs, but 64 single-CTA tiles).
+  const int sms = host::sm_count();
+  const long long pair_tiles = (long long)((p.M + 2 * kBM - 1) / (2 * kBM)) * ((p.N + 255) / 256) * bd.nb0 * bd.nb1;
+  const bool pair = p.N > 128 && p.M > kBM && (sms <= 0 || 4 * pair_tiles >= sms);
   const int bn = pair ? 256 : 128, cg = pair ? 2 : 1;
   p.tiles_m = (p.M + kBM * cg - 1) / (kBM * cg);
   p.tiles_n = (p.N + bn - 1) / bn;
