@@ -280,3 +280,31 @@ def test_backward_fp8_operands(nseq, nhead, s):
     gq = U.host_values(dQ)
     dq = U.code_distance(F.quantise_codes(gq, fm), F.quantise_codes(ref_q, fm), "e5m2")
     assert ((dq <= 1) | (np.abs(gq - F.quantise(ref_q, fm)) <= TOL * max(1.0, np.abs(ref_q).max()))).all()
+
+
+def test_separate_contiguous_operands_and_repeatability():
+    """Q, K, V as three contiguous [problems * s x 64] tensors (strides of a different shape than the packed QKV matrix),
+    different query and key counts, and bit-identical outputs from two launches (no atomics anywhere)."""
+    from paper_2303_11257_b200 import lib as L, synth
+    nb0, nb1, s_q, s_k = 2, 3, 200, 328
+    n = nb0 * nb1
+    q, k, v = (synth.normal(81, i, (n * r, 64)) for i, r in ((0, s_q), (1, s_k), (2, s_k)))
+    Q, K, V = U.to_device(q, "bf16"), U.to_device(k, "bf16"), U.to_device(v, "bf16")
+    ws = L.new_workspace()
+    a_s, sm, a_c = 0.125, float(s_k), s_k ** -0.5
+    bt = L.attention_batch((nb0, nb1), (nb1 * s_q * 64, s_q * 64), (nb1 * s_k * 64, s_k * 64), (nb1 * s_k * 64, s_k * 64),
+                           (nb1 * s_q * 64, s_q * 64), (nb1 * s_q * s_k, s_q * s_k))
+    outs = []
+    for _ in range(2):
+        Cx, P = U.empty(n * s_q, 64, "bf16"), U.empty(n * s_q, s_k, "bf16")
+        L.us_attention_fwd(Q[:s_q], K[:s_k], V[:s_k], a_s, sm, a_c, Cx[:s_q], P[:s_q], bt, ws)
+        assert L.us_workspace_status(ws) == 0
+        outs.append((U.codes_of(Cx), U.codes_of(P)))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    qv, kv, vv = (U.values_of(t, "bf16") for t in (q, k, v))
+    p_ref, _ = O.attention_fwd(qv.reshape(n, s_q, 64), kv.reshape(n, s_k, 64), vv.reshape(n, s_k, 64), a_s, sm, a_c, "f64")
+    p_dev = U.host_values(P).reshape(n, s_q, s_k)
+    assert (np.abs(p_dev - p_ref) <= U.ulp_of(p_ref, "bf16") + 3e-6 * sm).all()
+    c_ref = np.float64(np.float32(a_c)) * (p_dev @ vv.reshape(n, s_k, 64))
+    got = U.host_values(Cx).reshape(n, s_q, 64)
+    assert (np.abs(got - c_ref) <= TOL * max(1.0, np.abs(c_ref).max()) + U.ulp_of(c_ref, "bf16")).all()
