@@ -308,3 +308,38 @@ def test_separate_contiguous_operands_and_repeatability():
     c_ref = np.float64(np.float32(a_c)) * (p_dev @ vv.reshape(n, s_k, 64))
     got = U.host_values(Cx).reshape(n, s_q, 64)
     assert (np.abs(got - c_ref) <= TOL * max(1.0, np.abs(c_ref).max()) + U.ulp_of(c_ref, "bf16")).all()
+
+
+@pytest.mark.parametrize("s_q,s_k", [(100, 100), (37, 413), (130, 33)])
+def test_lengths_that_are_not_multiples_of_eight(s_q, s_k):
+    """Key counts that end inside a 32-column chunk and inside a 16-byte piece (masking of the zero-filled key rows);
+    P goes to a padded buffer so that its row pitch stays a multiple of 16 bytes."""
+    from paper_2303_11257_b200 import lib as L, synth
+    q, k, v = synth.normal(82, 0, (s_q, 64)), synth.normal(82, 1, (s_k, 64)), synth.normal(82, 2, (s_k, 64))
+    Q, K, V = U.to_device(q, "fp16"), U.to_device(k, "fp16"), U.to_device(v, "fp16")
+    ld = (s_k + 7) // 8 * 8
+    P = U.empty(s_q, s_k, "fp16", ld=ld)
+    Cx = U.empty(s_q, 64, "f32")
+    ws = L.new_workspace()
+    a_s, sm, a_c = 0.125, float(s_k), s_k ** -0.5
+    bt = L.attention_batch((1, 1), (0, 0), (0, 0), (0, 0), (0, 0))
+    L.us_attention_fwd(Q, K, V, a_s, sm, a_c, Cx, P, bt, ws)
+    assert L.us_workspace_status(ws) == 0
+    qv, kv, vv = (U.values_of(t, "fp16") for t in (q, k, v))
+    p_ref, _ = O.attention_fwd(qv, kv, vv, a_s, sm, a_c, "f64")
+    p_dev = U.host_values(P)
+    assert (np.abs(p_dev - p_ref) <= U.ulp_of(p_ref, "fp16") + 3e-6 * sm).all()
+    c_ref = np.float64(np.float32(a_c)) * (p_dev @ vv)
+    assert np.abs(U.host_values(Cx) - c_ref).max() <= TOL * max(1.0, np.abs(c_ref).max())
+    # backward on the same problem
+    dc = synth.normal(82, 3, (s_q, 64))
+    dCt, dS, dQ = U.to_device(dc, "fp16"), U.empty(s_q, s_k, "fp16", ld=ld), U.empty(s_q, 64, "f32")
+    btb = L.attention_bwd_batch((1, 1), *[(0, 0)] * 6)
+    L.us_attention_bwd(dCt, P, K, V, 0.125, sm, sm, 0.125, dS, dQ, btb, ws)
+    assert L.us_workspace_status(ws) == 0
+    dp = 0.125 * (U.values_of(dc, "fp16") @ vv.T)
+    ref = O.softmax_bwd(p_dev, dp, sm, sm)
+    got = U.host_values(dS)
+    assert (np.abs(got - ref) <= U.ulp_of(ref, "fp16") + 3e-6 * (np.abs(ref).max() + np.abs(dp).max())).all()
+    ref_q = 0.125 * (got @ kv)
+    assert np.abs(U.host_values(dQ) - ref_q).max() <= TOL * max(1.0, np.abs(ref_q).max())
