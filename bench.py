@@ -162,6 +162,7 @@ class ClockSampler:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         sm, smax, power, reasons = [], [], [], set()
+        parsed = []
         for ts, line in list(self.lines):
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
@@ -171,19 +172,33 @@ class ClockSampler:
             except ValueError:
                 continue
             smax.append(mx)
-            if any(t0 <= ts <= t1 + 0.06 for t0, t1 in windows):
-                sm.append(clk)
-                power.append(pw)
-                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
-        return {
+            parsed.append((ts, clk, pw, parts[5:9]))
+        inside = [r for r in parsed if any(t0 <= r[0] <= t1 + 0.06 for t0, t1 in windows)]
+        note = None
+        if not inside and parsed and windows:
+            # a timed region of a few milliseconds can fall between two samples (20 ms apart): take the nearest one
+            # (the warm-up steps run right before the region, so the GPU is under the same load there)
+            dist = lambda r: min(max(t0 - r[0], r[0] - t1, 0.0) for t0, t1 in windows)
+            best = min(parsed, key=dist)
+            if dist(best) <= 0.25:
+                inside = [best]
+                note = f"no sample inside the timed region; nearest one, {dist(best) * 1e3:.0f} ms away"
+        for ts, clk, pw, flags in inside:
+            sm.append(clk)
+            power.append(pw)
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), flags):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        out = {
             "sm_mhz": statistics.median(sm) if sm else None,
             "sm_max_mhz": max(smax) if smax else None,
             "power_w_max": max(power) if power else None,
             "samples_under_load": len(sm),
             "reasons": sorted(reasons),
         }
+        if note:
+            out["note"] = note
+        return out
 
 
 # ----------------------------------------------------------------------------- oracle legs (host cores)
