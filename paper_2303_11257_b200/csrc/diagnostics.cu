@@ -2,9 +2,9 @@
 // formats for deep learning", paragraph "Quantisation error": SNR = E[X^2] / E[(q(X) - X)^2]) and the
 // histogram of floor(log2 |x|) (appendix "Histograms of tensor-scaling within BERT").
 //
-// One pass over the tensor (an analysis tool, not on the training path: element-wise loads and a per-element
-// shared-memory histogram update; no bandwidth figure is claimed for it).  Every CTA accumulates its sums in double precision and its bin
-// counts in shared-memory integers, and writes one partial record to the caller's workspace; a second,
+// One pass over the tensor (an analysis tool, not on the training path: 128-bit loads where the tensor has no row
+// padding, a per-element update of a per-warp shared-memory histogram; bound by those updates and the double-precision
+// sums, not by memory).  Every CTA accumulates its sums in double precision and its bin counts in shared-memory integers, and writes one partial record to the caller's workspace; a second,
 // single-CTA kernel adds the records in order.  No global atomics and nothing to zero beforehand: the
 // result is the same from run to run.
 #include "common.cuh"
@@ -22,6 +22,7 @@ struct DiagArgs {
   float scale;
   int fmt;                 // format whose rounding error is measured
   int exp_lo, nbins;
+  int vec_ok;              // no row padding and a 16-byte aligned base: 128-bit loads
   unsigned long long* partial;   // [gridDim.x][kDiagRecord]
 };
 
@@ -34,15 +35,15 @@ __device__ __forceinline__ float round_to(float v, int fmt) {
 }
 
 __global__ void __launch_bounds__(kDiagThreads) quant_stats_kernel(const DiagArgs a) {
-  __shared__ unsigned int bins[kDiagMaxBins + 2];
+  // one histogram per warp (less contention on the few popular bins), added in warp order at the end
+  __shared__ unsigned int bins[kDiagThreads / 32][kDiagMaxBins + 2];
   __shared__ double warp_sums[2][kDiagThreads / 32];
-  for (int i = threadIdx.x; i < a.nbins + 2; i += kDiagThreads) bins[i] = 0u;
+  for (int i = threadIdx.x; i < (kDiagThreads / 32) * (kDiagMaxBins + 2); i += kDiagThreads) (&bins[0][0])[i] = 0u;
   __syncthreads();
+  unsigned int* my_bins = bins[threadIdx.x >> 5];
   double s_sig = 0.0, s_err = 0.0;
-  const int64_t total = a.rows * a.cols;
-  for (int64_t i = blockIdx.x * (int64_t)kDiagThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kDiagThreads) {
-    const int64_t r = i / a.cols, c = i - r * a.cols;
-    const float v = a.scale * load_one(a.src, a.src_dt, r * a.ld + c);
+  auto take = [&](float x) {
+    const float v = a.scale * x;
     const float e = round_to(v, a.fmt) - v;
     s_sig += (double)v * (double)v;
     s_err += (double)e * (double)e;
@@ -54,7 +55,25 @@ __global__ void __launch_bounds__(kDiagThreads) quant_stats_kernel(const DiagArg
     else if (ex < a.exp_lo) bin = 0;
     else if (ex >= a.exp_lo + a.nbins) bin = a.nbins + 1;
     else bin = 1 + ex - a.exp_lo;
-    atomicAdd(&bins[bin], 1u);
+    atomicAdd(&my_bins[bin], 1u);
+  };
+  const int64_t total = a.rows * a.cols;
+  if (a.vec_ok) {
+    // no row padding, 16-byte aligned: eight elements per thread and step with 128-bit loads
+    const int64_t chunks = total / 8;
+    const int es = dtype_size(a.src_dt);
+    for (int64_t c = blockIdx.x * (int64_t)kDiagThreads + threadIdx.x; c < chunks; c += (int64_t)gridDim.x * kDiagThreads) {
+      float x[8];
+      load_vec<8>(static_cast<const char*>(a.src) + c * 8 * es, a.src_dt, x);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) take(x[i]);
+    }
+    if (blockIdx.x == 0 && threadIdx.x < (int)(total - chunks * 8)) take(load_one(a.src, a.src_dt, chunks * 8 + threadIdx.x));
+  } else {
+    for (int64_t i = blockIdx.x * (int64_t)kDiagThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kDiagThreads) {
+      const int64_t r = i / a.cols, c = i - r * a.cols;
+      take(load_one(a.src, a.src_dt, r * a.ld + c));
+    }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -69,7 +88,11 @@ __global__ void __launch_bounds__(kDiagThreads) quant_stats_kernel(const DiagArg
     for (int w = 0; w < kDiagThreads / 32; ++w) t += warp_sums[threadIdx.x][w];
     rec[threadIdx.x] = (unsigned long long)__double_as_longlong(t);
   }
-  for (int i = threadIdx.x; i < a.nbins + 2; i += kDiagThreads) rec[2 + i] = bins[i];
+  for (int i = threadIdx.x; i < a.nbins + 2; i += kDiagThreads) {
+    unsigned int t = 0u;
+    for (int w = 0; w < kDiagThreads / 32; ++w) t += bins[w][i];
+    rec[2 + i] = t;
+  }
 }
 
 // sums[0..1] and hist[0 .. nbins + 1]: the CTAs' records added in CTA order.
@@ -121,6 +144,7 @@ extern "C" us_status us_quant_stats(const us_mat* src, float scale, us_dtype fmt
   DiagArgs a{};
   a.src = src->ptr; a.src_dt = src->dtype; a.ld = src->ld; a.rows = src->rows; a.cols = src->cols;
   a.scale = scale; a.fmt = fmt; a.exp_lo = exp_lo; a.nbins = nbins;
+  a.vec_ok = (src->ld == src->cols || src->rows <= 1) && reinterpret_cast<uintptr_t>(src->ptr) % 16 == 0;
   a.partial = static_cast<unsigned long long*>(ws);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   quant_stats_kernel<<<grid, kDiagThreads, 0, st>>>(a);         // an empty tensor still writes one zero record
