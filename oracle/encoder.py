@@ -68,7 +68,8 @@ def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16"
     norm = "post": ln = (w1, c1, w2, c2), each [d]; R1 = LN1(U1), R2 = LN2(U2) with U the residual sums.
     fused_scores: the scores S feed the softmax directly and are never stored, hence never rounded
     (ops.attention_fwd), and likewise the gradient dP of the weights in the backward pass
-    (ops.attention_bwd_scores); r.S and r.dP then hold the unrounded values."""
+    (ops.attention_bwd_scores); r.S and r.dP then hold the unrounded values, and dQ, dK, dV are rounded once, to E5
+    (the format of the one matmul operand they become), instead of first to the attention gradients' format."""
     T, d = X.shape
     hd = d // nhead
     f32 = lambda v: float(np.float32(v))
@@ -135,7 +136,9 @@ def encoder_layer(X, Wqkv, Wo, W1, W2, G, nseq, slen, nhead, tau=0.5, att="bf16"
     dK4 = f32(b_K) * (dS4.transpose(0, 1, 3, 2) @ Q)
     r.dP, r.dS = dP4.reshape(-1, slen), dS4.reshape(-1, slen)
     dQKV = np.concatenate([_unheads(t, nseq, slen, nhead, hd) for t in (dQ4, dK4, dV4)], axis=1)
-    r.dQKV, _ = O.store(dQKV, f_grad)
+    # dQ, dK, dV feed only the QKV projection's backward matmuls, whose gradient operand is E5; with fused_scores they are
+    # written once, in that format, instead of being stored in the attention gradients' format and cast afterwards
+    r.dQKV, _ = O.store(dQKV, "e5m2" if fused_scores else f_grad)
     dQKVq, _ = O.store(r.dQKV, "e5m2")
     ep = O.Epilogue(skip=g1, skip_coef=c_skip, out_coef=c_branch)
     r.dX, _, _ = O.apply_epilogue(O.linear_bwd_x(dQKVq, Wqkv_q, b_qkv), ep, "bf16")

@@ -66,7 +66,9 @@ class UnitScaledEncoderLayer:
         self.dP = None if fused_attention else e(nseq * nhead * slen, slen, wide_dt)
         self.dS = e(nseq * nhead * slen, slen, grad_dt)
         self.dQKVq = e(T, 3 * d, E5)
-        self.dQKV = self.dQKVq if attention == "fp8" else e(T, 3 * d, grad_dt)   # FP8: written as E5M2 directly
+        # dQ, dK, dV are consumed only as the E5M2 operand of the QKV projection's backward GEMMs: with FP8 attention
+        # operands, and with the fused attention kernels, their producers write that format directly (no cast launch)
+        self.dQKV = self.dQKVq if (attention == "fp8" or fused_attention) else e(T, 3 * d, grad_dt)
         self.dX = e(T, d, torch.bfloat16)
         self.dWqkv, self.dWo = e(d, 3 * d, torch.float32), e(d, d, torch.float32)
         self.ws = L.new_workspace(device)
@@ -89,7 +91,7 @@ class UnitScaledEncoderLayer:
         self.bt = dict(scores=L.batch(n, qkv, qkv, sq), ctx=L.batch(n, sq, qkv, td), dP=L.batch(n, td, qkv, sq),
                        dV=L.batch(n, sq, td, qkv), dQ=L.batch(n, sq, qkv, qkv), dK=L.batch(n, sq, qkv, qkv))
         # fused cast, attention forward, FFN forward + backward, attention backward (one cast fewer with FP8 attention)
-        self._launches = 1 + (3 if fused_attention else 5) + 7 + ((10 if attention == "fp8" else 11) - (2 if fused_attention else 0)) + (7 if norm == "post" else 0)
+        self._launches = 1 + (3 if fused_attention else 5) + 7 + ((10 if (attention == "fp8" or fused_attention) else 11) - (2 if fused_attention else 0)) + (7 if norm == "post" else 0)
         self.bt_fused = L.attention_batch(n, qkv, qkv, qkv, td, sq)
         self.bt_fused_bwd = L.attention_bwd_batch(n, td, sq, qkv, qkv, sq, qkv)
 

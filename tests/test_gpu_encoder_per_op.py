@@ -66,6 +66,7 @@ def _per_op(layer, host, problems, rows, wrows):
     Xq, Wqkv_q, Wo_q = H(layer.Xq), H(layer.Wqkv_q), H(layer.Wo_q)
     QKV, Cq = H(layer.QKV), H(layer.Cq)
     f_act, f_grad = _fmt_of(layer.QKV), _fmt_of(layer.dS)
+    f_qkv_grad = _fmt_of(layer.dQKV)          # E5M2 where the producers write the projection GEMMs' operand format directly
     f_wide = _fmt_of(layer.dP) if layer.dP is not None else None
     fused = layer.S is None          # fused attention forward: the scores are never stored
     # ---- QKV projection
@@ -97,14 +98,14 @@ def _per_op(layer, host, problems, rows, wrows):
             dPp = H(layer.dP[pr])
             _check(dPp, ref, f_wide, TOL * max(1.0, np.abs(ref).max()), "dP " + tag)
         ref = O.linear_bwd_w(Pp, dc, sc["beta_V"])
-        _check(dQKV[r, 2 * d + j * hd:2 * d + (j + 1) * hd], ref, f_grad, TOL * max(1.0, np.abs(ref).max()), "dV " + tag)
+        _check(dQKV[r, 2 * d + j * hd:2 * d + (j + 1) * hd], ref, f_qkv_grad, TOL * max(1.0, np.abs(ref).max()), "dV " + tag)
         ref = O.softmax_bwd(Pp, dPp, sc["sm"], sc["sm"])
         scale = np.abs(ref).max() + np.abs(dPp).max()
         _check(dSp, ref, f_grad, 3e-6 * scale * max(1.0, slen / 512), "dS " + tag)
         ref = O.linear_fwd(dSp, k, sc["beta_Q"])
-        _check(dQKV[r, j * hd:(j + 1) * hd], ref, f_grad, TOL * max(1.0, np.abs(ref).max()), "dQ " + tag)
+        _check(dQKV[r, j * hd:(j + 1) * hd], ref, f_qkv_grad, TOL * max(1.0, np.abs(ref).max()), "dQ " + tag)
         ref = O.linear_bwd_w(dSp, q, sc["beta_K"])
-        _check(dQKV[r, d + j * hd:d + (j + 1) * hd], ref, f_grad, TOL * max(1.0, np.abs(ref).max()), "dK " + tag)
+        _check(dQKV[r, d + j * hd:d + (j + 1) * hd], ref, f_qkv_grad, TOL * max(1.0, np.abs(ref).max()), "dK " + tag)
     # ---- output projection with the residual epilogue
     ref = O.weighted_add(X[rows].astype(np.float64), O.linear_fwd(Cq[rows], Wo_q, sc["alpha_o"]), cs, cb)
     _check(H(layer.R1)[rows], ref, "bf16", TOL, "R1")
