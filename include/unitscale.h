@@ -183,6 +183,39 @@ typedef struct {
 } us_linear_call;
 us_status us_linear_group(int count, const us_linear_call* calls, void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * us_ffn_hidden: both GEMMs that end in the hidden layer of the FFN block, as ONE kernel launch.
+ *
+ * The scaled FFN of the figure "PyTorch examples" is linear -> gelu -> linear; with the ops of section
+ * "Example" and the table row "gelu" its hidden layer takes part in
+ *
+ *   forward    H  = alpha  * X W1                 X [b x m], W1 [m x f]       (us_linear_fwd)
+ *              A  = act_out_scale * gelu(act_in_scale * H)                    (its US_ACT_GELU epilogue)
+ *   backward   dA = beta_x * G W2^T               G [b x n], W2 [f x n]       (us_linear_bwd_x)
+ *              dH = grad_out_scale * act_in_scale * gelu'(act_in_scale * H16) * dA   (its US_ACT_GELU_GRAD epilogue)
+ *
+ * where H16 is H rounded to h_dtype (US_BF16 or US_F16), the format in which the two separate calls hand the
+ * pre-activation from the forward to the backward pass.  When the gradient G of the block's output is at hand
+ * before the forward pass starts (a training step whose upstream gradient is an input, as in the benchmark of
+ * the FFN block, or a recomputed block), both GEMMs can run tile by tile side by side: H stays on the SM,
+ * rounded exactly as above, and is never written to or read from memory, which takes 4 bytes per element of
+ * the block's largest tensor off the path.  A and dH are bit-identical to what the two separate calls give.
+ *
+ * X, W1, G, W2: 8-bit operands (any mix of US_E4M3 / US_E5M2).  A, dH [b x f]: 8-bit outputs, rounded once,
+ * saturating.  H: NULL (or ptr NULL), or a [b x f] matrix of h_dtype that receives H16.
+ * Covered: b > 128 and f > 128.  Other valid shapes return US_ERR_UNSUPPORTED and launch nothing: use the
+ * two separate calls.  Alignment, workspace, status word and errors as for us_linear_fwd.
+ */
+us_status us_ffn_hidden(const us_mat* X, const us_mat* W1, float alpha, const us_mat* G, const us_mat* W2, float beta_x,
+                        float act_in_scale, float act_out_scale, float grad_out_scale, int32_t h_dtype, const us_mat* H,
+                        const us_mat* A, const us_mat* dH, void* ws, size_t ws_bytes, void* stream);
+
+/* us_test_ffn_hidden_starved: us_test_linear_fwd_starved for the kernel of us_ffn_hidden (no operand loads, every
+ * device-side wait gives up after `wait_limit` polls, 1 .. 65536): the kernel raises the status word, frees its
+ * tensor memory and returns by itself; A and dH are not valid afterwards.  All scales are 1. */
+us_status us_test_ffn_hidden_starved(const us_mat* X, const us_mat* W1, const us_mat* G, const us_mat* W2, const us_mat* A,
+                                     const us_mat* dH, void* ws, size_t ws_bytes, unsigned int wait_limit, void* stream);
+
 /* Bytes of device workspace the linear ops need. */
 size_t us_workspace_bytes(void);
 

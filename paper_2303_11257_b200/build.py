@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libunitscale.so")
-SOURCES = ["host.cu", "elementwise.cu", "softmax.cu", "layernorm.cu", "diagnostics.cu", "gemm.cu", "gemm_group.cu", "static_ws.cu", "attention.cu"]
+SOURCES = ["host.cu", "elementwise.cu", "softmax.cu", "layernorm.cu", "diagnostics.cu", "gemm.cu", "gemm_group.cu", "ffn_hidden.cu", "static_ws.cu", "attention.cu"]
 # (operand bytes, A MN-major, B MN-major): forward, backward-input, backward-weight for FP8 and 16-bit operands
 GEMM_PARTS = [(1, 0, 1), (1, 0, 0), (1, 1, 1), (2, 0, 1), (2, 0, 0), (2, 1, 1)]
 HEADERS = ["common.cuh", "rowwise.cuh", "sm100.cuh", "gemm_kernel.cuh", "gemm_group.cuh", "gemm_launch.h", "gemm_inst.cu", "host.h", os.path.join("..", "..", "include", "unitscale.h")]

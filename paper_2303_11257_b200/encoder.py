@@ -97,8 +97,9 @@ class UnitScaledEncoderLayer:
 
     @property
     def launches_per_step(self) -> int:
-        """Kernel launches of one step (the FFN block takes three fewer while its grouped launch covers the shape)."""
-        return self._launches - (3 if self.norm is None and self.ffn.grouped else 0)
+        """Kernel launches of one step (without layer norms the FFN block's six GEMMs go out in its grouped forms, as
+        two or three launches, while those cover the shape)."""
+        return self._launches - (6 - self.ffn.gemm_launches if self.norm is None else 0)
 
     def _heads(self, M, which):
         """Problem (0, 0) of a [T x 3d] matrix: rows of the first sequence, columns of head 0 of Q / K / V."""

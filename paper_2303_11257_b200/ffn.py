@@ -16,6 +16,10 @@ Backward, G = dL/dR (the branch output receives G unscaled):
     dW1 = beta_w Xq^T dH                                                  us_linear_bwd_w
 q is E4M3 for activations / weights and E5M2 for gradients in "fp8" mode; in "bf16" / "fp16"
 mode the matmul inputs are rounded to that format instead (no loss scale, same fixed scales).
+
+step() knows G when it starts.  In FP8 mode it therefore issues the two GEMMs that end in the hidden layer (H, A and
+dH above) as one us_ffn_hidden launch, in which H stays on the SM, and the other four GEMMs as one us_linear_group
+launch: three launches per step with the fused cast.  self.H is then written only with keep_h = True.
 """
 from __future__ import annotations
 
@@ -61,7 +65,7 @@ class UnitScaledFFN:
     """Buffers + call sequence for one FFN block of T tokens, width d, hidden width f."""
 
     def __init__(self, T: int, d: int, f: int, scales: FFNScales | None = None, operand: str = "fp8",
-                 h_dtype=torch.bfloat16, io_dtype=torch.bfloat16, device="cuda"):
+                 h_dtype=torch.bfloat16, io_dtype=torch.bfloat16, device="cuda", keep_h: bool = False):
         self.T, self.d, self.f = T, d, f
         self.sc = scales or FFNScales.unit(T, d, f)
         self.operand = operand
@@ -80,7 +84,6 @@ class UnitScaledFFN:
         # step() has all four tensors to quantise at hand when it starts, so in FP8 mode it casts them
         # with one launch; forward() / backward() on their own cast what they are given.
         self.fused_casts = operand == "fp8"
-        self.launches_per_step = 7 if self.fused_casts else 10
         # After the first GEMM, the second forward GEMM, the GELU-gradient GEMM and the first weight-gradient GEMM
         # depend on nothing but it, and the last two GEMMs only on the GELU-gradient one.  step() issues them on
         # three streams, so that the CTAs of one kernel fill the SMs another leaves idle in its last wave (64 or
@@ -90,8 +93,23 @@ class UnitScaledFFN:
         # FP8 operands: the four GEMMs that remain after the GELU-gradient GEMM are independent of one another and
         # go out as one us_linear_group launch (4 launches per step instead of 7).
         self.grouped = operand == "fp8"
-        if self.grouped:
-            self.launches_per_step = 4
+        # FP8 operands and G known up front: the first GEMM + GELU and the GELU-gradient GEMM are one us_ffn_hidden
+        # launch that keeps the pre-activation on the SM; keep_h = True also writes its 16-bit copy to self.H (the
+        # separate launches always do, the backward one reads it from there).
+        self.fused_hidden = operand == "fp8"
+        self.keep_h = keep_h
+
+    @property
+    def gemm_launches(self) -> int:
+        """Launches step_from_casts() makes for the six GEMMs."""
+        return 6 - ((3 + (1 if self.fused_hidden else 0)) if self.grouped else 0)
+
+    @property
+    def launches_per_step(self) -> int:
+        """Kernel launches of step(): the cast(s) plus gemm_launches in FP8 mode."""
+        if self.fused_casts:
+            return 1 + self.gemm_launches
+        return 10
 
     def _cast(self, src, dst, stream):
         if dst.dtype in (torch.float8_e4m3fn, torch.float8_e5m2):
@@ -103,8 +121,9 @@ class UnitScaledFFN:
     def stages(self, X, W1, W2, G, fused_casts: bool | None = None):
         """The launches of one pass, in order, as (name, kind, callable(stream)) triples.
 
-        kind is "cast" or "gemm"; step() runs exactly these (seven with the casts fused into one
-        launch, ten otherwise); forward() and backward() run the unfused ones they need."""
+        kind is "cast" or "gemm".  These are the unfused launches: step() runs exactly these (seven with the casts
+        fused into one launch, ten otherwise) unless it takes the grouped forms (step_launches); forward() and
+        backward() run the ones they need."""
         sc, (c_skip, c_branch) = self.sc, self._c
         fused = self.fused_casts if fused_casts is None else fused_casts
         ep1 = L.epilogue(act=L.US_ACT_GELU, act_in_scale=sc.s_in, act_out_scale=sc.alpha_g, aux=self.H)
@@ -139,6 +158,8 @@ class UnitScaledFFN:
             return [(n, k, 1 if k == "gemm" else 0, fn) for n, k, fn in st]
         by = {n: (k, fn) for n, k, fn in st}
         head = [(n, by[n][0], 1 if by[n][0] == "gemm" else 0, by[n][1]) for n in ("cast_all", "fwd1_gelu", "bwd_x2_gelu_grad")]
+        if self.fused_hidden:
+            head = head[:1] + [("hidden_fwd1_gelu_bwd_x2_gelu_grad", "group", 2, lambda stream=None: self._hidden(stream))]
         return head + [("group_fwd2_bwd_w2_bwd_x1_bwd_w1", "group", 4,
                         lambda stream=None: L.us_linear_group(self.group_calls(X, G), self.ws, stream))]
 
@@ -152,6 +173,12 @@ class UnitScaledFFN:
                 L.linear_call(L.US_OP_BWD_W, self.Xq, self.dHq, sc.beta_w, self.dW1),
                 L.linear_call(L.US_OP_FWD, self.Aq, self.W2q, sc.alpha2, self.R, ep2),
                 L.linear_call(L.US_OP_BWD_X, self.dHq, self.W1q, sc.beta_x1, self.dX, ep5)]
+
+    def _hidden(self, stream=None):
+        """H, A and dH in one launch (us_ffn_hidden) from the quantised operands."""
+        sc = self.sc
+        L.us_ffn_hidden(self.Xq, self.W1q, sc.alpha1, self.Gq, self.W2q, sc.beta_x2, sc.s_in, sc.alpha_g, sc.beta_g,
+                        self.Aq, self.dHq, self.ws, H=self.H if self.keep_h else None, h_dtype=self.H.dtype, stream=stream)
 
     def cast_weights(self, W1, W2, stream=None):
         self._cast(W1, self.W1q, stream)
@@ -228,12 +255,22 @@ class UnitScaledFFN:
         return self.dX, self.dW1, self.dW2
 
     def step_from_casts(self, X, G, stream=None):
-        """The GEMMs of one pass when self.Xq, W1q, W2q, Gq already hold the quantised operands (FP8 mode): three
-        launches -- first GEMM + GELU, GELU-gradient GEMM, the other four as one group.  X and G are the unquantised
-        skip inputs of the two residual epilogues."""
+        """The GEMMs of one pass when self.Xq, W1q, W2q, Gq already hold the quantised operands (FP8 mode): two
+        launches -- the hidden layer's two GEMMs with GELU and GELU gradient, the other four as one group -- or their
+        separate forms where a shape is not covered.  X and G are the unquantised skip inputs of the two residual
+        epilogues."""
         by = {name: fn for name, _, fn in self.stages(X, None, None, G)}
-        by["fwd1_gelu"](stream)
-        by["bwd_x2_gelu_grad"](stream)
+        fused = self.fused_hidden and self.grouped
+        if fused:
+            try:
+                self._hidden(stream)
+            except L.UnitScaleError as e:
+                if e.status != L.US_ERR_UNSUPPORTED:
+                    raise
+                fused = self.fused_hidden = False            # at most 128 tokens or hidden units: nothing was launched
+        if not fused:
+            by["fwd1_gelu"](stream)
+            by["bwd_x2_gelu_grad"](stream)
         if self.grouped:
             try:
                 L.us_linear_group(self.group_calls(X, G), self.ws, stream)
@@ -243,7 +280,7 @@ class UnitScaledFFN:
                     raise
                 # a shape the grouped form does not cover (an output of at most 128 rows or columns): nothing was
                 # launched; the four GEMMs go out one by one, now and in later steps
-                self.grouped, self.launches_per_step = False, 7
+                self.grouped = False
         for name in ("fwd2_residual", "bwd_w2", "bwd_x1_residual", "bwd_w1"):
             by[name](stream)
         return self.dX, self.dW1, self.dW2

@@ -97,6 +97,10 @@ def _load() -> C.CDLL:
     lib.us_test_linear_fwd_starved.restype = C.c_int
     lib.us_linear_group.argtypes = [C.c_int, C.POINTER(us_linear_call), V, SZ, V]
     lib.us_linear_group.restype = C.c_int
+    lib.us_ffn_hidden.argtypes = [MP, MP, F, MP, MP, F, F, F, F, C.c_int32, MP, MP, MP, V, SZ, V]
+    lib.us_ffn_hidden.restype = C.c_int
+    lib.us_test_ffn_hidden_starved.argtypes = [MP, MP, MP, MP, MP, MP, V, SZ, C.c_uint, V]
+    lib.us_test_ffn_hidden_starved.restype = C.c_int
     lib.us_workspace_bytes.argtypes = []
     lib.us_workspace_bytes.restype = SZ
     lib.us_workspace_status.argtypes = [V, V]
@@ -326,6 +330,26 @@ def us_test_linear_fwd_starved(X, W, alpha, Y, ws, wait_limit: int, stream=None)
     whose waits give up after wait_limit polls; the status word in ws is raised and the kernel returns."""
     _check("us_test_linear_fwd_starved",
            _lib.us_test_linear_fwd_starved(C.byref(mat(X)), C.byref(mat(W)), alpha, C.byref(mat(Y)), ws.data_ptr(),
+                                           ws.numel() * ws.element_size(), wait_limit, _stream(stream)))
+
+
+def us_ffn_hidden(X, W1, alpha, G, W2, beta_x, act_in_scale, act_out_scale, grad_out_scale, A, dH, ws,
+                  H=None, h_dtype=torch.bfloat16, stream=None):
+    """Hidden layer of the FFN block, forward and backward, in one launch (see the header): A and dH are written,
+    H (optional) receives the pre-activation rounded to h_dtype."""
+    hp = C.byref(mat(H)) if H is not None else None
+    _check("us_ffn_hidden",
+           _lib.us_ffn_hidden(C.byref(mat(X)), C.byref(mat(W1)), alpha, C.byref(mat(G)), C.byref(mat(W2)), beta_x,
+                              act_in_scale, act_out_scale, grad_out_scale, _TORCH_DTYPES[h_dtype], hp, C.byref(mat(A)),
+                              C.byref(mat(dH)), ws.data_ptr(), ws.numel() * ws.element_size(), _stream(stream)))
+    return A, dH
+
+
+def us_test_ffn_hidden_starved(X, W1, G, W2, A, dH, ws, wait_limit: int, stream=None):
+    """us_test_linear_fwd_starved for the kernel of us_ffn_hidden."""
+    _check("us_test_ffn_hidden_starved",
+           _lib.us_test_ffn_hidden_starved(C.byref(mat(X)), C.byref(mat(W1)), C.byref(mat(G)), C.byref(mat(W2)),
+                                           C.byref(mat(A)), C.byref(mat(dH)), ws.data_ptr(),
                                            ws.numel() * ws.element_size(), wait_limit, _stream(stream)))
 
 

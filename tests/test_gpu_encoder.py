@@ -88,7 +88,7 @@ def test_encoder_layer_fp8_attention(cfg):
     layer, host = _run(nseq, slen, d, nhead, f, seed=43, attention="fp8")
     r = E.encoder_layer(*host, nseq, slen, nhead, att="fp8")
     U.assert_close_stored(layer.QKV, r.QKV, "e4m3", 2e-3, "QKV")
-    assert layer.dQKV is layer.dQKVq and layer.launches_per_step == (20 if layer.ffn.grouped else 23)
+    assert layer.dQKV is layer.dQKVq and layer.launches_per_step == 23 - (6 - layer.ffn.gemm_launches)
 
     def close(got, ref, name, mean_tol):
         g = U.host_values(got)

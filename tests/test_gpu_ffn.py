@@ -20,7 +20,7 @@ def _run(shape, operand, seed=0, sigma_x=1.0, io="bf16"):
     ffn, L, synth = _mods()
     X, W1, W2, G = synth.ffn_tensors(shape, seed, sigma_x)
     blk = ffn.UnitScaledFFN(shape.tokens, shape.d_model, shape.d_ff, operand=operand,
-                            io_dtype=U.TORCH_OF[io])
+                            io_dtype=U.TORCH_OF[io], keep_h=True)
     dev = [torch.from_numpy(t).cuda() for t in (X, W1, W2, G)]
     blk.step(*dev)
     blk.check()
