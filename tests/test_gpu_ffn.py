@@ -112,6 +112,23 @@ def test_ffn_bert_large_full_oracle_chain(bert_large_fp8):
     _compare_chain(blk, r, None, "fp8")
 
 
+def test_ffn_bert_large_step_without_the_kept_pre_activation(bert_large_fp8):
+    """The benchmark's configuration: the hidden-layer launch keeps the pre-activation on the SM and writes no copy
+    (keep_h = False).  Every stored tensor must equal, bit for bit, the run above that also wrote the copy and
+    was compared with the oracle; the H buffer stays untouched."""
+    ffn, L, synth = _mods()
+    shape, ref, tensors = bert_large_fp8
+    blk = ffn.UnitScaledFFN(shape.tokens, shape.d_model, shape.d_ff)
+    assert blk.fused_hidden and not blk.keep_h and blk.launches_per_step == 3
+    blk.H.fill_(-7.0)
+    blk.step(*[torch.from_numpy(t).cuda() for t in tensors])
+    blk.check()
+    for name in ("Xq", "W1q", "W2q", "Gq", "Aq", "dHq", "R", "dX", "dW1", "dW2"):
+        a, b = getattr(blk, name), getattr(ref, name)
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), name
+    assert bool((blk.H == -7.0).all())
+
+
 @pytest.mark.parametrize("sigma", [2.0 ** 8, 2.0 ** -8])
 def test_ffn_saturation_and_underflow_in_fused_cast(sigma):
     """X ~ N(0, sigma^2): sigma = 2^8 saturates part of q_E4(X) and of the fused A cast; sigma = 2^-8
