@@ -12,7 +12,7 @@
 // one 256 x 256 output tile, first X W1 into accumulator 0 and then G W2^T into accumulator 1 of
 // tensor memory.  The sixteen epilogue warps turn accumulator 0 into A (stored as FP8) while the MMAs
 // of accumulator 1 run, keep H -- rounded to the 16-bit format the unfused path stores it in -- in
-// their staging memory, and turn accumulator 1 into dH while the next tile's X W1 runs: the two
+// registers, and turn accumulator 1 into dH while the next tile's X W1 runs: the two
 // accumulators alternate exactly as two consecutive tiles of gemm_kernel do, and H never leaves the SM
 // (unless the caller asks for a copy).  Results are bit-identical to us_linear_fwd + GELU epilogue
 // followed by us_linear_bwd_x + GELU-gradient epilogue.
@@ -25,7 +25,19 @@ namespace us {
 namespace {
 
 constexpr int kHidEW = 16;
-using HidSmem = GemmSmem<256, 2, kHidEW>;
+// Shared-memory plan: 32 KB operand stages (this CTA's 128 rows of A and 128 rows of B, 128 bytes of K each) and one
+// 32-row x 64-byte output box per epilogue warp.  The kept pre-activation lives in registers, which leaves room for
+// six stages.
+struct HidSmem {
+  static constexpr int kABytes = kBM * kStageKBytes;
+  static constexpr int kBBytes = 128 * kStageKBytes;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kEpiWarpBytes = 2048;
+  static constexpr int kEpiBytes = kHidEW * kEpiWarpBytes;
+  static constexpr int kStages = (229376 - kEpiBytes) / kStageBytes;
+  static constexpr int kBarrierBytes = 512;
+  static constexpr int kTotal = kStages * kStageBytes + kEpiBytes + kBarrierBytes + 1024;   // + alignment slack
+};
 
 struct HiddenParams {
   int M, N, K1, K2;                 // outputs are [M x N]; contraction lengths of X W1 and of G W2^T
@@ -34,7 +46,7 @@ struct HiddenParams {
   uint32_t idesc1, idesc2;
   float scale1, scale2;             // alpha, beta_x
   float act_in, act_out, grad_out;  // s_in, alpha_g, beta_g
-  int keep_h;                       // the rounded pre-activation is also written to global memory
+  uint8_t* h_ptr; long long h_ld;   // optional copy of the rounded pre-activation (NULL: none); ld in elements
   unsigned int* status;
   uint32_t wait_limit;
   int no_loads;                     // test hook: no operand loads are issued, so that the waits run out
@@ -45,7 +57,7 @@ __global__ void __launch_bounds__(gemm_threads(kHidEW), 1)
 ffn_hidden_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w1,
                   const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_w2,
                   const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_dh,
-                  const __grid_constant__ CUtensorMap tm_h, const HiddenParams p) {
+                  const HiddenParams p) {
   using S = HidSmem;
   constexpr int BN = 256, kBK = 128;
   constexpr uint32_t kChunkBytes = kBK * 128;       // an MN-major operand tile: 128 rows of K x 128 bytes
@@ -183,12 +195,11 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     }
   } else {
     // ------------------------------------------------------------ epilogue warps
-    // Warp (lane quarter q, part) owns 32 rows x 64 columns of the tile.  Staging (6 KB): [0, 4096) the
-    // rounded pre-activation, 32 rows x 128 bytes, 128-byte swizzle (lane l writes and reads row l only);
-    // [4096, 6144) the FP8 output box, 32 rows x 64 bytes, 64-byte swizzle.
+    // Warp (lane quarter q, part) owns 32 rows x 64 columns of the tile; a lane holds one row of them.  The rounded
+    // pre-activation of a tile stays in 32 registers of packed 16-bit pairs (hst) between the two phases; staging
+    // is one FP8 output box of 32 rows x 64 bytes (64-byte swizzle) per warp.
     const int q = warp & 3, part = (warp - 2) >> 2;
-    const uint32_t buf_h = epi_base + (warp - 2) * epi_warp_bytes(kHidEW), buf_out = buf_h + 4096u;
-    const uint32_t row128 = (uint32_t)lane * 128u, sw128 = (uint32_t)(lane & 7);
+    const uint32_t buf_out = epi_base + (warp - 2) * S::kEpiWarpBytes;
     const uint32_t row64 = (uint32_t)lane * 64u, sw64 = (uint32_t)((lane >> 1) & 3);
     const f32x2 s1 = splat2(p.scale1), s2 = splat2(p.scale2), in2 = splat2(p.act_in), os2 = splat2(p.grad_out * p.act_in);
     const float tail_k = fabsf(p.act_in) * (1.0f / kTailRange), act_oi = p.act_out * p.act_in;
@@ -198,22 +209,21 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(ptx::in_even_cta(acc_empty_bar(a)));
     };
+    uint32_t hst[32];
     // One 32-column slice s of accumulator 0: scale, keep round16(H), GELU, round, stage.
     auto slice_fwd = [&](const uint32_t (&r)[32], int s) {
       uint32_t held[2];
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
         f32x2 x[4];
-        uint32_t w[4];
         float y[8];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           x[k] = mul2(pack2(__uint_as_float(r[8 * g + 2 * k]), __uint_as_float(r[8 * g + 2 * k + 1])), s1);
           float a, b;
           unpack2(x[k], a, b);
-          w[k] = H_BF16 ? pack_bf16x2(a, b) : pack_f16x2(a, b);
+          hst[16 * s + 4 * g + k] = H_BF16 ? pack_bf16x2(a, b) : pack_f16x2(a, b);
         }
-        ptx::sts128(buf_h + row128 + ((((uint32_t)(4 * s + g)) ^ sw128) << 4), make_uint4(w[0], w[1], w[2], w[3]));
 #pragma unroll
         for (int k = 0; k < 4; ++k) gelu_scaled2<true>(x[k], tail_k, act_oi, y[2 * k], y[2 * k + 1]);
         const uint32_t lo = cvt_fp8x4<A_E5>(y[0], y[1], y[2], y[3]);
@@ -227,13 +237,11 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       uint32_t held[2];
 #pragma unroll
       for (int g = 0; g < 4; ++g) {
-        const uint4 raw = ptx::lds128(buf_h + row128 + ((((uint32_t)(4 * s + g)) ^ sw128) << 4));
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
         float y[8];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const f32x2 x = mul2(pack2(__uint_as_float(r[8 * g + 2 * k]), __uint_as_float(r[8 * g + 2 * k + 1])), s2);
-          const float2 h = H_BF16 ? unpack_bf16x2(w[k]) : unpack_f16x2(w[k]);
+          const float2 h = H_BF16 ? unpack_bf16x2(hst[16 * s + 4 * g + k]) : unpack_f16x2(hst[16 * s + 4 * g + k]);
           unpack2(gelu_grad_scaled2(pack2(h.x, h.y), x, in2, os2), y[2 * k], y[2 * k + 1]);
         }
         const uint32_t lo = cvt_fp8x4<D_E5>(y[0], y[1], y[2], y[3]);
@@ -271,11 +279,26 @@ ffn_hidden_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         release_acc(sub);                                       // the values are in registers
         if (active) {
           if (sub == 0) slice_fwd(r1, 1); else slice_bwd(r1, 1);
+          if (sub == 0 && p.h_ptr != nullptr && row0 + lane < p.M) {
+            // the copy of the rounded pre-activation: this lane's 64 columns, 8 at a time (16 aligned bytes)
+            uint8_t* dst = p.h_ptr + ((long long)(row0 + lane) * p.h_ld + n_w) * 2;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const int col = n_w + 8 * c;
+              if (col + 8 <= p.N) {
+                *reinterpret_cast<uint4*>(dst + 16 * c) = make_uint4(hst[4 * c], hst[4 * c + 1], hst[4 * c + 2], hst[4 * c + 3]);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                  if (col + j < p.N)
+                    *reinterpret_cast<uint16_t*>(dst + 16 * c + 2 * j) = (uint16_t)(hst[4 * c + (j >> 1)] >> (16 * (j & 1)));
+              }
+            }
+          }
           ptx::fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
             if (sub == 0) {
-              if (p.keep_h) ptx::tma_store_2d(&tm_h, buf_h, n_w, row0);
               ptx::tma_store_2d(&tm_a, buf_out, n_w, row0);
             } else {
               ptx::tma_store_2d(&tm_dh, buf_out, n_w, row0);
@@ -340,7 +363,7 @@ us_status launch_hidden(const CUtensorMap* t, const HiddenParams& p, int grid, c
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, t[0], t[1], t[2], t[3], t[4], t[5], t[6], p) == cudaSuccess ? US_OK : US_ERR_CUDA;
+  return cudaLaunchKernelEx(&cfg, kern, t[0], t[1], t[2], t[3], t[4], t[5], p) == cudaSuccess ? US_OK : US_ERR_CUDA;
 }
 
 us_status hidden_impl(const us_mat* X, const us_mat* W1, float alpha, const us_mat* G, const us_mat* W2, float beta_x,
@@ -373,17 +396,16 @@ us_status hidden_impl(const us_mat* X, const us_mat* W1, float alpha, const us_m
   p.idesc2 = make_idesc(G->dtype == US_E5M2, W2->dtype == US_E5M2, false, false, 256, 256);
   p.scale1 = alpha; p.scale2 = beta_x;
   p.act_in = act_in_scale; p.act_out = act_out_scale; p.grad_out = grad_out_scale;
-  p.keep_h = keep_h;
+  p.h_ptr = keep_h ? static_cast<uint8_t*>(H->ptr) : nullptr;
+  p.h_ld = keep_h ? H->ld : 0;
   p.status = static_cast<unsigned int*>(ws);
   p.wait_limit = wait_limit;
   p.no_loads = no_loads;
 
-  CUtensorMap t[7];
+  CUtensorMap t[6];
   if (!make_tmap(&t[0], X, 1, 128, 128) || !make_tmap(&t[1], W1, 1, 128, 128) || !make_tmap(&t[2], G, 1, 128, 128) ||
       !make_tmap(&t[3], W2, 1, 128, 128) || !make_tmap(&t[4], A, 1, 32, 64) || !make_tmap(&t[5], dH, 1, 32, 64))
     return US_ERR_CUDA;
-  t[6] = t[4];
-  if (keep_h && !make_tmap(&t[6], H, 2, 32, 128)) return US_ERR_CUDA;
 
   const int sms = host::sm_count();
   if (sms <= 0) return US_ERR_CUDA;
