@@ -151,3 +151,35 @@ def test_attention_entry_points_validate_before_any_launch(lib):
     e5 = lambda a, r, cc: M(a, lib.US_E5M2, r, cc)
     e4 = lambda a, r, cc: M(a, lib.US_E4M3, r, cc)
     assert bcall(e5(0x70000, 128, 64), e5(0x50000, 128, 256), e4(0x20000, 256, 64), e4(0x30000, 256, 64), e5(0x80000, 128, 256), dq) == 2   # P must be E4M3
+
+
+def test_ffn_hidden_validates_before_any_launch(lib):
+    """Host checks of us_ffn_hidden (1 invalid argument, 2 unsupported, 3 alignment, 4 workspace): nothing is
+    launched, so fake device addresses are safe."""
+    raw = lib.raw()
+    M = lambda addr, dt, r, c, ld=None: lib.us_mat(addr, dt, r, c, ld or c)
+    E4, E5, BF = lib.US_E4M3, lib.US_E5M2, lib.US_BF16
+    X, W1, G, W2 = M(0x10000, E4, 272, 144), M(0x20000, E4, 144, 400), M(0x30000, E5, 272, 208), M(0x40000, E4, 400, 208)
+    A, dH = M(0x50000, E4, 272, 400), M(0x60000, E5, 272, 400)
+    ws = (0x70000, 256)
+
+    def call(X=X, W1=W1, G=G, W2=W2, A=A, dH=dH, H=None, h_dtype=BF, w=ws):
+        return raw.us_ffn_hidden(C.byref(X), C.byref(W1), 1.0, C.byref(G), C.byref(W2), 1.0, 1.0, 1.7, 1.5, h_dtype,
+                                 C.byref(H) if H is not None else None, C.byref(A), C.byref(dH), w[0], w[1], None)
+
+    assert call(X=M(None, E4, 272, 144)) == 1                                   # null data pointer
+    assert call(W1=M(0x20000, E4, 160, 400)) == 1                               # contraction lengths disagree
+    assert call(G=M(0x30000, E5, 256, 208)) == 1                                # token counts disagree
+    assert call(W2=M(0x40000, E4, 400, 224)) == 1                               # second contraction lengths disagree
+    assert call(dH=M(0x60000, E5, 272, 384)) == 1                               # output shape
+    assert call(h_dtype=lib.US_F32) == 1                                        # the kept format is BF16 or F16
+    assert call(H=M(0x80000, lib.US_F16, 272, 400)) == 1                        # copy in another format than h_dtype
+    assert call(w=(None, 0)) == 4                                               # no workspace
+    assert call(X=M(0x10008, E4, 272, 144)) == 3                                # misaligned base address
+    assert call(A=M(0x50000, E4, 272, 400, 408)) == 3                           # row pitch not a multiple of 16 bytes
+    assert call(X=M(0x10000, BF, 272, 144)) == 2                                # 16-bit operands: use the separate calls
+    assert call(dH=M(0x60000, BF, 272, 400)) == 2                               # outputs are 8-bit
+    small = dict(X=M(0x10000, E4, 128, 144), G=M(0x30000, E5, 128, 208), A=M(0x50000, E4, 128, 400), dH=M(0x60000, E5, 128, 400))
+    assert call(**small) == 2                                                   # at most 128 tokens: use the separate calls
+    assert raw.us_test_ffn_hidden_starved(C.byref(X), C.byref(W1), C.byref(G), C.byref(W2), C.byref(A), C.byref(dH),
+                                          ws[0], ws[1], 0, None) == 1           # wait limit out of range
